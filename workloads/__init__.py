@@ -1,0 +1,245 @@
+"""Seeded synthetic inputs for CHOCO-Gossip / CHOCO-SGD runs.
+
+This module only *builds inputs*: communication graphs with their mixing
+matrices in CSR form, initial iterates, gradient pools and the convex
+logistic-regression problem.  It holds none of the method's arithmetic (no
+compression operator, no gossip update), so that the CPU oracle and the CUDA
+library can both be fed from it without sharing any of the code under test.
+
+Mixing weights follow the rule the paper's experiments use (Section 3, below
+Assumption 1): w_ij = 1 / max(deg(i), deg(j)) on edges, with the self-loop
+counted in the degree, and the diagonal filled so that rows sum to one.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Optional
+
+import numpy as np
+
+# --------------------------------------------------------------------------
+# graphs -> mixing matrix W in CSR (diagonal stored, columns ascending)
+# --------------------------------------------------------------------------
+
+
+@dataclasses.dataclass(frozen=True)
+class MixingCSR:
+    """W as CSR over n rows: int32 row_ptr[n+1], int32 col[nnz], float32 val[nnz]."""
+
+    n: int
+    row_ptr: np.ndarray
+    col: np.ndarray
+    val: np.ndarray
+
+    def dense(self, dtype=np.float64) -> np.ndarray:
+        w = np.zeros((self.n, self.n), dtype=dtype)
+        for i in range(self.n):
+            for e in range(self.row_ptr[i], self.row_ptr[i + 1]):
+                w[i, self.col[e]] = self.val[e]
+        return w
+
+
+def _csr_from_neighbours(neigh: list[set[int]]) -> MixingCSR:
+    """Edge sets (without self) -> max-degree weights, self-loop counted in deg."""
+    n = len(neigh)
+    deg = [len(s) + 1 for s in neigh]          # +1: the self-loop {i} is an edge
+    row_ptr = np.zeros(n + 1, dtype=np.int32)
+    cols: list[int] = []
+    vals: list[float] = []
+    for i in range(n):
+        off = {j: 1.0 / max(deg[i], deg[j]) for j in neigh[i]}
+        diag = 1.0 - sum(off.values())
+        row = dict(off)
+        row[i] = diag
+        for j in sorted(row):
+            cols.append(j)
+            vals.append(row[j])
+        row_ptr[i + 1] = len(cols)
+    return MixingCSR(n, row_ptr, np.asarray(cols, dtype=np.int32),
+                     np.asarray(vals, dtype=np.float32))
+
+
+def ring(n: int) -> MixingCSR:
+    """Ring of n nodes; for n >= 3 every weight is 1/3 (self and both neighbours)."""
+    neigh = [set() for _ in range(n)]
+    for i in range(n):
+        for j in ((i - 1) % n, (i + 1) % n):
+            if j != i:
+                neigh[i].add(j)
+    return _csr_from_neighbours(neigh)
+
+
+def torus(rows: int, cols: int) -> MixingCSR:
+    """2-D torus; duplicate neighbours (side length 2) are merged, so the 2x2
+    torus is the 4-ring.  For sides >= 3 every weight is 1/5."""
+    n = rows * cols
+    neigh = [set() for _ in range(n)]
+    for r in range(rows):
+        for c in range(cols):
+            i = r * cols + c
+            for rr, cc in ((r - 1, c), (r + 1, c), (r, c - 1), (r, c + 1)):
+                j = (rr % rows) * cols + (cc % cols)
+                if j != i:
+                    neigh[i].add(j)
+    return _csr_from_neighbours(neigh)
+
+
+def random_graph(n: int, max_degree: int, seed: int) -> MixingCSR:
+    """Connected irregular graph: a ring plus seeded random chords, node degrees
+    (without self) capped at max_degree.  A stand-in with the degree profile of
+    the paper's 32-node social-network topology (max degree 14); not that graph."""
+    rng = np.random.default_rng(seed)
+    neigh = [set() for _ in range(n)]
+    for i in range(n):
+        neigh[i].add((i + 1) % n)
+        neigh[(i + 1) % n].add(i)
+    hubs = rng.permutation(n)[: max(1, n // 6)]
+    for h in hubs:
+        want = int(rng.integers(max_degree // 2, max_degree + 1))
+        for j in rng.permutation(n):
+            if len(neigh[h]) >= want:
+                break
+            if j != h and j not in neigh[h] and len(neigh[j]) < max_degree:
+                neigh[h].add(int(j))
+                neigh[int(j)].add(int(h))
+    return _csr_from_neighbours(neigh)
+
+
+def spectral_gap(w: MixingCSR) -> float:
+    """1 - |lambda_2(W)| by a dense symmetric eigen-solve (Assumption 1)."""
+    ev = np.sort(np.abs(np.linalg.eigvalsh(w.dense())))[::-1]
+    return float(1.0 - ev[1])
+
+
+def beta_norm(w: MixingCSR) -> float:
+    """beta = ||I - W||_2 (Theorem 4.1)."""
+    return float(np.max(np.abs(np.linalg.eigvalsh(np.eye(w.n) - w.dense()))))
+
+
+# --------------------------------------------------------------------------
+# dense inputs
+# --------------------------------------------------------------------------
+
+
+def normal_rows(n: int, d: int, variance: float, seed: int,
+                mean: Optional[np.ndarray] = None) -> np.ndarray:
+    """float32 [n, d] ~ N(mean_i, variance); one PCG64 stream per (seed, row)."""
+    out = np.empty((n, d), dtype=np.float32)
+    sd = math.sqrt(variance)
+    for i in range(n):
+        rng = np.random.default_rng([seed, i])
+        out[i] = rng.standard_normal(d, dtype=np.float32) * np.float32(sd)
+        if mean is not None:
+            out[i] += np.float32(mean[i])
+    return out
+
+
+def k_of(a_num: int, a_den: int, d: int) -> int:
+    """floor(a * d) with a = a_num / a_den, in integer arithmetic."""
+    return (d * a_num) // a_den
+
+
+# --------------------------------------------------------------------------
+# the five workload shapes (shapes, scales and stepsizes only)
+# --------------------------------------------------------------------------
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    name: str
+    n: int
+    d: int
+    graph: str            # "ring" | "torus8x8" ...
+    q: str                # "topk" | "randk" | "qsgd" | "sign"
+    k: int = 0
+    s: int = 0
+    bucket: int = 0
+    eta: float = 0.0
+    gamma: float = 0.0
+    steps: int = 0
+    x_var: float = 1.0
+    g_var: float = 0.0
+    g_mean_var: float = 0.0
+    sgd: bool = True
+
+    def mixing(self) -> MixingCSR:
+        if self.graph == "ring":
+            return ring(self.n)
+        if self.graph.startswith("torus"):
+            r, c = self.graph[5:].split("x")
+            return torus(int(r), int(c))
+        raise ValueError(self.graph)
+
+
+WORKLOADS = {
+    # average consensus only, 4-ring, top-k k=10
+    "c1_ring4_topk": Workload("c1_ring4_topk", 4, 1024, "ring", "topk", k=10,
+                              gamma=0.05, steps=200, x_var=1.0, sgd=False),
+    # logistic regression d=2000 on a 16-ring: random-k 1 % and QSGD s=16 (whole-row norm)
+    "c2_ring16_randk": Workload("c2_ring16_randk", 16, 2000, "ring", "randk",
+                                k=k_of(1, 100, 2000), eta=0.1, gamma=0.1, steps=2000, x_var=0.0),
+    "c2_ring16_qsgd": Workload("c2_ring16_qsgd", 16, 2000, "ring", "qsgd", s=16, bucket=0,
+                               eta=0.1, gamma=0.1, steps=2000, x_var=0.0),
+    # ResNet-20-sized flat vector, 8-ring, scaled sign
+    "c3_ring8_sign": Workload("c3_ring8_sign", 8, 272474, "ring", "sign", eta=0.1, gamma=0.4,
+                              steps=1000, x_var=0.01, g_var=1e-2, g_mean_var=1e-3),
+    # the headline shape: 8x8 torus, d = 1e6, top-1 %
+    "c4_torus64_topk": Workload("c4_torus64_topk", 64, 1_000_000, "torus8x8", "topk",
+                                k=k_of(1, 100, 1_000_000), eta=0.05, gamma=0.2, steps=500,
+                                x_var=1.0, g_var=1e-2),
+    # ResNet-50-sized flat vector, 32-ring: QSGD s=16 in 512-buckets, or top-0.1 %
+    "c5_ring32_qsgd": Workload("c5_ring32_qsgd", 32, 25_557_032, "ring", "qsgd", s=16,
+                               bucket=512, eta=0.1, gamma=0.1, steps=200, x_var=0.01,
+                               g_var=1e-3),
+    "c5_ring32_topk": Workload("c5_ring32_topk", 32, 25_557_032, "ring", "topk",
+                               k=k_of(1, 1000, 25_557_032), eta=0.1, gamma=0.1, steps=200,
+                               x_var=0.01, g_var=1e-3),
+}
+
+
+# --------------------------------------------------------------------------
+# the convex problem of the d = 2000 workload (caller-side gradient, Alg. 1 line 8)
+# --------------------------------------------------------------------------
+
+
+class LogisticProblem:
+    """L2-regularised logistic regression split non-IID over n workers.
+
+    Features ~ N(0, 1/d), labels sign(a . w*) for a seeded planted w*; all samples
+    are sorted by label and dealt contiguously to the workers.  The gradient is the
+    caller's job in Algorithm 1 (line 8); it is evaluated here in float64 and handed,
+    as float32, to whichever implementation is being driven.
+    """
+
+    def __init__(self, n: int, d: int, per_worker: int, seed: int, lam: float = 1e-4):
+        rng = np.random.default_rng(seed)
+        m = n * per_worker
+        a = rng.standard_normal((m, d)) / math.sqrt(d)
+        w_star = rng.standard_normal(d)
+        y = np.where(a @ w_star >= 0.0, 1.0, -1.0)
+        order = np.argsort(y, kind="stable")
+        self.a = a[order].reshape(n, per_worker, d)
+        self.y = y[order].reshape(n, per_worker)
+        self.n, self.d, self.per_worker, self.lam, self.seed = n, d, per_worker, lam, seed
+
+    def minibatch(self, step: int, worker: int, batch: int) -> np.ndarray:
+        rng = np.random.default_rng([self.seed, 7, step, worker])
+        return rng.integers(0, self.per_worker, size=batch)
+
+    def gradient(self, x: np.ndarray, step: int, batch: int = 32) -> np.ndarray:
+        g = np.empty((self.n, self.d), dtype=np.float32)
+        for i in range(self.n):
+            rows = self.minibatch(step, i, batch)
+            a, y = self.a[i, rows], self.y[i, rows]
+            xi = x[i].astype(np.float64)
+            margin = y * (a @ xi)
+            coef = -y / (1.0 + np.exp(margin))
+            g[i] = ((coef[:, None] * a).mean(axis=0) + self.lam * xi).astype(np.float32)
+        return g
+
+    def loss(self, xbar: np.ndarray) -> float:
+        a = self.a.reshape(-1, self.d)
+        y = self.y.reshape(-1)
+        margin = y * (a @ xbar.astype(np.float64))
+        return float(np.mean(np.logaddexp(0.0, -margin)) + 0.5 * self.lam * float(xbar @ xbar))
