@@ -1,0 +1,190 @@
+/*
+ * choco.h -- C interface of libchoco: the CHOCO-Gossip / CHOCO-SGD step for n simulated
+ * workers on one GPU (Koloskova, Lin, Stich, Jaggi, "Decentralized Deep Learning with
+ * Arbitrary Communication Compression", ICLR 2020).
+ *
+ * State (caller-owned DEVICE memory, float32, row-major, row pitch `ld` elements):
+ *     X    [n, ld]   private iterates x_i                       (Algorithm 1)
+ *     Xhat [n, ld]   public copies x^_i                          (Algorithm 1)
+ *     S    [n, ld]   neighbour sums s_i = sum_j w_ij x^_j        (the "3 vectors per
+ *                    node" storage of Section 3, last paragraph)
+ *     G    [n, ld]   stochastic gradients g_i, read-only          (Algorithm 1, line 8)
+ * A fresh run starts from Xhat = S = 0 (Algorithm 1, input); any state with
+ * S = W Xhat resumes one.  Only the first d elements of each row are used.
+ *
+ * One step call performs, for every worker i at once,
+ *     q_i    = Q(x_i - x^_i)                     Algorithm 1, line 3
+ *     x^_i  += q_i                               line 6 with j = i
+ *     s_i   += sum_j w_ij q_j                    line 6 for all neighbours j, folded into s_i
+ *     x_i    = (x_i - eta g_i) + gamma (s_i - x^_i)
+ *                                                line 9, then line 2 of the next iteration
+ *                                                (sum_j w_ij (x^_j - x^_i) = s_i - x^_i as
+ *                                                rows of W sum to one)
+ * i.e. the gossip scheme h of Appendix A.1 ("Example: CHOCO-SGD"), with the communication
+ * and gradient parts in the rotated order that Appendix A.1 notes only shifts the initial
+ * values.  The messages q_i are written to library-owned device buffers in compressed form
+ * and read back from there by every neighbour.
+ *
+ * Arithmetic: float32, round to nearest, no fused multiply-add, neighbours accumulated in
+ * CSR column order from +0, norms summed as a pairwise tree over the coordinate index.
+ * Results are deterministic: same inputs, seed and step number give the same bits.
+ *
+ * All functions return 0 on success or a negative choco_status; on error nothing has been
+ * enqueued.  Calls on one context must be issued in stream order, from one host thread at
+ * a time.  `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ * Step calls are asynchronous: they enqueue kernels on `stream` and return.
+ */
+#ifndef CHOCO_H_
+#define CHOCO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct choco_ctx choco_ctx; /* opaque; owns the CSR copy of W, messages, workspace */
+
+typedef enum {
+    CHOCO_OK = 0,
+    CHOCO_ERR_INVALID_ARG = -1, /* null pointer, n < 1, d < 1, ld < d, k outside [1, d], ...  */
+    CHOCO_ERR_BAD_W = -2,       /* W violates Assumption 1 or the CSR rules below             */
+    CHOCO_ERR_ALLOC = -3,       /* device or host allocation failed                           */
+    CHOCO_ERR_CUDA = -4,        /* a CUDA runtime call failed (see choco_last_cuda_error)      */
+    CHOCO_ERR_MISALIGNED = -5,  /* a state pointer is not 4-byte aligned                       */
+    CHOCO_ERR_UNSUPPORTED = -6, /* valid in the paper, not built (e.g. an odd QSGD bucket)     */
+    CHOCO_ERR_TOO_LARGE = -7    /* a size exceeds a documented limit                           */
+} choco_status;
+
+/* Compression operator Q (Appendix C, "Compression Schemes"). */
+typedef enum {
+    CHOCO_Q_IDENTITY = 0, /* q = v: exact gossip, the delta = 1 case of Theorem 4.1           */
+    CHOCO_Q_TOPK = 1,     /* top_a: k largest |v|, ties to the lower index                    */
+    CHOCO_Q_RANDK = 2,    /* random_a, biased form v (.) u, ||u||_1 = k                        */
+    CHOCO_Q_QSGD = 3,     /* gsgd_b with s = 2^(b-1) levels, dithered, per block               */
+    CHOCO_Q_SIGN = 4      /* (||v||_1 / d) sgn(v), one bit per coordinate                      */
+} choco_q_kind;
+
+typedef struct {
+    int32_t kind;        /* choco_q_kind                                                       */
+    int32_t s;           /* QSGD: number of levels 2^(b-1), a power of two in [2, 128]         */
+    int32_t bucket;      /* QSGD: block length for the norm; 0 = whole row, else a power of    */
+                         /*       two in [128, 1024] (the last block of a row may be shorter)  */
+    int32_t qsgd_biased; /* QSGD: 1 = divide by tau = 1 + min(len/s^2, sqrt(len)/s) (the       */
+                         /*       delta = 1/tau operator CHOCO uses), 0 = unbiased form        */
+    int64_t k;           /* TOPK / RANDK: entries kept per row, floor(a d), in [1, d]          */
+} choco_params;
+
+/*
+ * choco_init -- Algorithm 1, "input": the communication graph with its mixing matrix W
+ * (Assumption 1), the compression operator and the shared random seed (Appendix C,
+ * random_a: "if it knows the random seed").
+ *   n, d, ld     workers, coordinates per worker, row pitch of all state arrays (ld >= d;
+ *                d < 2^31).
+ *   w_row_ptr[n+1], w_col[nnz], w_val[nnz]   HOST pointers to W in CSR; copied.  Every row
+ *                must list its columns in strictly ascending order and include the diagonal;
+ *                weights in [0, 1], row sums within 1e-5 of one, W symmetric within 1e-6.
+ *   p            Q and its parameter (copied).
+ *   seed         keys the counter-based generator (Philox4x32-10) together with
+ *                (step, worker, coordinate); used by RANDK and QSGD.
+ * Allocates all device memory the steps need on the current device; steps allocate nothing.
+ * The step counter starts at 0.  On success *out owns the context; free with choco_destroy.
+ */
+int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t* w_row_ptr,
+               const int32_t* w_col, const float* w_val, const choco_params* p, uint64_t seed);
+
+/* Frees everything choco_init allocated.  Synchronises the device first. */
+int choco_destroy(choco_ctx* ctx);
+
+/*
+ * choco_gossip_step -- one application of CHOCO-Gossip (the averaging scheme h of Appendix
+ * A.1: X+ = X + gamma Y (W - I), Y+ = Y + Q(X+ - Y), Y = Xhat) in the rotated order given at
+ * the top: compress, update Xhat and S, then x_i += gamma (s_i - x^_i).  No gradient.
+ * X, Xhat, S: DEVICE pointers, updated in place.  Advances the step counter by one.
+ */
+int choco_gossip_step(choco_ctx* ctx, float* X, float* Xhat, float* S, float gamma, void* stream);
+
+/*
+ * choco_sgd_step -- Algorithm 1, lines 3-9 of iteration t followed by line 2 of iteration
+ * t+1, with g_i = G[i] the gradient the caller evaluated at the current x_i (line 8).
+ * G: DEVICE pointer, read-only.  Advances the step counter by one.
+ */
+int choco_sgd_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float eta,
+                   float gamma, void* stream);
+
+/*
+ * choco_sgd_momentum_step -- Algorithm 2 (CHOCO-SGD with momentum): line 9 becomes
+ *     m_i = (g_i + lambda x_i) + beta m_i ;   x_i = (x_i - eta m_i) + gamma (s_i - x^_i)
+ * with M [n, ld] the local momentum memory (DEVICE, updated in place, starts at 0).
+ */
+int choco_sgd_momentum_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G,
+                            float* M, float eta, float gamma, float lambda, float beta,
+                            void* stream);
+
+/*
+ * choco_sgd_step_host -- the same step as choco_sgd_step on HOST arrays (pageable or
+ * pinned): copies X, Xhat, S, G to library-owned device staging buffers (allocated on the
+ * first such call), runs the step, copies X, Xhat, S back and synchronises `stream` before
+ * returning.  G may be NULL for a gossip-only step.
+ */
+int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G,
+                        float eta, float gamma, void* stream);
+
+/*
+ * The library may carry work across calls: while forming x_i of this step it can already
+ * prepare the next step's compression from the registers it holds.  That is valid only if
+ * the caller leaves X and Xhat untouched between two step calls and passes the same
+ * pointers; a change of pointers is detected, a change of contents is not.
+ * choco_invalidate -- call after modifying X or Xhat outside the library (for example
+ * when loading a checkpoint into the same buffers).
+ */
+int choco_invalidate(choco_ctx* ctx);
+
+/* Step counter t (keys the generator).  Setting it, together with restoring X, Xhat and S,
+ * resumes a run bit-exactly; choco_set_step implies choco_invalidate. */
+int choco_get_step(const choco_ctx* ctx, uint64_t* t);
+int choco_set_step(choco_ctx* ctx, uint64_t t);
+
+/*
+ * Message size of one step by the paper's accounting (Appendix C): TOPK 2*32*k bits per
+ * worker, RANDK 32*k, SIGN d + 32 (stored: 4*ceil(d/32) + 4 bytes), QSGD 32 bits per block
+ * plus one sign bit and one level field (1, 2, 4 or 8 bits) per coordinate, IDENTITY 32*d.
+ */
+int choco_message_bytes(const choco_ctx* ctx, int64_t* per_worker, int64_t* total);
+
+/*
+ * Debug access to the message most recently formed for `worker` (valid until the next step
+ * call).  plane: 0 = indices (u32[k]) or packed sign bits (u32[ceil(d/32)]); 1 = values
+ * (f32[k]), the sign scale (f32[1]), QSGD block norms (f32[blocks]) or the dense q
+ * (IDENTITY, f32[d]); 2 = QSGD level fields (bytes).  Returns a DEVICE pointer into
+ * library-owned memory and its size; a plane the operator does not use gives nbytes = 0.
+ */
+int choco_get_message(const choco_ctx* ctx, int32_t worker, int32_t plane, const void** dev_ptr,
+                      int64_t* nbytes);
+
+/* Same planes, copied to a HOST buffer of `capacity` bytes after synchronising `stream`;
+ * *nbytes receives the plane's size (nothing is copied if it exceeds the capacity). */
+int choco_read_message(choco_ctx* ctx, int32_t worker, int32_t plane, void* host_dst,
+                       int64_t capacity, int64_t* nbytes, void* stream);
+
+/* Consensus distance of Section 6 times n: sum_i ||x_i - xbar||^2, accumulated in float64.
+ * X: DEVICE pointer.  Synchronises `stream`; *out is a HOST double. */
+int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* stream);
+
+/* Counters since choco_init (HOST struct filled after synchronising `stream`). */
+typedef struct {
+    uint64_t steps;            /* step calls enqueued                                         */
+    uint64_t prepared_rows;    /* rows whose compression was prepared by the previous step     */
+    uint64_t recompressed_rows;/* rows compressed by a separate pass over X and Xhat           */
+    uint64_t exact_rows;       /* rows that needed the slow exact selection                    */
+} choco_stats;
+int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
+
+const char* choco_strerror(int code);
+/* cudaError_t of the last failing CUDA call on this context (0 if none). */
+int choco_last_cuda_error(const choco_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHOCO_H_ */

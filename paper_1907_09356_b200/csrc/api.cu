@@ -1,0 +1,417 @@
+// C entry points of libchoco: argument checks, allocation, and the order in which one step
+// enqueues its kernels.  No arithmetic of the method lives here.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "internal.h"
+
+using namespace choco;
+
+namespace {
+
+int fail_cuda(choco_ctx* ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return CHOCO_ERR_CUDA;
+}
+
+template <typename T>
+cudaError_t dev_alloc(choco_ctx* ctx, T** out, int64_t count)
+{
+    void* p = nullptr;
+    const size_t bytes = (size_t)(count > 0 ? count : 1) * sizeof(T);
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(p, 0, bytes);
+    if (e != cudaSuccess) { cudaFree(p); return e; }
+    if (ctx->nallocs >= (int)(sizeof(ctx->allocs) / sizeof(ctx->allocs[0]))) { cudaFree(p); return cudaErrorMemoryAllocation; }
+    ctx->allocs[ctx->nallocs++] = p;
+    *out = (T*)p;
+    return cudaSuccess;
+}
+
+int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+// Assumption 1 plus the CSR rules of choco.h
+int check_w(int32_t n, const int32_t* rp, const int32_t* col, const float* val)
+{
+    if (rp[0] != 0) return CHOCO_ERR_BAD_W;
+    for (int32_t i = 0; i < n; ++i) {
+        if (rp[i + 1] <= rp[i]) return CHOCO_ERR_BAD_W;
+        double sum = 0.0;
+        bool diag = false;
+        for (int32_t e = rp[i]; e < rp[i + 1]; ++e) {
+            if (col[e] < 0 || col[e] >= n) return CHOCO_ERR_BAD_W;
+            if (e > rp[i] && col[e] <= col[e - 1]) return CHOCO_ERR_BAD_W;
+            if (!(val[e] >= 0.0f && val[e] <= 1.0f)) return CHOCO_ERR_BAD_W;
+            if (col[e] == i) diag = true;
+            sum += (double)val[e];
+        }
+        if (!diag || std::fabs(sum - 1.0) > 1e-5) return CHOCO_ERR_BAD_W;
+    }
+    // symmetry: every (i, j, w) needs a (j, i, w')
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t e = rp[i]; e < rp[i + 1]; ++e) {
+            const int32_t j = col[e];
+            bool found = false;
+            for (int32_t f = rp[j]; f < rp[j + 1]; ++f)
+                if (col[f] == i) { found = std::fabs((double)val[f] - (double)val[e]) <= 1e-6; break; }
+            if (!found) return CHOCO_ERR_BAD_W;
+        }
+    return CHOCO_OK;
+}
+
+bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+float qsgd_tau(int64_t len, int32_t s, bool biased)
+{
+    if (!biased) return 1.0f;
+    const double a = (double)len / ((double)s * (double)s);
+    const double b = std::sqrt((double)len) / (double)s;
+    return (float)(1.0 + (a < b ? a : b));
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
+
+int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+             float gamma, float lambda, float beta, void* stream)
+{
+    if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    if (!aligned4(X) || !aligned4(Xhat) || !aligned4(S) || !aligned4(G) || !aligned4(M))
+        return CHOCO_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Dev& dv = ctx->dv;
+    StepArgs a;
+    a.X = X; a.Xhat = Xhat; a.S = S; a.G = G; a.M = M;
+    a.eta = eta; a.gamma = gamma; a.lambda = lambda; a.beta = beta;
+    a.step = ctx->step;
+    a.vec = (dv.ld % 4 == 0) && aligned16(X) && aligned16(Xhat) && aligned16(S) &&
+            (!G || aligned16(G)) && (!M || aligned16(M));
+    if (ctx->last_x != X || ctx->last_xhat != Xhat) ctx->prepared = false;
+
+    cudaError_t e = cudaSuccess;
+    const bool sparse = dv.kind == CHOCO_Q_TOPK || dv.kind == CHOCO_Q_RANDK;
+    if (sparse) {
+        if (!ctx->prepared) e = launch_select_prepare(dv, a, st);
+        if (e == cudaSuccess) e = launch_select_emit(dv, a, st);
+    } else {
+        e = launch_compress_dense(dv, a, st);
+    }
+    if (e == cudaSuccess) e = launch_apply(dv, a, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->prepared = false; // nothing is carried across steps yet
+    ctx->last_x = X;
+    ctx->last_xhat = Xhat;
+    ctx->step += 1;
+    ctx->steps_enqueued += 1;
+    return CHOCO_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t* w_row_ptr,
+               const int32_t* w_col, const float* w_val, const choco_params* p, uint64_t seed)
+{
+    if (!out || !w_row_ptr || !w_col || !w_val || !p) return CHOCO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n < 1 || d < 1 || ld < d) return CHOCO_ERR_INVALID_ARG;
+    if (d >= (int64_t)1 << 31) return CHOCO_ERR_TOO_LARGE;
+    if (n > 65535) return CHOCO_ERR_TOO_LARGE; // rows index gridDim.y
+    const int rcw = check_w(n, w_row_ptr, w_col, w_val);
+    if (rcw) return rcw;
+    const int32_t nnz = w_row_ptr[n];
+    switch (p->kind) {
+    case CHOCO_Q_IDENTITY:
+    case CHOCO_Q_SIGN:
+        break;
+    case CHOCO_Q_TOPK:
+    case CHOCO_Q_RANDK:
+        if (p->k < 1 || p->k > d) return CHOCO_ERR_INVALID_ARG;
+        break;
+    case CHOCO_Q_QSGD:
+        if (!is_pow2(p->s) || p->s < 2 || p->s > 128) return CHOCO_ERR_INVALID_ARG;
+        if (p->bucket < 0) return CHOCO_ERR_INVALID_ARG;
+        if (p->bucket != 0 && !(is_pow2(p->bucket) && p->bucket >= 128 && p->bucket <= 1024))
+            return CHOCO_ERR_UNSUPPORTED;
+        break;
+    default:
+        return CHOCO_ERR_INVALID_ARG;
+    }
+
+    choco_ctx* ctx = new (std::nothrow) choco_ctx();
+    if (!ctx) return CHOCO_ERR_ALLOC;
+    std::memset(ctx, 0, sizeof(*ctx));
+    ctx->params = *p;
+    Dev& dv = ctx->dv;
+    dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
+    dv.ntiles = (d + kTile - 1) / kTile;
+    dv.nchunks = (d + kChunk - 1) / kChunk;
+
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    int32_t *rp = nullptr, *col = nullptr;
+    float* wv = nullptr;
+    if (e == cudaSuccess) e = dev_alloc(ctx, &rp, n + 1);
+    if (e == cudaSuccess) e = dev_alloc(ctx, &col, nnz);
+    if (e == cudaSuccess) e = dev_alloc(ctx, &wv, nnz);
+    if (e == cudaSuccess) e = cudaMemcpy(rp, w_row_ptr, sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(col, w_col, sizeof(int32_t) * nnz, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(wv, w_val, sizeof(float) * nnz, cudaMemcpyHostToDevice);
+    dv.row_ptr = rp; dv.col = col; dv.wval = wv;
+    if (e == cudaSuccess) e = dev_alloc(ctx, &dv.stats, 1);
+
+    const int64_t nwords = (d + 31) / 32;
+    if (p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK) {
+        dv.k = p->k;
+        dv.kpitch = round_up(p->k, 4);
+        int64_t cap = 4 * p->k > p->k + 8192 ? 4 * p->k : p->k + 8192;
+        dv.cap = cap < d ? cap : d;
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_idx, n * dv.kpitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_val, n * dv.kpitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_ptr, n * (dv.ntiles + 1));
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.hist, (int64_t)n * kHistBins);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_lo, n);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_count, n);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_flags, n);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.cand_idx, n * dv.cap);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.cand_val, n * dv.cap);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.seg_off, n * dv.ntiles);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.seg_cnt, n * dv.ntiles);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_a, n * dv.ntiles);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_b, n * dv.ntiles);
+        ctx->msg_bytes_per_worker = (p->kind == CHOCO_Q_TOPK ? 8 : 4) * p->k;
+    } else if (p->kind == CHOCO_Q_SIGN) {
+        dv.wpitch = round_up(nwords, 4);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_bits, n * dv.wpitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_scale, n);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial, n * dv.nchunks);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial2, n * dv.nchunks);
+        ctx->msg_bytes_per_worker = 4 * nwords + 4;
+    } else if (p->kind == CHOCO_Q_QSGD) {
+        dv.s = p->s;
+        dv.bucket = p->bucket;
+        int w = 1;
+        while ((1 << w) < p->s) w *= 2;
+        dv.wbits = w;
+        const int64_t blen = p->bucket > 0 ? p->bucket : d;
+        dv.nbuckets = (d + blen - 1) / blen;
+        dv.npitch = round_up(dv.nbuckets, 4);
+        dv.tau_full = qsgd_tau(blen, p->s, p->qsgd_biased != 0);
+        dv.tau_tail = qsgd_tau(d % blen ? d % blen : blen, p->s, p->qsgd_biased != 0);
+        dv.wpitch = round_up(nwords, 4);
+        const int64_t lbytes = (d * w + 7) / 8;
+        dv.lpitch = round_up(lbytes, 16) + 16;
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_bits, n * dv.wpitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_norms, n * dv.npitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_levels, n * dv.lpitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial, n * dv.nchunks);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial2, n * dv.nchunks);
+        ctx->msg_bytes_per_worker = 4 * dv.nbuckets + 4 * nwords + lbytes;
+    } else {
+        dv.dpitch = round_up(d, 4);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_dense, n * dv.dpitch);
+        ctx->msg_bytes_per_worker = 4 * d;
+    }
+    ctx->cons_blocks = (d + 255) / 256;
+    if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->cons_scratch, ctx->cons_blocks);
+    if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->cons_out, 1);
+    if (e != cudaSuccess) {
+        for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
+        const bool oom = e == cudaErrorMemoryAllocation;
+        delete ctx;
+        return oom ? CHOCO_ERR_ALLOC : CHOCO_ERR_CUDA;
+    }
+    *out = ctx;
+    return CHOCO_OK;
+}
+
+int choco_destroy(choco_ctx* ctx)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
+    for (int i = 0; i < 4; ++i)
+        if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    delete ctx;
+    return CHOCO_OK;
+}
+
+int choco_gossip_step(choco_ctx* ctx, float* X, float* Xhat, float* S, float gamma, void* stream)
+{
+    return run_step(ctx, X, Xhat, S, nullptr, nullptr, 0.f, gamma, 0.f, 0.f, stream);
+}
+
+int choco_sgd_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float eta,
+                   float gamma, void* stream)
+{
+    if (!G) return CHOCO_ERR_INVALID_ARG;
+    return run_step(ctx, X, Xhat, S, G, nullptr, eta, gamma, 0.f, 0.f, stream);
+}
+
+int choco_sgd_momentum_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G,
+                            float* M, float eta, float gamma, float lambda, float beta,
+                            void* stream)
+{
+    if (!G || !M) return CHOCO_ERR_INVALID_ARG;
+    return run_step(ctx, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+}
+
+int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G,
+                        float eta, float gamma, void* stream)
+{
+    if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = (size_t)ctx->dv.n * (size_t)ctx->dv.ld * sizeof(float);
+    for (int i = 0; i < 4; ++i)
+        if (!ctx->stage[i]) {
+            cudaError_t e = cudaMalloc((void**)&ctx->stage[i], bytes);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CHOCO_ERR_ALLOC; }
+        }
+    const float* src[4] = {X, Xhat, S, G};
+    for (int i = 0; i < 4; ++i) {
+        if (!src[i]) continue;
+        cudaError_t e = cudaMemcpyAsync(ctx->stage[i], src[i], bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    ctx->prepared = false; // the staging contents changed
+    const int rc = run_step(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], G ? ctx->stage[3] : nullptr,
+                            nullptr, eta, gamma, 0.f, 0.f, stream);
+    if (rc) return rc;
+    float* dst[3] = {X, Xhat, S};
+    for (int i = 0; i < 3; ++i) {
+        cudaError_t e = cudaMemcpyAsync(dst[i], ctx->stage[i], bytes, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->prepared = false;
+    return CHOCO_OK;
+}
+
+int choco_invalidate(choco_ctx* ctx)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    ctx->prepared = false;
+    return CHOCO_OK;
+}
+
+int choco_get_step(const choco_ctx* ctx, uint64_t* t)
+{
+    if (!ctx || !t) return CHOCO_ERR_INVALID_ARG;
+    *t = ctx->step;
+    return CHOCO_OK;
+}
+
+int choco_set_step(choco_ctx* ctx, uint64_t t)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    if (t >> 56) return CHOCO_ERR_TOO_LARGE;
+    ctx->step = t;
+    ctx->prepared = false;
+    return CHOCO_OK;
+}
+
+int choco_message_bytes(const choco_ctx* ctx, int64_t* per_worker, int64_t* total)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    if (per_worker) *per_worker = ctx->msg_bytes_per_worker;
+    if (total) *total = ctx->msg_bytes_per_worker * ctx->dv.n;
+    return CHOCO_OK;
+}
+
+int choco_get_message(const choco_ctx* ctx, int32_t worker, int32_t plane, const void** dev_ptr,
+                      int64_t* nbytes)
+{
+    if (!ctx || !dev_ptr || !nbytes || worker < 0 || worker >= ctx->dv.n || plane < 0 || plane > 2)
+        return CHOCO_ERR_INVALID_ARG;
+    const Dev& dv = ctx->dv;
+    const int64_t nwords = (dv.d + 31) / 32;
+    *dev_ptr = nullptr;
+    *nbytes = 0;
+    switch (dv.kind) {
+    case CHOCO_Q_TOPK:
+    case CHOCO_Q_RANDK:
+        if (plane == 0) { *dev_ptr = dv.msg_idx + worker * dv.kpitch; *nbytes = 4 * dv.k; }
+        if (plane == 1) { *dev_ptr = dv.msg_val + worker * dv.kpitch; *nbytes = 4 * dv.k; }
+        break;
+    case CHOCO_Q_SIGN:
+        if (plane == 0) { *dev_ptr = dv.msg_bits + worker * dv.wpitch; *nbytes = 4 * nwords; }
+        if (plane == 1) { *dev_ptr = dv.msg_scale + worker; *nbytes = 4; }
+        break;
+    case CHOCO_Q_QSGD:
+        if (plane == 0) { *dev_ptr = dv.msg_bits + worker * dv.wpitch; *nbytes = 4 * nwords; }
+        if (plane == 1) { *dev_ptr = dv.msg_norms + worker * dv.npitch; *nbytes = 4 * dv.nbuckets; }
+        if (plane == 2) { *dev_ptr = dv.msg_levels + worker * dv.lpitch; *nbytes = (dv.d * dv.wbits + 7) / 8; }
+        break;
+    default:
+        if (plane == 1) { *dev_ptr = dv.msg_dense + worker * dv.dpitch; *nbytes = 4 * dv.d; }
+        break;
+    }
+    return CHOCO_OK;
+}
+
+int choco_read_message(choco_ctx* ctx, int32_t worker, int32_t plane, void* host_dst,
+                       int64_t capacity, int64_t* nbytes, void* stream)
+{
+    if (!host_dst || capacity < 0) return CHOCO_ERR_INVALID_ARG;
+    const void* src = nullptr;
+    const int rc = choco_get_message(ctx, worker, plane, &src, nbytes);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess && *nbytes > 0 && *nbytes <= capacity)
+        e = cudaMemcpy(host_dst, src, (size_t)*nbytes, cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? CHOCO_OK : fail_cuda(ctx, e);
+}
+
+int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* stream)
+{
+    if (!ctx || !X || !out) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = launch_consensus(X, ctx->dv.n, ctx->dv.d, ctx->dv.ld, ctx->cons_scratch,
+                                     ctx->cons_blocks, ctx->cons_out, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out, ctx->cons_out, sizeof(double), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? CHOCO_OK : fail_cuda(ctx, e);
+}
+
+int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
+{
+    if (!ctx || !out) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    Stats h;
+    cudaError_t e = cudaMemcpyAsync(&h, ctx->dv.stats, sizeof(h), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    out->steps = ctx->steps_enqueued;
+    out->prepared_rows = h.prepared_rows;
+    out->recompressed_rows = h.recompressed_rows;
+    out->exact_rows = h.exact_rows;
+    return CHOCO_OK;
+}
+
+const char* choco_strerror(int code)
+{
+    switch (code) {
+    case CHOCO_OK: return "ok";
+    case CHOCO_ERR_INVALID_ARG: return "invalid argument";
+    case CHOCO_ERR_BAD_W: return "mixing matrix violates Assumption 1 or the CSR rules";
+    case CHOCO_ERR_ALLOC: return "allocation failed";
+    case CHOCO_ERR_CUDA: return "CUDA runtime error";
+    case CHOCO_ERR_MISALIGNED: return "pointer not 4-byte aligned";
+    case CHOCO_ERR_UNSUPPORTED: return "unsupported configuration";
+    case CHOCO_ERR_TOO_LARGE: return "size exceeds a documented limit";
+    default: return "unknown error";
+    }
+}
+
+int choco_last_cuda_error(const choco_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+} // extern "C"

@@ -1,0 +1,246 @@
+// The update half of a CHOCO step (Algorithm 1, lines 6, 2 and 9; Algorithm 2 for the
+// momentum variant): every worker reads its neighbours' messages back and forms
+//     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
+//     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i).
+// One block owns 4096 coordinates of one row.
+#include "common.cuh"
+#include "internal.h"
+
+namespace choco {
+
+struct Upd {
+    float eta, gamma, lambda, beta;
+};
+
+// x' from the updated s and x^ of one coordinate
+template <bool HAS_G, bool HAS_M>
+__device__ __forceinline__ float next_x(float x, float sn, float hn, float g, float& m, const Upd& u)
+{
+    const float cons = __fsub_rn(sn, hn);
+    float xn = x;
+    if (HAS_M) {
+        m = __fadd_rn(__fadd_rn(g, __fmul_rn(u.lambda, x)), __fmul_rn(u.beta, m));
+        xn = __fsub_rn(x, __fmul_rn(u.eta, m));
+    } else if (HAS_G) {
+        xn = __fsub_rn(x, __fmul_rn(u.eta, g));
+    }
+    return __fadd_rn(xn, __fmul_rn(u.gamma, cons));
+}
+
+// ---------------------------------------------------------------------------------------
+// dense Q: decode each neighbour's message on the fly
+// ---------------------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ float4 decode_quad(const Dev& dv, int j, int64_t c)
+{
+    if (KIND == CHOCO_Q_IDENTITY)
+        return __ldg(reinterpret_cast<const float4*>(dv.msg_dense + (int64_t)j * dv.dpitch + c));
+    const uint32_t word = __ldg(dv.msg_bits + (int64_t)j * dv.wpitch + (c >> 5));
+    const uint32_t nib = (word >> (c & 31)) & 0xFu;
+    float m[4];
+    if (KIND == CHOCO_Q_SIGN) {
+        const float sc = __ldg(dv.msg_scale + j);
+        m[0] = m[1] = m[2] = m[3] = sc;
+    } else {
+        const int64_t b = dv.bucket > 0 ? c / dv.bucket : 0;
+        const float nu = __ldg(dv.msg_norms + (int64_t)j * dv.npitch + b);
+        const bool tail = dv.bucket > 0 && b == dv.nbuckets - 1 && (dv.d % dv.bucket) != 0;
+        const float scale = __fdiv_rn(nu, __fmul_rn(tail ? dv.tau_tail : dv.tau_full, (float)dv.s));
+        const uint8_t* lrow = dv.msg_levels + (int64_t)j * dv.lpitch;
+        uint32_t packed, width = (uint32_t)dv.wbits;
+        if (width == 8) packed = __ldg(reinterpret_cast<const uint32_t*>(lrow + c));
+        else if (width == 4) packed = __ldg(reinterpret_cast<const uint16_t*>(lrow + (c >> 1)));
+        else if (width == 2) packed = __ldg(lrow + (c >> 2));
+        else packed = (__ldg(lrow + (c >> 3)) >> (c & 7)) & 0xFu;
+        const uint32_t mask = (1u << width) - 1u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m[e] = __fmul_rn(scale, (float)((packed >> (e * width)) & mask));
+    }
+    return make_float4(nib & 1u ? -m[0] : m[0], nib & 2u ? -m[1] : m[1], nib & 4u ? -m[2] : m[2],
+                       nib & 8u ? -m[3] : m[3]);
+}
+
+template <bool VEC, int KIND, bool HAS_G, bool HAS_M>
+__global__ void __launch_bounds__(kThreads) apply_dense_kernel(Dev dv, StepArgs a)
+{
+    const int row = blockIdx.y;
+    const int64_t c0 = (int64_t)blockIdx.x * kTile;
+    const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
+    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
+    float* xr = a.X + (int64_t)row * dv.ld;
+    float* hr = a.Xhat + (int64_t)row * dv.ld;
+    float* sr = a.S + (int64_t)row * dv.ld;
+    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld : nullptr;
+    float* mr = HAS_M ? a.M + (int64_t)row * dv.ld : nullptr;
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
+        if (c >= dv.d) continue;
+        const float4 x = load_quad<VEC>(xr, c, dv.d);
+        const float4 h = load_quad<VEC>(hr, c, dv.d);
+        const float4 s = load_quad<VEC>(sr, c, dv.d);
+        float4 g = make_float4(0.f, 0.f, 0.f, 0.f), m = g;
+        if (HAS_G) g = load_quad_stream<VEC>(gr, c, dv.d);
+        if (HAS_M) m = load_quad<VEC>(mr, c, dv.d);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), qs = acc;
+        for (int e = e0; e < e1; ++e) {
+            const int j = dv.col[e];
+            const float w = dv.wval[e];
+            const float4 q = decode_quad<KIND>(dv, j, c);
+            acc.x = __fadd_rn(acc.x, __fmul_rn(w, q.x));
+            acc.y = __fadd_rn(acc.y, __fmul_rn(w, q.y));
+            acc.z = __fadd_rn(acc.z, __fmul_rn(w, q.z));
+            acc.w = __fadd_rn(acc.w, __fmul_rn(w, q.w));
+            if (j == row) qs = q;
+        }
+        const float4 hn = make_float4(__fadd_rn(h.x, qs.x), __fadd_rn(h.y, qs.y),
+                                      __fadd_rn(h.z, qs.z), __fadd_rn(h.w, qs.w));
+        const float4 sn = make_float4(__fadd_rn(s.x, acc.x), __fadd_rn(s.y, acc.y),
+                                      __fadd_rn(s.z, acc.z), __fadd_rn(s.w, acc.w));
+        float4 xn;
+        xn.x = next_x<HAS_G, HAS_M>(x.x, sn.x, hn.x, g.x, m.x, u);
+        xn.y = next_x<HAS_G, HAS_M>(x.y, sn.y, hn.y, g.y, m.y, u);
+        xn.z = next_x<HAS_G, HAS_M>(x.z, sn.z, hn.z, g.z, m.z, u);
+        xn.w = next_x<HAS_G, HAS_M>(x.w, sn.w, hn.w, g.w, m.w, u);
+        store_quad<VEC>(hr, c, dv.d, hn);
+        store_quad<VEC>(sr, c, dv.d, sn);
+        store_quad<VEC>(xr, c, dv.d, xn);
+        if (HAS_M) store_quad<VEC>(mr, c, dv.d, m);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// sparse Q: the neighbours' (index, value) lists are scattered into a shared-memory tile,
+// one neighbour after the other so that the additions happen in CSR order, then the tile is
+// streamed against x, x^, s and g.  x^ and s are written only where a message touched them.
+// ---------------------------------------------------------------------------------------
+template <bool VEC, bool HAS_G, bool HAS_M>
+__global__ void __launch_bounds__(kThreads) apply_sparse_kernel(Dev dv, StepArgs a)
+{
+    __shared__ __align__(16) float acc[kTile];
+    __shared__ __align__(16) float qself[kTile];
+    __shared__ uint32_t touched[kTile / 32];
+    __shared__ uint32_t tself[kTile / 32];
+    const int row = blockIdx.y;
+    const int64_t tile = blockIdx.x;
+    const int64_t c0 = tile * kTile;
+    const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
+    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
+    float* xr = a.X + (int64_t)row * dv.ld;
+    float* hr = a.Xhat + (int64_t)row * dv.ld;
+    float* sr = a.S + (int64_t)row * dv.ld;
+    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld : nullptr;
+    float* mr = HAS_M ? a.M + (int64_t)row * dv.ld : nullptr;
+
+    // start the dense loads before touching the messages
+    float4 x[kIters], h[kIters], s[kIters], g[kIters];
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
+        x[it] = load_quad_stream<VEC>(xr, c, dv.d);
+        h[it] = load_quad_stream<VEC>(hr, c, dv.d);
+        s[it] = load_quad_stream<VEC>(sr, c, dv.d);
+        if (HAS_G) g[it] = load_quad_stream<VEC>(gr, c, dv.d);
+        else g[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        reinterpret_cast<float4*>(acc)[it * kThreads + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4*>(qself)[it * kThreads + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (threadIdx.x < kTile / 32) { touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; }
+    __syncthreads();
+    for (int e = e0; e < e1; ++e) {
+        const int j = dv.col[e];
+        const float w = dv.wval[e];
+        const uint32_t* tp = dv.tile_ptr + (int64_t)j * (dv.ntiles + 1) + tile;
+        const uint32_t lo = __ldg(tp), hi = __ldg(tp + 1);
+        const uint32_t* mi = dv.msg_idx + (int64_t)j * dv.kpitch;
+        const float* mv = dv.msg_val + (int64_t)j * dv.kpitch;
+        for (uint32_t p = lo + threadIdx.x; p < hi; p += kThreads) {
+            const uint32_t lc = __ldg(mi + p) - (uint32_t)c0;
+            const float val = __ldg(mv + p);
+            acc[lc] = __fadd_rn(acc[lc], __fmul_rn(w, val));
+            atomicOr(&touched[lc >> 5], 1u << (lc & 31));
+            if (j == row) {
+                qself[lc] = val;
+                atomicOr(&tself[lc >> 5], 1u << (lc & 31));
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int li = (it * kThreads + threadIdx.x) * kQuad;
+        const int64_t c = c0 + li;
+        if (c >= dv.d) continue;
+        const float4 av = reinterpret_cast<const float4*>(acc)[it * kThreads + threadIdx.x];
+        const float4 qv = reinterpret_cast<const float4*>(qself)[it * kThreads + threadIdx.x];
+        const uint32_t tb = (touched[li >> 5] >> (li & 31)) & 0xFu;
+        const uint32_t sb = (tself[li >> 5] >> (li & 31)) & 0xFu;
+        float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (HAS_M) m = load_quad<VEC>(mr, c, dv.d);
+        const float xs[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+        const float hs[4] = {h[it].x, h[it].y, h[it].z, h[it].w};
+        const float ss[4] = {s[it].x, s[it].y, s[it].z, s[it].w};
+        const float gs[4] = {g[it].x, g[it].y, g[it].z, g[it].w};
+        const float as[4] = {av.x, av.y, av.z, av.w};
+        const float qq[4] = {qv.x, qv.y, qv.z, qv.w};
+        float ms[4] = {m.x, m.y, m.z, m.w};
+        float xn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float hn = (sb >> e) & 1u ? __fadd_rn(hs[e], qq[e]) : hs[e];
+            const float sn = (tb >> e) & 1u ? __fadd_rn(ss[e], as[e]) : ss[e];
+            xn[e] = next_x<HAS_G, HAS_M>(xs[e], sn, hn, gs[e], ms[e], u);
+            if (c + e < dv.d) {
+                if ((sb >> e) & 1u) hr[c + e] = hn;
+                if ((tb >> e) & 1u) sr[c + e] = sn;
+            }
+        }
+        store_quad<VEC>(xr, c, dv.d, make_float4(xn[0], xn[1], xn[2], xn[3]));
+        if (HAS_M) store_quad<VEC>(mr, c, dv.d, make_float4(ms[0], ms[1], ms[2], ms[3]));
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------
+
+template <bool VEC, bool HAS_G, bool HAS_M>
+static void apply_pick(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
+    switch (dv.kind) {
+    case CHOCO_Q_TOPK:
+    case CHOCO_Q_RANDK:
+        apply_sparse_kernel<VEC, HAS_G, HAS_M><<<grid, kThreads, 0, st>>>(dv, a);
+        break;
+    case CHOCO_Q_SIGN:
+        apply_dense_kernel<VEC, CHOCO_Q_SIGN, HAS_G, HAS_M><<<grid, kThreads, 0, st>>>(dv, a);
+        break;
+    case CHOCO_Q_QSGD:
+        apply_dense_kernel<VEC, CHOCO_Q_QSGD, HAS_G, HAS_M><<<grid, kThreads, 0, st>>>(dv, a);
+        break;
+    default:
+        apply_dense_kernel<VEC, CHOCO_Q_IDENTITY, HAS_G, HAS_M><<<grid, kThreads, 0, st>>>(dv, a);
+        break;
+    }
+}
+
+template <bool VEC>
+static void apply_vec(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    if (a.M) apply_pick<VEC, true, true>(dv, a, st);
+    else if (a.G) apply_pick<VEC, true, false>(dv, a, st);
+    else apply_pick<VEC, false, false>(dv, a, st);
+}
+
+cudaError_t launch_apply(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    if (a.vec) apply_vec<true>(dv, a, st);
+    else apply_vec<false>(dv, a, st);
+    return cudaGetLastError();
+}
+
+} // namespace choco

@@ -1,0 +1,147 @@
+// Device helpers shared by the kernels of libchoco (sm_100a).
+//
+// Arithmetic rules every kernel follows so that results are reproducible bit for bit:
+// float32, round to nearest even, no fused multiply-add (the library is compiled with
+// -fmad=false), IEEE division and square root, norms summed as a pairwise tree over the
+// coordinate index (level 0 = the terms, each level adds elements 2j and 2j+1, missing
+// elements count as +0).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace choco {
+
+constexpr int kThreads = 256;            // threads per block of the streaming kernels
+constexpr int kQuad = 4;                 // coordinates per thread per iteration (one 128-bit access)
+constexpr int kChunk = kThreads * kQuad; // 1024 coordinates: one block iteration, one tree leaf group
+constexpr int kIters = 4;                // iterations per block
+constexpr int kTile = kChunk * kIters;   // 4096 coordinates per block
+
+constexpr uint32_t kStreamRandK = 0;     // generator stream of the random-k selection keys
+constexpr uint32_t kStreamDither = 1;    // generator stream of the QSGD dither
+
+// ---------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  Counter = (coord / 4, worker, step low,
+// (step high << 8) | stream), key = the two halves of the seed; coordinate c uses word c % 4.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) {
+            key.x += 0x9E3779B9u;
+            key.y += 0xBB67AE85u;
+        }
+        const uint32_t hi0 = __umulhi(0xD2511F53u, ctr.x);
+        const uint32_t lo0 = 0xD2511F53u * ctr.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, ctr.z);
+        const uint32_t lo1 = 0xCD9E8D57u * ctr.z;
+        ctr = make_uint4(hi1 ^ ctr.y ^ key.x, lo1, hi0 ^ ctr.w ^ key.y, lo0);
+    }
+    return ctr;
+}
+
+__device__ __forceinline__ uint4 coord_words(uint64_t seed, uint64_t step, uint32_t worker,
+                                             uint32_t stream, int64_t c)
+{
+    const uint4 ctr = make_uint4((uint32_t)(c >> 2), worker, (uint32_t)step,
+                                 ((uint32_t)(step >> 32) << 8) | stream);
+    return philox4x32_10(ctr, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
+}
+
+__device__ __forceinline__ float word_to_unit(uint32_t w)
+{
+    return (float)(w >> 8) * 0x1p-24f; // exact: 24 bits
+}
+
+// ---------------------------------------------------------------------------------------
+// Row access.  A quad is coordinates [c, c+4) with c % 4 == 0.  VEC rows (16-byte aligned
+// base, pitch a multiple of 4) use one 128-bit access for full quads; other rows and the
+// ragged last quad use scalar accesses.  Out-of-range coordinates read as +0.
+// ---------------------------------------------------------------------------------------
+template <bool VEC>
+__device__ __forceinline__ float4 load_quad(const float* __restrict__ row, int64_t c, int64_t d)
+{
+    if (VEC && c + 4 <= d) return *reinterpret_cast<const float4*>(row + c);
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < d) r.x = row[c];
+    if (c + 1 < d) r.y = row[c + 1];
+    if (c + 2 < d) r.z = row[c + 2];
+    if (c + 3 < d) r.w = row[c + 3];
+    return r;
+}
+
+// streaming variant (evict-first hint): data that is read once per step
+template <bool VEC>
+__device__ __forceinline__ float4 load_quad_stream(const float* __restrict__ row, int64_t c,
+                                                   int64_t d)
+{
+    if (VEC && c + 4 <= d) return __ldcs(reinterpret_cast<const float4*>(row + c));
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < d) r.x = __ldcs(row + c);
+    if (c + 1 < d) r.y = __ldcs(row + c + 1);
+    if (c + 2 < d) r.z = __ldcs(row + c + 2);
+    if (c + 3 < d) r.w = __ldcs(row + c + 3);
+    return r;
+}
+
+template <bool VEC>
+__device__ __forceinline__ void store_quad(float* __restrict__ row, int64_t c, int64_t d, float4 v)
+{
+    if (VEC && c + 4 <= d) {
+        *reinterpret_cast<float4*>(row + c) = v;
+        return;
+    }
+    if (c < d) row[c] = v.x;
+    if (c + 1 < d) row[c + 1] = v.y;
+    if (c + 2 < d) row[c + 2] = v.z;
+    if (c + 3 < d) row[c + 3] = v.w;
+}
+
+__device__ __forceinline__ float quad_get(const float4& q, int e)
+{
+    return e == 0 ? q.x : e == 1 ? q.y : e == 2 ? q.z : q.w;
+}
+
+// ---------------------------------------------------------------------------------------
+// Pairwise tree pieces.  quad_tree: two levels inside a quad.  warp_tree: five more levels
+// by xor-butterfly (a + b is commutative, so both lanes of a pair hold the same bits); all
+// lanes end with the sum over the warp's 128 coordinates.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float quad_tree(float a, float b, float c, float d)
+{
+    return __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
+}
+
+__device__ __forceinline__ float warp_tree(float v)
+{
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, m));
+    return v;
+}
+
+// Tree over the 8 warp sums of a 256-thread block (ws[0..8) in shared memory).
+__device__ __forceinline__ float tree8(const float* ws)
+{
+    return __fadd_rn(__fadd_rn(__fadd_rn(ws[0], ws[1]), __fadd_rn(ws[2], ws[3])),
+                     __fadd_rn(__fadd_rn(ws[4], ws[5]), __fadd_rn(ws[6], ws[7])));
+}
+
+// Combine four sign flags per lane (bit e = coordinate 4*lane + e is negative) of 8
+// neighbouring lanes into the 32-bit word that covers coordinates [32w, 32w+32).
+__device__ __forceinline__ uint32_t gather_sign_word(uint32_t nib, int lane)
+{
+    uint32_t w = nib << (4 * (lane & 7));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    w |= __shfl_xor_sync(0xffffffffu, w, 2);
+    w |= __shfl_xor_sync(0xffffffffu, w, 4);
+    return w;
+}
+
+__device__ __forceinline__ uint32_t abs_key(float v)
+{
+    return __float_as_uint(v) & 0x7FFFFFFFu;
+}
+
+} // namespace choco

@@ -1,0 +1,121 @@
+// Internal layout of a libchoco context and the launchers of its kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/choco.h"
+
+namespace choco {
+
+// Row flags of the selection pipeline (top-k, random-k).
+constexpr uint32_t kRowExact = 1u;    // candidates unusable: run the exact one-block selection
+
+constexpr int kHistBins = 2048;       // first radix digit: top 11 bits of the ordering key
+
+struct Stats {
+    unsigned long long prepared_rows;
+    unsigned long long recompressed_rows;
+    unsigned long long exact_rows;
+};
+
+// Everything the kernels need; passed by value.
+struct Dev {
+    int32_t n;
+    int32_t kind;
+    int64_t d;
+    int64_t ld;
+    int64_t ntiles;              // ceil(d / 4096)
+    int64_t nchunks;             // ceil(d / 1024)
+    // W (CSR)
+    const int32_t* row_ptr;
+    const int32_t* col;
+    const float* wval;
+    // generator
+    uint64_t seed;
+    // sparse messages: idx / val [n, kpitch], tile_ptr [n, ntiles + 1]
+    int64_t k;
+    int64_t kpitch;
+    uint32_t* msg_idx;
+    float* msg_val;
+    uint32_t* tile_ptr;
+    // selection workspace
+    int64_t cap;                 // candidate capacity per row
+    uint32_t* hist;              // [n, kHistBins]
+    uint32_t* row_lo;            // [n] lower bound of the ordering key for candidates
+    uint32_t* row_count;         // [n] candidates collected
+    uint32_t* row_flags;         // [n]
+    uint32_t* cand_idx;          // [n, cap]
+    uint32_t* cand_val;          // [n, cap] value bits (top-k) or random word (random-k)
+    uint32_t* seg_off;           // [n, ntiles] first candidate of a tile
+    uint32_t* seg_cnt;           // [n, ntiles]
+    uint32_t* tile_a;            // [n, ntiles] scratch
+    uint32_t* tile_b;            // [n, ntiles] scratch
+    Stats* stats;
+    // dense messages
+    int64_t wpitch;              // sign-plane words per row (multiple of 4)
+    uint32_t* msg_bits;          // [n, wpitch]
+    float* msg_scale;            // sign: [n]
+    int64_t nbuckets;            // qsgd blocks per row
+    int64_t npitch;              // floats per row of msg_norms
+    float* msg_norms;            // qsgd: [n, npitch]
+    int64_t lpitch;              // bytes per row of msg_levels (multiple of 16)
+    uint8_t* msg_levels;         // qsgd: [n, lpitch]
+    int64_t dpitch;              // identity: floats per row of msg_dense
+    float* msg_dense;            // identity: [n, dpitch]
+    // qsgd parameters
+    int32_t s;
+    int32_t bucket;              // 0 = whole row
+    int32_t wbits;               // level field width
+    float tau_full;              // tau of a full block (or of the whole row)
+    float tau_tail;              // tau of the ragged last block
+    // norm workspace
+    float* partial;              // [n, nchunks] per-1024 partial sums
+    float* partial2;             // [n, nchunks] ping-pong for the tree
+};
+
+struct StepArgs {
+    float* X;
+    float* Xhat;
+    float* S;
+    const float* G;              // may be null
+    float* M;                    // momentum memory, may be null
+    float eta, gamma, lambda, beta;
+    uint64_t step;
+    bool vec;                    // rows 16-byte aligned: 128-bit accesses
+};
+
+// selection (top-k / random-k)
+cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t st);
+cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, cudaStream_t st);
+// dense compressors
+cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st);
+// apply
+cudaError_t launch_apply(const Dev& dv, const StepArgs& a, cudaStream_t st);
+// metrics
+cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,
+                             int64_t nblocks, double* out, cudaStream_t st);
+
+} // namespace choco
+
+struct choco_ctx {
+    choco::Dev dv;
+    choco_params params;
+    uint64_t step;
+    uint64_t steps_enqueued;
+    int device;
+    int last_cuda_error;
+    bool prepared;               // next step's candidates/messages already formed
+    const float* last_x;
+    const float* last_xhat;
+    int64_t msg_bytes_per_worker;
+    // host staging for choco_sgd_step_host
+    float* stage[4];
+    // consensus scratch
+    double* cons_scratch;
+    int64_t cons_blocks;
+    double* cons_out;
+    // all device allocations, for choco_destroy
+    void* allocs[64];
+    int nallocs;
+};

@@ -1,0 +1,253 @@
+"""CUDA library vs CPU oracle, through the C interface, on the same seeded inputs.
+
+Acceptance: selected indices, packed sign bits, level fields and random-k indices are
+bit-exact; float32 state within 1e-5 * max|x| of the oracle after a step.  The library
+follows a fixed operation order, so the tests additionally require the float32 state to be
+identical (values compared with ==, which treats +0 and -0 alike).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1907_09356_b200 as choco
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _dev(a, ld=None):
+    """Host [n, d] -> device tensor with row pitch ld (a view of a larger buffer when ld > d)."""
+    n, d = a.shape
+    ld = ld or d
+    if ld == d:
+        return torch.from_numpy(a).to(DEV).contiguous()
+    buf = torch.full((n, ld), float("nan"), dtype=torch.float32, device=DEV)
+    buf[:, :d] = torch.from_numpy(a).to(DEV)
+    return buf
+
+
+def _host(t, d):
+    return t[:, :d].cpu().numpy()
+
+
+def assert_state(got, want, what):
+    """spec tolerance, then the stricter equality the fixed operation order gives."""
+    tol = 1e-5 * max(float(np.max(np.abs(want))), 1e-30)
+    assert np.max(np.abs(got.astype(np.float64) - want.astype(np.float64))) <= tol, what
+    assert np.array_equal(got, want), f"{what}: within tolerance but not identical"
+
+
+def check_messages(ctx, kind, msgs, d):
+    for i, m in msgs.items():
+        p0 = choco.choco_read_message(ctx, i, 0)
+        p1 = choco.choco_read_message(ctx, i, 1)
+        p2 = choco.choco_read_message(ctx, i, 2)
+        if kind in ("topk", "randk"):
+            assert np.array_equal(p0.view(np.uint32), m.idx), f"indices of worker {i}"
+            assert np.array_equal(p1.view(np.uint32), m.val.view(np.uint32)), f"values of worker {i}"
+        elif kind == "sign":
+            assert np.array_equal(p0.view(np.uint32), m.bits), f"sign bits of worker {i}"
+            assert p1.view(np.float32)[0] == m.scale, f"scale of worker {i}"
+        elif kind == "qsgd":
+            assert np.array_equal(p0.view(np.uint32), m.bits), f"sign bits of worker {i}"
+            assert np.array_equal(p1.view(np.float32), m.norms), f"norms of worker {i}"
+            assert np.array_equal(p2, m.levels), f"levels of worker {i}"
+        else:
+            assert np.array_equal(p1.view(np.float32), m.q)
+
+
+def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed=0, ld=None,
+                 eta=0.1, gamma=0.2, x_var=1.0, g_var=0.01, sgd=True, momentum=False,
+                 x_init=None, check_msgs=True, grad_fn=None):
+    ld = ld or d
+    X = workloads.normal_rows(n, d, x_var, 1000 + seed) if x_init is None else x_init.copy()
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    M = np.zeros_like(X) if momentum else None
+    p = oracle.Params(kind, k=k, s=s, bucket=bucket, biased=biased, seed=seed)
+    ch = choco.Choco(w, d, kind, k=k, s=s, bucket=bucket, qsgd_biased=biased, seed=seed, ld=ld)
+    dX, dXh, dS = _dev(X, ld), _dev(Xh, ld), _dev(S, ld)
+    dM = _dev(M, ld) if momentum else None
+    try:
+        for t in range(steps):
+            if grad_fn is not None:
+                G = grad_fn(t, X)
+            elif sgd:
+                G = workloads.normal_rows(n, d, g_var, 5000 + 97 * seed + t)
+            else:
+                G = None
+            dG = _dev(G, ld) if G is not None else None
+            if momentum:
+                msgs = oracle.step(w, p, X, Xh, S, G, eta, gamma, t, M=M, lam=1e-3, beta=0.9)
+                ch.sgd_momentum_step(dX, dXh, dS, dG, dM, eta, gamma, 1e-3, 0.9)
+            elif G is not None:
+                msgs = oracle.step(w, p, X, Xh, S, G, eta, gamma, t)
+                ch.sgd_step(dX, dXh, dS, dG, eta, gamma)
+            else:
+                msgs = oracle.step(w, p, X, Xh, S, None, 0.0, gamma, t)
+                ch.gossip_step(dX, dXh, dS, gamma)
+            torch.cuda.synchronize()
+            if check_msgs:
+                check_messages(ch.ctx, kind, msgs, d)
+            assert_state(_host(dXh, d), Xh, f"Xhat after step {t}")
+            assert_state(_host(dS, d), S, f"S after step {t}")
+            assert_state(_host(dX, d), X, f"X after step {t}")
+            if momentum:
+                assert_state(_host(dM, d), M, f"M after step {t}")
+        assert choco.choco_get_step(ch.ctx) == steps
+        if ld != d:   # the pad between rows is never written
+            assert bool(torch.isnan(dX[:, d:]).all()) and bool(torch.isnan(dS[:, d:]).all())
+        return ch, (dX, dXh, dS), (X, Xh, S)
+    except Exception:
+        ch.close()
+        raise
+
+
+SHAPES = [(1, None), (31, None), (33, 36), (513, None), (2000, 2000), (4097, 4100), (10007, None)]
+
+
+@pytest.mark.parametrize("d,ld", SHAPES)
+def test_sign_shapes(d, ld):
+    ch, _, _ = run_lockstep(workloads.ring(5), "sign", 5, d, 3, ld=ld, seed=d)
+    assert choco.choco_message_bytes(ch.ctx)[0] == 4 * ((d + 31) // 32) + 4
+    ch.close()
+
+
+@pytest.mark.parametrize("d,ld", SHAPES)
+@pytest.mark.parametrize("bucket", [0, 128, 512, 1024])
+def test_qsgd_shapes(d, ld, bucket):
+    run_lockstep(workloads.ring(4), "qsgd", 4, d, 3, s=16, bucket=bucket, ld=ld, seed=d + bucket)[0].close()
+
+
+@pytest.mark.parametrize("s", [2, 4, 8, 32, 128])
+@pytest.mark.parametrize("biased", [True, False])
+def test_qsgd_level_counts(s, biased):
+    run_lockstep(workloads.ring(4), "qsgd", 4, 3000, 2, s=s, bucket=256, biased=biased, seed=s)[0].close()
+
+
+@pytest.mark.parametrize("d,ld", SHAPES)
+def test_identity_shapes(d, ld):
+    run_lockstep(workloads.torus(3, 3), "identity", 9, d, 2, ld=ld, seed=d, gamma=1.0)[0].close()
+
+
+@pytest.mark.parametrize("d,k,ld", [(1, 1, None), (31, 5, None), (33, 33, 36), (513, 1, None),
+                                    (2000, 20, None), (4097, 300, 4100), (10007, 100, None),
+                                    (10007, 10007, None), (50000, 500, None)])
+def test_topk_shapes(d, k, ld):
+    ch, _, _ = run_lockstep(workloads.ring(5), "topk", 5, d, 3, k=k, ld=ld, seed=d + k)
+    assert choco.choco_message_bytes(ch.ctx) == (8 * k, 8 * k * 5)
+    ch.close()
+
+
+@pytest.mark.parametrize("d,k,ld", [(1, 1, None), (33, 7, 36), (2000, 20, None), (4097, 300, None),
+                                    (10007, 100, None), (10007, 10007, None), (50000, 5000, None)])
+def test_randk_shapes(d, k, ld):
+    ch, _, _ = run_lockstep(workloads.ring(5), "randk", 5, d, 3, k=k, ld=ld, seed=d + k)
+    assert choco.choco_message_bytes(ch.ctx) == (4 * k, 4 * k * 5)
+    ch.close()
+
+
+def test_topk_ties_zeros_and_signed_zero():
+    n, d, k = 4, 9000, 700
+    rng = np.random.default_rng(0)
+    x = np.zeros((n, d), dtype=np.float32)
+    x[0] = rng.choice([-2.0, 2.0, 1.0, -1.0], size=d).astype(np.float32)      # massive ties
+    x[1, ::3] = -0.0                                                         # all-zero row, some -0
+    x[2] = rng.integers(-3, 4, size=d).astype(np.float32)                   # few distinct values
+    x[3] = rng.standard_normal(d).astype(np.float32)
+    x[3, 100:140] = x[3, 50]                                                 # a tie at some value
+    ch, _, _ = run_lockstep(workloads.ring(n), "topk", n, d, 4, k=k, x_init=x, seed=1)
+    st = choco.choco_get_stats(ch.ctx)
+    assert st["exact_rows"] > 0          # the tie-heavy rows went through the exact selection
+    ch.close()
+
+
+def test_irregular_graph_sparse_and_dense():
+    w = workloads.random_graph(32, 14, 1)
+    run_lockstep(w, "topk", 32, 6000, 3, k=60, seed=2)[0].close()
+    run_lockstep(w, "sign", 32, 6000, 2, seed=3)[0].close()
+
+
+def test_momentum_variant():
+    run_lockstep(workloads.ring(4), "topk", 4, 5000, 4, k=50, momentum=True, seed=4)[0].close()
+    run_lockstep(workloads.ring(4), "sign", 4, 5000, 3, momentum=True, seed=5)[0].close()
+
+
+def test_config1_full_run_and_consensus():
+    wl = workloads.WORKLOADS["c1_ring4_topk"]
+    X0 = workloads.normal_rows(wl.n, wl.d, 1.0, 0)
+    e0 = oracle.consensus_error(X0)
+    ch, (dX, _, _), (X, _, _) = run_lockstep(wl.mixing(), "topk", wl.n, wl.d, wl.steps, k=wl.k,
+                                             gamma=wl.gamma, sgd=False, x_init=X0, check_msgs=False)
+    got = choco.choco_consensus_error(ch.ctx, dX) / e0
+    want = oracle.consensus_error(X) / e0
+    assert abs(got - want) <= 1e-4 * want
+    assert want < 0.1
+    ch.close()
+
+
+@pytest.mark.parametrize("name", ["c2_ring16_randk", "c2_ring16_qsgd"])
+def test_config2_logistic_regression(name):
+    wl = workloads.WORKLOADS[name]
+    prob = workloads.LogisticProblem(wl.n, wl.d, 256, seed=3)
+    x0 = np.zeros((wl.n, wl.d), dtype=np.float32)
+    ch, _, (X, _, _) = run_lockstep(wl.mixing(), wl.q, wl.n, wl.d, 120, k=wl.k, s=wl.s,
+                                    bucket=wl.bucket, eta=wl.eta, gamma=wl.gamma, x_init=x0, seed=9,
+                                    grad_fn=lambda t, x: prob.gradient(x, t), check_msgs=False)
+    assert prob.loss(X.mean(axis=0)) < prob.loss(np.zeros(wl.d, np.float32))
+    ch.close()
+
+
+def test_config3_shape_sign():
+    wl = workloads.WORKLOADS["c3_ring8_sign"]
+    ch, _, _ = run_lockstep(wl.mixing(), "sign", wl.n, wl.d, 4, eta=wl.eta, gamma=wl.gamma,
+                            x_var=wl.x_var, g_var=wl.g_var, seed=3)
+    assert choco.choco_message_bytes(ch.ctx)[0] == 34064
+    ch.close()
+
+
+def test_resume_from_checkpoint_is_bit_exact():
+    w = workloads.ring(6)
+    n, d = 6, 7000
+    X0 = workloads.normal_rows(n, d, 1.0, 77)
+    G = [_dev(workloads.normal_rows(n, d, 0.01, 900 + t)) for t in range(6)]
+
+    def run(ch, state, t0, t1):
+        for t in range(t0, t1):
+            ch.sgd_step(state[0], state[1], state[2], G[t], 0.05, 0.1)
+
+    a = choco.Choco(w, d, "qsgd", s=16, bucket=512, seed=5)
+    sa = [_dev(X0), torch.zeros(n, d, device=DEV), torch.zeros(n, d, device=DEV)]
+    run(a, sa, 0, 6)
+    b = choco.Choco(w, d, "qsgd", s=16, bucket=512, seed=5)
+    sb = [_dev(X0), torch.zeros(n, d, device=DEV), torch.zeros(n, d, device=DEV)]
+    run(b, sb, 0, 3)
+    saved = [t.clone() for t in sb]
+    b.close()
+    c = choco.Choco(w, d, "qsgd", s=16, bucket=512, seed=5)
+    choco.choco_set_step(c.ctx, 3)
+    run(c, saved, 3, 6)
+    torch.cuda.synchronize()
+    for x, y in zip(sa, saved):
+        assert torch.equal(x, y)
+    a.close(); c.close()
+
+
+def test_host_buffer_entry_point():
+    w = workloads.ring(4)
+    n, d = 4, 5000
+    X = workloads.normal_rows(n, d, 1.0, 1)
+    G = workloads.normal_rows(n, d, 0.01, 2)
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    oX, oXh, oS = X.copy(), Xh.copy(), S.copy()
+    ch = choco.Choco(w, d, "topk", k=50)
+    p = oracle.Params("topk", k=50)
+    for t in range(2):
+        oracle.step(w, p, oX, oXh, oS, G, 0.1, 0.2, t)
+        choco.choco_sgd_step_host(ch.ctx, X, Xh, S, G, 0.1, 0.2)
+        assert_state(X, oX, "X (host call)")
+        assert_state(Xh, oXh, "Xhat (host call)")
+        assert_state(S, oS, "S (host call)")
+    ch.close()
