@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Throughput of the CHOCO-SGD step (coordinates per second) on synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one call of choco_sgd_step over all n workers: compress x - x^, update the
+public copies and neighbour sums, gossip correction and SGD step.  The default workload is
+the 8x8-torus, d = 1e6, top-1 % shape.  Prints ONE JSON line.
+
+The path does not shard (one GPU holds all simulated workers), so --gpus N > 1 runs N
+independent replicas, one per process, and reports their aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+L2_BYTES = 126 * 2 ** 20
+NOMINAL_HBM_GBS = 8000.0           # the figure the 60 % target is quoted against
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# byte model: what one step must move (each dense array once, messages once per reader)
+# ------------------------------------------------------------------------------------------
+
+
+def message_bytes(wl) -> int:
+    d = wl.d
+    if wl.q == "topk":
+        return 8 * wl.k
+    if wl.q == "randk":
+        return 4 * wl.k
+    if wl.q == "sign":
+        return 4 * ((d + 31) // 32) + 4
+    if wl.q == "qsgd":
+        blen = wl.bucket or d
+        wbits = 1
+        while (1 << wbits) < wl.s:
+            wbits *= 2
+        return 4 * ((d + blen - 1) // blen) + 4 * ((d + 31) // 32) + (d * wbits + 7) // 8
+    return 4 * d
+
+
+def step_min_bytes(wl, w, sgd=True) -> int:
+    """Whole step: X, Xhat, S (and G) read once, every densely changing array written once,
+    messages written once and read once per off-diagonal neighbour, sparse updates at 4 B."""
+    N = wl.n * wl.d
+    nnz = int(w.row_ptr[-1])
+    deg_off = nnz - wl.n
+    msg = message_bytes(wl)
+    if wl.q in ("topk", "randk"):
+        dense = (20 if sgd else 16) * N
+        return dense + msg * wl.n + msg * deg_off + 4 * (wl.n * wl.k + nnz * wl.k)
+    dense = (28 if sgd else 24) * N
+    return dense + msg * wl.n + msg * deg_off
+
+
+def update_kernel_bytes(wl, w, sgd=True) -> int:
+    """The update kernel alone: reads X, Xhat, S, G and every neighbour's message (self
+    included), writes X densely and Xhat, S where touched (all of them for dense Q)."""
+    N = wl.n * wl.d
+    nnz = int(w.row_ptr[-1])
+    msg = message_bytes(wl)
+    if wl.q in ("topk", "randk"):
+        per_entry = 8                                   # index + value as read by the kernel
+        return (20 if sgd else 16) * N + per_entry * wl.k * nnz + 4 * (wl.n * wl.k + nnz * wl.k)
+    return (28 if sgd else 24) * N + msg * nnz
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 6] or \
+               [r for _, r in self.rows if len(r) >= 6]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        mhz = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
+                "samples": len(rows)}
+
+
+# ------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands (baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------
+
+
+def oracle_sample(wl, w, budget_rows=None):
+    """Run one oracle step on (a row sample of) the workload; returns (coords, seconds, text)."""
+    import oracle
+    rows = list(range(wl.n)) if budget_rows is None else list(range(min(budget_rows, wl.n)))
+    need = sorted({int(c) for i in rows for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]]})
+    remap = {j: a for a, j in enumerate(need)}
+    X = workloads.normal_rows(len(need), wl.d, wl.x_var or 1.0, 11)
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    G = workloads.normal_rows(len(need), wl.d, wl.g_var or 1e-2, 12)
+    # a sub-problem holding only the needed rows, W's rows restricted accordingly
+    rp, col, val = [0], [], []
+    for j in need:
+        if j in rows:
+            for e in range(w.row_ptr[j], w.row_ptr[j + 1]):
+                col.append(remap[int(w.col[e])]); val.append(float(w.val[e]))
+        else:
+            col.append(remap[j]); val.append(1.0)
+        rp.append(len(col))
+    sub = workloads.MixingCSR(len(need), np.asarray(rp, np.int32), np.asarray(col, np.int32),
+                              np.asarray(val, np.float32))
+    p = oracle.Params(wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=1)
+    t0 = time.perf_counter()
+    oracle.step(sub, p, X, Xh, S, G, wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
+    dt = time.perf_counter() - t0
+    text = (f"one oracle step for {len(rows)} of {wl.n} workers of {wl.name} "
+            f"(their {len(need)} neighbours' messages formed too), single thread")
+    return len(rows) * wl.d, dt, text
+
+
+def rows_for_budget(wl) -> int:
+    # about 10-30 s of single-thread work: ~0.15 s per million coordinates compressed + applied
+    per_row = 0.25 * wl.d / 1e6 * (3 if wl.q in ("topk", "randk") else 1)
+    return max(1, min(wl.n, int(20.0 / max(per_row, 1e-3))))
+
+
+# ------------------------------------------------------------------------------------------
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="c4_torus64_topk", choices=sorted(workloads.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pool", type=int, default=8, help="gradient tensors cycled through (>= 2)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = workloads.WORKLOADS[args.workload]
+    w = wl.mixing()
+    N = wl.n * wl.d
+    config = {"workload": wl.name, "n": wl.n, "d": wl.d, "graph": wl.graph, "Q": wl.q,
+              "k": wl.k, "s": wl.s, "bucket": wl.bucket, "eta": wl.eta, "gamma": wl.gamma,
+              "parallelism": "replicas only" if args.gpus > 1 else "single GPU",
+              "l2": "inputs per step exceed L2" if 20 * N > 2 * L2_BYTES else "state fits L2 (no flush)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        times = []
+        coords = 0
+        text = ""
+        rows = rows_for_budget(wl)
+        rows = max(1, rows // max(1, args.steps + args.warmup))
+        for i in range(args.warmup + args.steps):
+            coords, dt, text = oracle_sample(wl, w, rows)
+            if i >= args.warmup:
+                times.append(dt)
+        val = coords * len(times) / sum(times)
+        print(json.dumps({
+            "impl": "reference", "metric": "coords_per_sec", "value": val, "unit": "coords/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": val, "unit": "coords/s", "cores": 1, "kind": "oracle",
+                             "sample": text},
+            "e2e": {"value": val, "unit": "coords/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_1907_09356_b200 as choco
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234 + rank)
+    X = torch.randn(wl.n, wl.d, device=dev, generator=gen) * float(np.sqrt(wl.x_var or 1.0))
+    Xh = torch.zeros_like(X)
+    S = torch.zeros_like(X)
+    free_b = torch.cuda.mem_get_info(dev)[0]
+    pool_n = int(max(2, min(args.pool, (free_b * 0.5) // (4 * N))))
+    pool = [torch.randn(wl.n, wl.d, device=dev, generator=gen) * float(np.sqrt(wl.g_var or 1e-2))
+            for _ in range(pool_n)]
+    ch = choco.Choco(w, wl.d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=7)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        ch.sgd_step(X, Xh, S, pool[t % pool_n], wl.eta, wl.gamma)
+    barrier()
+    st0 = choco.choco_get_stats(ch.ctx)
+    choco.choco_profile_enable(ch.ctx, args.steps)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record()
+    for t in range(args.steps):
+        ch.sgd_step(X, Xh, S, pool[(args.warmup + t) % pool_n], wl.eta, wl.gamma)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    st1 = choco.choco_get_stats(ch.ctx)
+    nrec, upd_ms = choco.choco_profile_read(ch.ctx)
+    finite = bool(torch.isfinite(X).all())
+
+    # end to end: host buffers in, host buffers out, through choco_sgd_step_host
+    e2e = None
+    if args.e2e_steps > 0:
+        hX, hXh, hS = (t.cpu().pin_memory() for t in (X, Xh, S))
+        hG = pool[0].cpu().pin_memory()
+        choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)      # warm-up, allocates staging
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        e2e = {"seconds": e2e_s, "steps": args.e2e_steps}
+
+    if world > 1:
+        tt = torch.tensor([ms, e2e["seconds"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt[0]);
+        if e2e:
+            e2e["seconds"] = float(tt[1])
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        ms_step = ms / args.steps
+        value = world * N * args.steps / (ms * 1e-3)
+        upd_bytes = update_kernel_bytes(wl, w)
+        upd_avg_s = (upd_ms / max(nrec, 1)) * 1e-3
+        achieved = upd_bytes / upd_avg_s / 1e9 if nrec else None
+        step_bytes = step_min_bytes(wl, w)
+        step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
+        out = {
+            "metric": "coords_per_sec", "value": value, "unit": "coords/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config,
+            "steps_per_sec": 1e3 / ms_step,
+            "compressed_bytes_per_step": message_bytes(wl) * wl.n,
+            "step_min_bytes": step_bytes, "step_hbm_gbs": step_gbs,
+            "step_frac_of_measured_peak": step_gbs / peak,
+            "step_frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "kernel": "update (apply) kernel", "achieved": achieved,
+                         "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                         "frac": (achieved / peak) if achieved else None,
+                         "traffic": None, "algorithmic_bytes_per_launch": upd_bytes,
+                         "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec},
+            "gpu_launches": int(st1["kernel_launches"] - st0["kernel_launches"]),
+            "selection": {k: int(st1[k] - st0[k]) for k in ("prepared_rows", "recompressed_rows", "exact_rows")},
+            "finite": finite,
+            "clocks": clocks,
+        }
+        if e2e:
+            out["e2e"] = {"value": world * N * e2e["steps"] / e2e["seconds"], "unit": "coords/s",
+                          "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,
+                          "steps": e2e["steps"], "api": "choco_sgd_step_host, pinned host buffers"}
+        if not args.no_cpu_baseline and world == 1:
+            coords, dt, text = oracle_sample(wl, w, rows_for_budget(wl))
+            out["cpu_baseline"] = {"value": coords / dt, "unit": "coords/s", "cores": 1,
+                                   "kind": "oracle", "sample": text, "seconds": dt}
+        print(json.dumps(out))
+    ch.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

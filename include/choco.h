@@ -177,8 +177,20 @@ typedef struct {
     uint64_t prepared_rows;    /* rows whose compression was prepared by the previous step     */
     uint64_t recompressed_rows;/* rows compressed by a separate pass over X and Xhat           */
     uint64_t exact_rows;       /* rows that needed the slow exact selection                    */
+    uint64_t kernel_launches;  /* kernels the step calls have enqueued                         */
 } choco_stats;
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
+
+/*
+ * Optional timing of the update kernel (the one pass that streams X, Xhat, S and G): after
+ * choco_profile_enable the next `max_steps` step calls record a CUDA event before and after
+ * that kernel on the step's stream.  choco_profile_read synchronises `stream` and returns
+ * how many steps were recorded and the sum of their update-kernel durations in
+ * milliseconds, then clears the record.  Not part of the method; used by benchmarks.
+ */
+int choco_profile_enable(choco_ctx* ctx, int32_t max_steps);
+int choco_profile_read(choco_ctx* ctx, int32_t* steps_recorded, double* update_ms_total,
+                       void* stream);
 
 const char* choco_strerror(int code);
 /* cudaError_t of the last failing CUDA call on this context (0 if none). */

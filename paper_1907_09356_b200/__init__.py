@@ -23,7 +23,8 @@ EXPORTS = [
     "choco_sgd_momentum_step", "choco_sgd_step_host", "choco_invalidate", "choco_get_step",
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error",
-    "choco_get_stats", "choco_strerror", "choco_last_cuda_error",
+    "choco_get_stats", "choco_profile_enable", "choco_profile_read", "choco_strerror",
+    "choco_last_cuda_error",
 ]
 
 
@@ -38,7 +39,8 @@ class choco_params(ctypes.Structure):
 
 class choco_stats(ctypes.Structure):
     _fields_ = [("steps", ctypes.c_uint64), ("prepared_rows", ctypes.c_uint64),
-                ("recompressed_rows", ctypes.c_uint64), ("exact_rows", ctypes.c_uint64)]
+                ("recompressed_rows", ctypes.c_uint64), ("exact_rows", ctypes.c_uint64),
+                ("kernel_launches", ctypes.c_uint64)]
 
 
 _lib = None
@@ -69,6 +71,8 @@ def load() -> ctypes.CDLL:
         lib.choco_read_message.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
         lib.choco_consensus_error.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), vp]
         lib.choco_get_stats.argtypes = [vp, ctypes.POINTER(choco_stats), vp]
+        lib.choco_profile_enable.argtypes = [vp, i32]
+        lib.choco_profile_read.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double), vp]
         lib.choco_strerror.argtypes = [ctypes.c_int]
         lib.choco_strerror.restype = ctypes.c_char_p
         lib.choco_last_cuda_error.argtypes = [vp]
@@ -195,6 +199,17 @@ def choco_get_stats(ctx, stream=None) -> dict:
     st = choco_stats()
     _check(load().choco_get_stats(ctx, ctypes.byref(st), _stream(stream)), ctx)
     return {f: getattr(st, f) for f, _ in choco_stats._fields_}
+
+
+def choco_profile_enable(ctx, max_steps: int) -> None:
+    _check(load().choco_profile_enable(ctx, max_steps), ctx)
+
+
+def choco_profile_read(ctx, stream=None) -> tuple[int, float]:
+    """(steps recorded, total milliseconds spent in the update kernel over them)."""
+    n, ms = ctypes.c_int32(), ctypes.c_double()
+    _check(load().choco_profile_read(ctx, ctypes.byref(n), ctypes.byref(ms), _stream(stream)), ctx)
+    return n.value, ms.value
 
 
 # --------------------------------------------------------------------------- convenience

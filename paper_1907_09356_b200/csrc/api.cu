@@ -91,6 +91,7 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     a.X = X; a.Xhat = Xhat; a.S = S; a.G = G; a.M = M;
     a.eta = eta; a.gamma = gamma; a.lambda = lambda; a.beta = beta;
     a.step = ctx->step;
+    a.launches = &ctx->launches;
     a.vec = (dv.ld % 4 == 0) && aligned16(X) && aligned16(Xhat) && aligned16(S) &&
             (!G || aligned16(G)) && (!M || aligned16(M));
     if (ctx->last_x != X || ctx->last_xhat != Xhat) ctx->prepared = false;
@@ -103,7 +104,13 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     } else {
         e = launch_compress_dense(dv, a, st);
     }
+    const bool prof = ctx->prof_ev && ctx->prof_n < ctx->prof_cap;
+    if (e == cudaSuccess && prof) e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], st);
     if (e == cudaSuccess) e = launch_apply(dv, a, st);
+    if (e == cudaSuccess && prof) {
+        e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], st);
+        ctx->prof_n += 1;
+    }
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->prepared = false; // nothing is carried across steps yet
     ctx->last_x = X;
@@ -239,6 +246,10 @@ int choco_destroy(choco_ctx* ctx)
     for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
     for (int i = 0; i < 4; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    if (ctx->prof_ev) {
+        for (int i = 0; i < 2 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+        delete[] ctx->prof_ev;
+    }
     delete ctx;
     return CHOCO_OK;
 }
@@ -394,6 +405,50 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
     out->prepared_rows = h.prepared_rows;
     out->recompressed_rows = h.recompressed_rows;
     out->exact_rows = h.exact_rows;
+    out->kernel_launches = ctx->launches;
+    return CHOCO_OK;
+}
+
+int choco_profile_enable(choco_ctx* ctx, int32_t max_steps)
+{
+    if (!ctx || max_steps < 1 || max_steps > 100000) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->prof_ev) {
+        for (int i = 0; i < 2 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+        delete[] ctx->prof_ev;
+        ctx->prof_ev = nullptr;
+    }
+    ctx->prof_ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_steps];
+    if (!ctx->prof_ev) return CHOCO_ERR_ALLOC;
+    ctx->prof_cap = 0;
+    ctx->prof_n = 0;
+    for (int i = 0; i < 2 * max_steps; ++i) {
+        cudaError_t e = cudaEventCreate(&ctx->prof_ev[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(ctx->prof_ev[j]);
+            delete[] ctx->prof_ev;
+            ctx->prof_ev = nullptr;
+            return fail_cuda(ctx, e);
+        }
+    }
+    ctx->prof_cap = max_steps;
+    return CHOCO_OK;
+}
+
+int choco_profile_read(choco_ctx* ctx, int32_t* steps_recorded, double* update_ms_total,
+                       void* stream)
+{
+    if (!ctx || !steps_recorded || !update_ms_total) return CHOCO_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    double total = 0.0;
+    for (int i = 0; e == cudaSuccess && i < ctx->prof_n; ++i) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]);
+        total += (double)ms;
+    }
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    *steps_recorded = ctx->prof_n;
+    *update_ms_total = total;
+    ctx->prof_n = 0;
     return CHOCO_OK;
 }
 

@@ -240,6 +240,7 @@ cudaError_t launch_apply(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
     if (a.vec) apply_vec<true>(dv, a, st);
     else apply_vec<false>(dv, a, st);
+    *a.launches += 1;
     return cudaGetLastError();
 }
 

@@ -208,11 +208,13 @@ static cudaError_t compress_impl(const Dev& dv, const StepArgs& a, cudaStream_t 
     case CHOCO_Q_SIGN:
         norm_partial_kernel<VEC, NORM_L1, true><<<grid, kThreads, 0, st>>>(dv, a);
         norm_finish_kernel<NORM_L1><<<dv.n, 1024, 0, st>>>(dv);
+        *a.launches += 2;
         break;
     case CHOCO_Q_QSGD:
         if (dv.bucket == 0) {
             norm_partial_kernel<VEC, NORM_L2SQ, false><<<grid, kThreads, 0, st>>>(dv, a);
             norm_finish_kernel<NORM_L2SQ><<<dv.n, 1024, 0, st>>>(dv);
+            *a.launches += 2;
         }
         switch (dv.wbits) {
         case 1: launch_qsgd_pack<VEC, 1>(dv, a, grid, st); break;
@@ -220,9 +222,11 @@ static cudaError_t compress_impl(const Dev& dv, const StepArgs& a, cudaStream_t 
         case 4: launch_qsgd_pack<VEC, 4>(dv, a, grid, st); break;
         default: launch_qsgd_pack<VEC, 8>(dv, a, grid, st); break;
         }
+        *a.launches += 1;
         break;
     default:
         identity_kernel<VEC><<<grid, kThreads, 0, st>>>(dv, a);
+        *a.launches += 1;
         break;
     }
     return cudaGetLastError();

@@ -83,6 +83,7 @@ struct StepArgs {
     float eta, gamma, lambda, beta;
     uint64_t step;
     bool vec;                    // rows 16-byte aligned: 128-bit accesses
+    unsigned long long* launches; // host counter of kernels enqueued (not used on the device)
 };
 
 // selection (top-k / random-k)
@@ -115,6 +116,10 @@ struct choco_ctx {
     double* cons_scratch;
     int64_t cons_blocks;
     double* cons_out;
+    unsigned long long launches;
+    // optional event pairs around the update kernel
+    cudaEvent_t* prof_ev;
+    int prof_cap, prof_n;
     // all device allocations, for choco_destroy
     void* allocs[64];
     int nallocs;

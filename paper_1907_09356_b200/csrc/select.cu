@@ -473,15 +473,18 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
         if (a.vec) hist_kernel<true><<<grid, kThreads, 0, st>>>(dv, a);
         else hist_kernel<false><<<grid, kThreads, 0, st>>>(dv, a);
         bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv);
+        *a.launches += 2;
     } else {
         // keep words <= hi: about k + 6 sqrt(k) + 16 of d coordinates
         const double kk = (double)dv.k;
         double frac = (kk + 6.0 * sqrt(kk) + 16.0) / (double)dv.d;
         uint32_t hi = frac >= 1.0 ? 0xFFFFFFFFu : (uint32_t)(frac * 4294967296.0);
         randk_bound_kernel<<<(dv.n + 127) / 128, 128, 0, st>>>(dv, ~hi);
+        *a.launches += 1;
     }
     if (a.vec) collect_kernel<KIND, true><<<grid, kThreads, 0, st>>>(dv, a);
     else collect_kernel<KIND, false><<<grid, kThreads, 0, st>>>(dv, a);
+    *a.launches += 1;
     return cudaGetLastError();
 }
 
@@ -497,6 +500,7 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, cudaStream_t st)
     emit_kernel<KIND><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     if (a.vec) exact_kernel<KIND, true><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     else exact_kernel<KIND, false><<<dv.n, kSelThreads, 0, st>>>(dv, a);
+    *a.launches += 2;
     return cudaGetLastError();
 }
 
