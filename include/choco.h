@@ -137,8 +137,12 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
  * pointers; a change of pointers is detected, a change of contents is not.
  * choco_invalidate -- call after modifying X or Xhat outside the library (for example
  * when loading a checkpoint into the same buffers).
+ * choco_set_carry -- enable = 0 turns the carrying off (every step then compresses from X
+ * and Xhat as it finds them, at the cost of one more pass over both); default on.  The
+ * results are the same either way.
  */
 int choco_invalidate(choco_ctx* ctx);
+int choco_set_carry(choco_ctx* ctx, int32_t enable);
 
 /* Step counter t (keys the generator).  Setting it, together with restoring X, Xhat and S,
  * resumes a run bit-exactly; choco_set_step implies choco_invalidate. */
@@ -178,6 +182,7 @@ typedef struct {
     uint64_t recompressed_rows;/* rows compressed by a separate pass over X and Xhat           */
     uint64_t exact_rows;       /* rows that needed the slow exact selection                    */
     uint64_t kernel_launches;  /* kernels the step calls have enqueued                         */
+    uint64_t device_timeouts;  /* bounded waits inside kernels that ran out (must stay 0)      */
 } choco_stats;
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
 

@@ -98,21 +98,24 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
 
     cudaError_t e = cudaSuccess;
     const bool sparse = dv.kind == CHOCO_Q_TOPK || dv.kind == CHOCO_Q_RANDK;
+    const bool was_prepared = ctx->prepared;
     if (sparse) {
-        if (!ctx->prepared) e = launch_select_prepare(dv, a, st);
-        if (e == cudaSuccess) e = launch_select_emit(dv, a, st);
+        if (!was_prepared) e = launch_select_prepare(dv, a, st);
+        if (e == cudaSuccess) e = launch_select_emit(dv, a, was_prepared, st);
     } else {
         e = launch_compress_dense(dv, a, st);
     }
+    // the update kernel can collect the next step's candidates from the x' - x^' it holds
+    const bool emit = ctx->carry_enabled && apply_can_emit(dv, a);
     const bool prof = ctx->prof_ev && ctx->prof_n < ctx->prof_cap;
     if (e == cudaSuccess && prof) e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], st);
-    if (e == cudaSuccess) e = launch_apply(dv, a, st);
+    if (e == cudaSuccess) e = launch_apply(dv, a, emit, st);
     if (e == cudaSuccess && prof) {
         e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], st);
         ctx->prof_n += 1;
     }
     if (e != cudaSuccess) return fail_cuda(ctx, e);
-    ctx->prepared = false; // nothing is carried across steps yet
+    ctx->prepared = emit;
     ctx->last_x = X;
     ctx->last_xhat = Xhat;
     ctx->step += 1;
@@ -157,6 +160,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     if (!ctx) return CHOCO_ERR_ALLOC;
     std::memset(ctx, 0, sizeof(*ctx));
     ctx->params = *p;
+    ctx->carry_enabled = true;
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
     dv.ntiles = (d + kTile - 1) / kTile;
@@ -178,7 +182,8 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     if (p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK) {
         dv.k = p->k;
         dv.kpitch = round_up(p->k, 4);
-        int64_t cap = 4 * p->k > p->k + 8192 ? 4 * p->k : p->k + 8192;
+        // candidates per row: aimed at 2.5-3.5 k, with room for a bound that was guessed low
+        int64_t cap = 8 * p->k > p->k + 8192 ? 8 * p->k : p->k + 8192;
         dv.cap = cap < d ? cap : d;
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_idx, n * dv.kpitch);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_val, n * dv.kpitch);
@@ -292,8 +297,11 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     ctx->prepared = false; // the staging contents changed
+    const bool carry = ctx->carry_enabled;
+    ctx->carry_enabled = false; // the next call overwrites the staging buffers anyway
     const int rc = run_step(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], G ? ctx->stage[3] : nullptr,
                             nullptr, eta, gamma, 0.f, 0.f, stream);
+    ctx->carry_enabled = carry;
     if (rc) return rc;
     float* dst[3] = {X, Xhat, S};
     for (int i = 0; i < 3; ++i) {
@@ -309,6 +317,14 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
 int choco_invalidate(choco_ctx* ctx)
 {
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    ctx->prepared = false;
+    return CHOCO_OK;
+}
+
+int choco_set_carry(choco_ctx* ctx, int32_t enable)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    ctx->carry_enabled = enable != 0;
     ctx->prepared = false;
     return CHOCO_OK;
 }
@@ -405,6 +421,7 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
     out->prepared_rows = h.prepared_rows;
     out->recompressed_rows = h.recompressed_rows;
     out->exact_rows = h.exact_rows;
+    out->device_timeouts = h.timeouts;
     out->kernel_launches = ctx->launches;
     return CHOCO_OK;
 }

@@ -15,8 +15,8 @@ namespace choco {
 constexpr int kThreads = 256;            // threads per block of the streaming kernels
 constexpr int kQuad = 4;                 // coordinates per thread per iteration (one 128-bit access)
 constexpr int kChunk = kThreads * kQuad; // 1024 coordinates: one block iteration, one tree leaf group
-constexpr int kIters = 4;                // iterations per block
-constexpr int kTile = kChunk * kIters;   // 4096 coordinates per block
+constexpr int kIters = 2;                // iterations per block
+constexpr int kTile = kChunk * kIters;   // coordinates per block (2048)
 
 constexpr uint32_t kStreamRandK = 0;     // generator stream of the random-k selection keys
 constexpr uint32_t kStreamDither = 1;    // generator stream of the QSGD dither

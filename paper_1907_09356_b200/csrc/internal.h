@@ -17,6 +17,7 @@ struct Stats {
     unsigned long long prepared_rows;
     unsigned long long recompressed_rows;
     unsigned long long exact_rows;
+    unsigned long long timeouts;   // bounded device waits that ran out
 };
 
 // Everything the kernels need; passed by value.
@@ -88,11 +89,13 @@ struct StepArgs {
 
 // selection (top-k / random-k)
 cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t st);
-cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, cudaStream_t st);
+// fused: the candidates came from the previous step's update kernel (statistics only)
+cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st);
 // dense compressors
 cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st);
-// apply
-cudaError_t launch_apply(const Dev& dv, const StepArgs& a, cudaStream_t st);
+// update kernel; emit: also collect the next step's top-k candidates (if apply_can_emit)
+bool apply_can_emit(const Dev& dv, const StepArgs& a);
+cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 // metrics
 cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,
                              int64_t nblocks, double* out, cudaStream_t st);
@@ -107,6 +110,7 @@ struct choco_ctx {
     int device;
     int last_cuda_error;
     bool prepared;               // next step's candidates/messages already formed
+    bool carry_enabled;          // steps may prepare the next step's compression
     const float* last_x;
     const float* last_xhat;
     int64_t msg_bytes_per_worker;

@@ -1,34 +1,23 @@
 // Per-row selection of the k largest ordering keys: top_a and random_a of the paper's
 // Appendix C ("Compression Schemes").
 //
-// Ordering key of a coordinate: top_a -> bit pattern of |x - x^| (monotone for finite
-// floats; +0 and -0 tie); random_a -> complement of the coordinate's Philox word (so the k smallest words
-// win).  Ties go to the lower coordinate.  The message lists the chosen coordinates in
-// ascending order with their values x - x^, plus a table tile_ptr[t] = number of chosen
-// coordinates below 4096 t that lets a reader find any 4096-coordinate tile directly.
+// Ties go to the lower coordinate.  The message lists the chosen coordinates in ascending
+// order with their values x - x^, plus a table tile_ptr[t] = number of chosen coordinates
+// below kTile * t that lets a reader find any tile of coordinates directly.
 //
 // Pipeline (all device-side, no host decisions):
 //   prepare : histogram of the top 11 key bits -> lower key bound per row that keeps at
 //             least k coordinates -> collect those coordinates ("candidates") tile by tile,
-//             in ascending order inside a tile.
+//             in ascending order inside a tile.  (For top-k the update kernel of the previous
+//             step normally did this already, with a bound guessed from that step.)
 //   emit    : one block per row: exact k-th key by radix refinement over the candidates,
-//             tie ranks, ordered compaction into the message.
-//   exact   : rows whose candidates are unusable (too many equal keys, overflow) run a
+//             tie ranks, ordered compaction into the message; the candidate bound for the
+//             next step.
+//   exact   : rows whose candidates are unusable (too many, too few, overflow) run a
 //             one-block exact selection straight from the dense row.
-#include "common.cuh"
-#include "internal.h"
+#include "select.cuh"
 
 namespace choco {
-
-constexpr int kSelThreads = 1024;
-enum { SEL_TOPK = 0, SEL_RANDK = 1 };
-
-template <int KIND>
-__device__ __forceinline__ uint32_t order_key(uint32_t bits)
-{
-    // |v| without its sign bit, shifted up so that all 32 bits carry order information
-    return KIND == SEL_TOPK ? (bits << 1) : ~bits;
-}
 
 // value bits of the four coordinates of a quad (top-k: x - x^; random-k: Philox words)
 template <int KIND, bool VEC>
@@ -49,68 +38,7 @@ __device__ __forceinline__ void quad_bits(const Dev& dv, const StepArgs& a, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// block-wide helpers
-// ---------------------------------------------------------------------------------------
-
-// Exclusive prefix sum over the block (NT threads, NT a multiple of 32, at most 1024).
-// `sm` needs 33 words.  Returns the exclusive prefix; *total gets the block sum.
-template <int NT>
-__device__ __forceinline__ uint32_t block_scan_excl(uint32_t v, uint32_t* sm, uint32_t* total)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += t;
-    }
-    __syncthreads(); // protect sm from the previous use
-    if (lane == 31) sm[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t w = lane < NT / 32 ? sm[lane] : 0u;
-        uint32_t winc = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, winc, o);
-            if (lane >= o) winc += t;
-        }
-        sm[lane] = winc - w;
-        if (lane == 31) sm[32] = winc;
-    }
-    __syncthreads();
-    *total = sm[32];
-    return sm[warp] + inc - v;
-}
-
-// Given hist[0..nbins) (shared memory) find the largest digit D with
-// sum_{b >= D} hist[b] >= need; *above = sum_{b > D} hist[b].  nbins <= 2 * NT.
-// All threads return the same values.  `sm` needs 36 words.
-template <int NT>
-__device__ __forceinline__ void block_find_digit(const uint32_t* hist, int nbins, uint32_t need,
-                                                 uint32_t* sm, uint32_t* digit, uint32_t* above)
-{
-    const int r0 = 2 * threadIdx.x, r1 = r0 + 1;
-    const uint32_t h0 = r0 < nbins ? hist[nbins - 1 - r0] : 0u;
-    const uint32_t h1 = r1 < nbins ? hist[nbins - 1 - r1] : 0u;
-    uint32_t total;
-    const uint32_t ex = block_scan_excl<NT>(h0 + h1, sm, &total);
-    if (threadIdx.x == 0) { sm[34] = 0u; sm[35] = 0u; }
-    __syncthreads();
-    if (ex < need && need <= ex + h0) {
-        sm[34] = (uint32_t)(nbins - 1 - r0);
-        sm[35] = ex;
-    } else if (ex + h0 < need && need <= ex + h0 + h1) {
-        sm[34] = (uint32_t)(nbins - 1 - r1);
-        sm[35] = ex + h0;
-    }
-    __syncthreads();
-    *digit = sm[34];
-    *above = sm[35];
-}
-
-// ---------------------------------------------------------------------------------------
-// prepare 1: histogram of the top 11 bits of |x - x^| (top-k only)
+// prepare 1: histogram of the top 11 bits of the key of x - x^ (top-k only)
 // ---------------------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a)
@@ -149,8 +77,11 @@ __global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv)
         g[b] = 0u; // ready for the next use
     }
     __syncthreads();
+    // keep down to rank 3.5 k (not just k) so that emit can place the next step's bound
+    const uint64_t want = 3 * (uint64_t)dv.k + (uint64_t)dv.k / 2;
+    const uint32_t need = (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d);
     uint32_t digit, above;
-    block_find_digit<kSelThreads>(h, kHistBins, (uint32_t)dv.k, sm, &digit, &above);
+    block_find_digit<kSelThreads>(h, kHistBins, need, sm, &digit, &above);
     if (threadIdx.x == 0) {
         dv.row_lo[row] = digit << 21;
         dv.row_count[row] = 0u;
@@ -172,7 +103,7 @@ __global__ void randk_bound_kernel(Dev dv, uint32_t lo)
 }
 
 // ---------------------------------------------------------------------------------------
-// prepare 3: collect candidates, ascending inside each 4096-coordinate tile
+// prepare 3: collect candidates, ascending inside each tile
 // ---------------------------------------------------------------------------------------
 template <int KIND, bool VEC>
 __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
@@ -183,7 +114,6 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
     if (dv.row_flags[row] & kRowExact) return;
     const uint32_t lo = dv.row_lo[row];
     const int64_t c0 = (int64_t)blockIdx.x * kTile;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     uint32_t bits[kIters][4];
     uint32_t take = 0; // bit (4 it + e)
@@ -202,42 +132,17 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
                 }
         }
     }
-    // ordered slots: order is (iteration, thread, element).  Counts are scanned over the
-    // threads for the four iterations at once, two 16-bit fields per word.
-    uint32_t wa = cnt[0] | (cnt[1] << 16), wb = cnt[2] | (cnt[3] << 16);
-    uint32_t ia = wa, ib = wb;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o);
-        const uint32_t tb = __shfl_up_sync(0xffffffffu, ib, o);
-        if (lane >= o) { ia += ta; ib += tb; }
-    }
-    if (lane == 31) { sm[0][warp] = ia; sm[1][warp] = ib; }
-    __syncthreads();
+    uint32_t start[kIters], total;
+    ordered_starts(cnt, sm, start, &total);
     if (threadIdx.x == 0) {
-        uint32_t ra = 0, rb = 0;
-        for (int w = 0; w < kThreads / 32; ++w) {
-            const uint32_t ta = sm[0][w], tb = sm[1][w];
-            sm[0][w] = ra; sm[1][w] = rb;
-            ra += ta; rb += tb;
-        }
-        sm[0][8] = ra; sm[1][8] = rb;
-        const uint32_t total = (ra & 0xFFFFu) + (ra >> 16) + (rb & 0xFFFFu) + (rb >> 16);
         const uint32_t base = total ? atomicAdd(&dv.row_count[row], total) : 0u;
         dv.seg_off[(int64_t)row * dv.ntiles + blockIdx.x] = base;
         dv.seg_cnt[(int64_t)row * dv.ntiles + blockIdx.x] = total;
-        s_base = base;
-        if ((int64_t)base + total > dv.cap) s_base = 0xFFFFFFFFu; // overflow: emit sees count > cap
+        // past the capacity nothing is written; emit sees row_count > cap and gives up
+        s_base = ((int64_t)base + total > dv.cap) ? 0xFFFFFFFFu : base;
     }
     __syncthreads();
     if (s_base == 0xFFFFFFFFu) return;
-    const uint32_t ea = sm[0][warp] + ia - wa, eb = sm[1][warp] + ib - wb; // exclusive, per thread
-    const uint32_t ta = sm[0][8], tb = sm[1][8];
-    uint32_t start[kIters];
-    start[0] = ea & 0xFFFFu;
-    start[1] = (ta & 0xFFFFu) + (ea >> 16);
-    start[2] = (ta & 0xFFFFu) + (ta >> 16) + (eb & 0xFFFFu);
-    start[3] = (ta & 0xFFFFu) + (ta >> 16) + (tb & 0xFFFFu) + (eb >> 16);
     uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + s_base;
     uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + s_base;
 #pragma unroll
@@ -257,8 +162,61 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
 // ---------------------------------------------------------------------------------------
 // emit: exact selection among the candidates of a row, ordered output
 // ---------------------------------------------------------------------------------------
+
+// Radix refinement over the candidate values cv[0..ncand): the key of rank `rank`
+// (1 = largest) and how many candidates are strictly above it.
 template <int KIND>
-__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a)
+__device__ __forceinline__ void rank_key(const uint32_t* cv, uint32_t ncand, uint32_t rank,
+                                         uint32_t* h, uint32_t* sm, uint32_t* key_out,
+                                         uint32_t* above_out)
+{
+    uint32_t prefix = 0, pmask = 0, need = rank, above_total = 0;
+    const int shifts[3] = {21, 10, 0};
+    const int nbins[3] = {2048, 2048, 1024};
+    for (int pass = 0; pass < 3; ++pass) {
+        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
+        __syncthreads();
+        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+            const uint32_t key = order_key<KIND>(cv[p]);
+            if ((key & pmask) == prefix) atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
+        }
+        __syncthreads();
+        uint32_t digit, above;
+        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
+        need -= above;
+        above_total += above;
+        prefix |= digit << shifts[pass];
+        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
+        __syncthreads();
+    }
+    *key_out = prefix;
+    *above_out = above_total;
+}
+
+// Lower a key bound by `eighths` eighths of an octave (about 8 % of the value each).
+__device__ __forceinline__ uint32_t lower_bound_key(uint32_t key, uint32_t eighths)
+{
+    const uint32_t dec = eighths << 21;
+    return key > dec ? key - dec : 0u;
+}
+
+// Rank aimed at by the candidate bound: 3.5 k (the k chosen leave, about 2.5 k stay)
+__host__ __device__ __forceinline__ uint64_t target_rank(uint64_t k) { return 3 * k + k / 2; }
+
+// lo: bound the ncand candidates were collected with (their rank-ncand key, roughly);
+// T: key of rank k.  Linear in the key between the two ranks, at most half an octave down.
+__device__ __forceinline__ uint32_t next_bound(uint32_t lo, uint32_t T, uint32_t ncand, uint32_t k)
+{
+    if (ncand <= k || T < lo) return lower_bound_key(lo, 4u);
+    const uint64_t span = T - lo, want = target_rank(k), den = ncand - k;
+    if (ncand >= want) return lo + (uint32_t)((ncand - want) * span / den);
+    uint64_t dec = (want - ncand) * span / den;
+    if (dec > (4ull << 21)) dec = 4ull << 21;
+    return lo > dec ? (uint32_t)(lo - dec) : 0u;
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused)
 {
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t sm[36];
@@ -279,27 +237,17 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a)
     const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
     const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
 
-    // k-th largest key T by three radix digits (11, 11, 10 bits)
-    uint32_t prefix = 0, pmask = 0, need = k;
-    const int shifts[3] = {21, 10, 0};
-    const int nbins[3] = {2048, 2048, 1024};
-    for (int pass = 0; pass < 3; ++pass) {
-        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
-        __syncthreads();
-        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
-            const uint32_t key = order_key<KIND>(cv[p]);
-            if ((key & pmask) == prefix) atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
-        }
-        __syncthreads();
-        uint32_t digit, above;
-        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
-        need -= above;
-        prefix |= digit << shifts[pass];
-        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
-        __syncthreads();
+    uint32_t T, above;
+    rank_key<KIND>(cv, ncand, k, h, sm, &T, &above);
+    const uint32_t r = k - above; // how many coordinates with key == T are kept (lowest first)
+
+    if (KIND == SEL_TOPK) {
+        // Candidate bound for the next step: only a guess (the next step verifies that it kept
+        // at least k coordinates and otherwise selects exactly from the dense row).  The k
+        // chosen coordinates drop to ~0, so aim the bound at today's rank 3.5 k, reading the
+        // key of that rank off a straight line through (rank k, T) and (rank ncand, bound).
+        if (threadIdx.x == 0) dv.row_lo[row] = next_bound(dv.row_lo[row], T, ncand, k);
     }
-    const uint32_t T = prefix;  // k-th largest key
-    const uint32_t r = need;    // how many coordinates with key == T are kept (lowest first)
 
     // per tile: candidates above T, candidates equal to T
     const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
@@ -372,7 +320,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a)
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
-        atomicAdd(&dv.stats->recompressed_rows, 1ull);
+        atomicAdd(fused ? &dv.stats->prepared_rows : &dv.stats->recompressed_rows, 1ull);
     }
 }
 
@@ -388,7 +336,9 @@ __global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
     const int row = blockIdx.x;
     if (!(dv.row_flags[row] & kRowExact)) return;
     const uint32_t k = (uint32_t)dv.k;
-    const int64_t span = (int64_t)kSelThreads * kQuad; // 4096 = one tile per iteration
+    const int64_t span = (int64_t)kSelThreads * kQuad; // coordinates per block iteration
+    const int64_t nspan = (dv.d + span - 1) / span;
+    constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
     uint32_t prefix = 0, pmask = 0, need = k;
     const int shifts[3] = {21, 10, 0};
     const int nbins[3] = {2048, 2048, 1024};
@@ -419,9 +369,9 @@ __global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
     uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
     const float* xr = a.X + (int64_t)row * dv.ld;
     const float* hr = a.Xhat + (int64_t)row * dv.ld;
-    uint32_t run_gt = 0, run_eq = 0; // coordinates above / equal to T before this tile
-    for (int64_t t = 0; t < dv.ntiles; ++t) {
-        const int64_t c = t * span + (int64_t)threadIdx.x * kQuad;
+    uint32_t run_gt = 0, run_eq = 0; // coordinates above / equal to T before this span
+    for (int64_t sp = 0; sp < nspan; ++sp) {
+        const int64_t c = sp * span + (int64_t)threadIdx.x * kQuad;
         uint32_t bits[4] = {0u, 0u, 0u, 0u};
         uint32_t gtm = 0, eqm = 0;
         if (c < dv.d) {
@@ -437,8 +387,12 @@ __global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
         }
         uint32_t tot;
         const uint32_t ex = block_scan_excl<kSelThreads>(__popc(gtm) | (__popc(eqm) << 16), sm, &tot);
-        if (threadIdx.x == 0) tp[t] = run_gt + (run_eq < r ? run_eq : r);
         uint32_t g = run_gt + (ex & 0xFFFFu), q = run_eq + (ex >> 16);
+        // the first thread of every tile records how many coordinates were chosen before it
+        if ((threadIdx.x % (kTile / kQuad)) == 0) {
+            const int64_t t = sp * kTilesPerSpan + threadIdx.x / (kTile / kQuad);
+            if (t < dv.ntiles) tp[t] = g + (q < r ? q : r);
+        }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const bool isgt = (gtm >> e) & 1u, iseq = (eqm >> e) & 1u;
@@ -457,6 +411,8 @@ __global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
     if (threadIdx.x == 0) {
         tp[dv.ntiles] = k;
         dv.row_flags[row] = 0u;
+        dv.row_count[row] = 0u;
+        if (KIND == SEL_TOPK) dv.row_lo[row] = lower_bound_key(T, 3u);
         atomicAdd(&dv.stats->exact_rows, 1ull);
     }
 }
@@ -495,18 +451,19 @@ cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t
 }
 
 template <int KIND>
-static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, cudaStream_t st)
+static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
 {
-    emit_kernel<KIND><<<dv.n, kSelThreads, 0, st>>>(dv, a);
+    emit_kernel<KIND><<<dv.n, kSelThreads, 0, st>>>(dv, a, fused ? 1 : 0);
     if (a.vec) exact_kernel<KIND, true><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     else exact_kernel<KIND, false><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     *a.launches += 2;
     return cudaGetLastError();
 }
 
-cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, cudaStream_t st)
+cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
 {
-    return dv.kind == CHOCO_Q_TOPK ? emit_impl<SEL_TOPK>(dv, a, st) : emit_impl<SEL_RANDK>(dv, a, st);
+    return dv.kind == CHOCO_Q_TOPK ? emit_impl<SEL_TOPK>(dv, a, fused, st)
+                                   : emit_impl<SEL_RANDK>(dv, a, fused, st);
 }
 
 } // namespace choco

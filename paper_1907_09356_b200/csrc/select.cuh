@@ -1,0 +1,120 @@
+// Pieces shared by the selection kernels (top_a / random_a of the paper's Appendix C) and by
+// the update kernel, which collects the next step's candidates while it still holds
+// x - x^ in registers.
+#pragma once
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace choco {
+
+constexpr int kSelThreads = 1024;
+enum { SEL_TOPK = 0, SEL_RANDK = 1 };
+
+// Ordering key: larger key = kept first.  top_a: |v| without its sign bit, shifted up so that
+// all 32 bits carry order information (+0 and -0 tie).  random_a: complement of the Philox
+// word, so that the k smallest words win.
+template <int KIND>
+__device__ __forceinline__ uint32_t order_key(uint32_t bits)
+{
+    return KIND == SEL_TOPK ? (bits << 1) : ~bits;
+}
+
+// Exclusive prefix sum over the block (NT threads, NT a multiple of 32, at most 1024).
+// `sm` needs 33 words.  Returns the exclusive prefix; *total gets the block sum.
+template <int NT>
+__device__ __forceinline__ uint32_t block_scan_excl(uint32_t v, uint32_t* sm, uint32_t* total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads(); // protect sm from the previous use
+    if (lane == 31) sm[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < NT / 32 ? sm[lane] : 0u;
+        uint32_t winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        sm[lane] = winc - w;
+        if (lane == 31) sm[32] = winc;
+    }
+    __syncthreads();
+    *total = sm[32];
+    return sm[warp] + inc - v;
+}
+
+// Given hist[0..nbins) (shared memory) find the largest digit D with
+// sum_{b >= D} hist[b] >= need; *above = sum_{b > D} hist[b].  nbins <= 2 * NT.
+// All threads return the same values.  `sm` needs 36 words.
+template <int NT>
+__device__ __forceinline__ void block_find_digit(const uint32_t* hist, int nbins, uint32_t need,
+                                                 uint32_t* sm, uint32_t* digit, uint32_t* above)
+{
+    const int r0 = 2 * threadIdx.x, r1 = r0 + 1;
+    const uint32_t h0 = r0 < nbins ? hist[nbins - 1 - r0] : 0u;
+    const uint32_t h1 = r1 < nbins ? hist[nbins - 1 - r1] : 0u;
+    uint32_t total;
+    const uint32_t ex = block_scan_excl<NT>(h0 + h1, sm, &total);
+    if (threadIdx.x == 0) { sm[34] = 0u; sm[35] = 0u; }
+    __syncthreads();
+    if (ex < need && need <= ex + h0) {
+        sm[34] = (uint32_t)(nbins - 1 - r0);
+        sm[35] = ex;
+    } else if (ex + h0 < need && need <= ex + h0 + h1) {
+        sm[34] = (uint32_t)(nbins - 1 - r1);
+        sm[35] = ex + h0;
+    }
+    __syncthreads();
+    *digit = sm[34];
+    *above = sm[35];
+}
+
+// A 256-thread block holds, per thread and per iteration `it` < kIters, cnt[it] <= 4 chosen
+// coordinates of its tile; thread t's quad in iteration it covers coordinates
+// (it * 256 + t) * 4 ... + 3.  Computes the slot of each thread's first chosen coordinate in
+// ascending coordinate order (start[it]) and the number chosen in the whole tile.
+// `sm` needs 2 x 9 words; contains two block barriers.
+__device__ __forceinline__ void ordered_starts(const uint32_t cnt[kIters], uint32_t (*sm)[9],
+                                               uint32_t start[kIters], uint32_t* total)
+{
+    static_assert(kIters == 2 || kIters == 4, "two 16-bit fields per word");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t wa = cnt[0] | (cnt[1] << 16);
+    const uint32_t wb = kIters == 4 ? (cnt[kIters - 2] | (cnt[kIters - 1] << 16)) : 0u;
+    uint32_t ia = wa, ib = wb;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o);
+        const uint32_t tb = __shfl_up_sync(0xffffffffu, ib, o);
+        if (lane >= o) { ia += ta; ib += tb; }
+    }
+    __syncthreads(); // protect sm from the previous use
+    if (lane == 31) { sm[0][warp] = ia; sm[1][warp] = ib; }
+    __syncthreads();
+    uint32_t pa = 0, pb = 0, ta = 0, tb = 0; // exclusive over warps, totals
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+        const uint32_t xa = sm[0][w], xb = sm[1][w];
+        if (w < warp) { pa += xa; pb += xb; }
+        ta += xa; tb += xb;
+    }
+    const uint32_t ea = pa + ia - wa, eb = pb + ib - wb; // exclusive, per thread
+    const uint32_t t0 = ta & 0xFFFFu, t1 = ta >> 16, t2 = tb & 0xFFFFu, t3 = tb >> 16;
+    start[0] = ea & 0xFFFFu;
+    start[1] = t0 + (ea >> 16);
+    if (kIters == 4) {
+        start[kIters - 2] = t0 + t1 + (eb & 0xFFFFu);
+        start[kIters - 1] = t0 + t1 + t2 + (eb >> 16);
+    }
+    *total = t0 + t1 + t2 + t3;
+}
+
+} // namespace choco

@@ -97,6 +97,7 @@ def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed
             if momentum:
                 assert_state(_host(dM, d), M, f"M after step {t}")
         assert choco.choco_get_step(ch.ctx) == steps
+        assert choco.choco_get_stats(ch.ctx)["device_timeouts"] == 0
         if ld != d:   # the pad between rows is never written
             assert bool(torch.isnan(dX[:, d:]).all()) and bool(torch.isnan(dS[:, d:]).all())
         return ch, (dX, dXh, dS), (X, Xh, S)
@@ -161,6 +162,58 @@ def test_topk_ties_zeros_and_signed_zero():
     ch, _, _ = run_lockstep(workloads.ring(n), "topk", n, d, 4, k=k, x_init=x, seed=1)
     st = choco.choco_get_stats(ch.ctx)
     assert st["exact_rows"] > 0          # the tie-heavy rows went through the exact selection
+    ch.close()
+
+
+def test_topk_carry_across_steps():
+    """The update kernel prepares the next step's selection; results do not depend on it."""
+    w = workloads.torus(4, 4)
+    n, d, k, steps = 16, 40000, 400, 12
+    ch, (dX, dXh, dS), _ = run_lockstep(w, "topk", n, d, steps, k=k, seed=11, gamma=0.1, check_msgs=False)
+    st = choco.choco_get_stats(ch.ctx)
+    assert st["prepared_rows"] >= n * (steps - 3)          # all but the first step (and rare misses)
+    assert st["prepared_rows"] + st["recompressed_rows"] + st["exact_rows"] >= n * steps
+    ch.close()
+    # the same run with carrying switched off
+    X = workloads.normal_rows(n, d, 1.0, 1000 + 11)
+    ch2 = choco.Choco(w, d, "topk", k=k, seed=11)
+    choco.choco_set_carry(ch2.ctx, False)
+    eX, eXh, eS = _dev(X), torch.zeros(n, d, device=DEV), torch.zeros(n, d, device=DEV)
+    for t in range(steps):
+        G = _dev(workloads.normal_rows(n, d, 0.01, 5000 + 97 * 11 + t))
+        ch2.sgd_step(eX, eXh, eS, G, 0.1, 0.1)
+    torch.cuda.synchronize()
+    assert choco.choco_get_stats(ch2.ctx)["prepared_rows"] == 0
+    assert torch.equal(eX, dX) and torch.equal(eXh, dXh) and torch.equal(eS, dS)
+    ch2.close()
+
+
+def test_invalidate_after_external_change():
+    w = workloads.ring(4)
+    n, d, k = 4, 20000, 200
+    X = workloads.normal_rows(n, d, 1.0, 5)
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    G = workloads.normal_rows(n, d, 0.01, 6)
+    p = oracle.Params("topk", k=k)
+    ch = choco.Choco(w, d, "topk", k=k)
+    dX, dXh, dS, dG = _dev(X), _dev(Xh), _dev(S), _dev(G)
+    oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, 0)
+    ch.sgd_step(dX, dXh, dS, dG, 0.1, 0.2)
+    # the caller overwrites X in place (say, loads a checkpoint) and tells the library
+    X[:] = workloads.normal_rows(n, d, 4.0, 7)
+    dX.copy_(torch.from_numpy(X))
+    choco.choco_invalidate(ch.ctx)
+    oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, 1)
+    ch.sgd_step(dX, dXh, dS, dG, 0.1, 0.2)
+    torch.cuda.synchronize()
+    assert_state(_host(dX, d), X, "X after invalidate")
+    assert_state(_host(dXh, d), Xh, "Xhat after invalidate")
+    # a change of buffers is noticed without being told
+    dX2 = dX.clone()
+    oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, 2)
+    ch.sgd_step(dX2, dXh, dS, dG, 0.1, 0.2)
+    torch.cuda.synchronize()
+    assert_state(_host(dX2, d), X, "X after pointer change")
     ch.close()
 
 
