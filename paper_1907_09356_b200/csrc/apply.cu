@@ -258,6 +258,18 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     return false;
 }
 
+constexpr int kMaxNb = 64; // neighbours handled per batch
+constexpr int kMaxE = 2;   // message entries a thread holds per batch
+
+struct NbrTable {
+    uint32_t lo[kMaxNb];       // first entry of neighbour r's message inside this tile
+    uint32_t len[kMaxNb];      // number of such entries
+    uint32_t pref[kMaxNb + 1]; // exclusive prefix of len
+    int j[kMaxNb];             // the neighbour's row
+    float w[kMaxNb];           // w_ij
+    uint32_t self[2];          // this row's own range
+};
+
 template <bool HAS_G, bool HAS_M>
 __host__ __device__ constexpr int bulk_arrays() { return 3 + (HAS_G ? 1 : 0) + (HAS_M ? 1 : 0); }
 
@@ -266,7 +278,8 @@ constexpr size_t bulk_smem_bytes()
 {
     return (size_t)(bulk_arrays<HAS_G, HAS_M>() + 1) * kTile * sizeof(float) // tiles + acc
            + 2 * (kTile / 32) * sizeof(uint32_t)                              // touched, self
-           + 2 * 9 * sizeof(uint32_t) + 16;                                   // scan scratch, barrier, base
+           + 2 * 9 * sizeof(uint32_t) + 16                                    // scan scratch, barrier, base
+           + sizeof(NbrTable);
 }
 
 template <bool HAS_G, bool HAS_M, bool EMIT>
@@ -284,6 +297,7 @@ __global__ void __launch_bounds__(kThreads) update_sparse_bulk_kernel(Dev dv, St
     uint32_t(*scan)[9] = reinterpret_cast<uint32_t(*)[9]>(tself + kTile / 32);
     uint64_t* bar = reinterpret_cast<uint64_t*>(reinterpret_cast<uint32_t*>(scan) + 18);
     uint32_t* s_base = reinterpret_cast<uint32_t*>(bar + 1);
+    NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
 
     const int row = blockIdx.y;
     const int64_t tile = blockIdx.x;
@@ -313,22 +327,67 @@ __global__ void __launch_bounds__(kThreads) update_sparse_bulk_kernel(Dev dv, St
     __syncthreads();
 
     // neighbours in CSR order: acc += w * q_j on the coordinates j's message lists in this tile
-    uint32_t self_lo = 0, self_hi = 0;
-    for (int e = e0; e < e1; ++e) {
-        const int j = dv.col[e];
-        const float w = dv.wval[e];
-        const uint32_t* tp = dv.tile_ptr + (int64_t)j * (dv.ntiles + 1) + tile;
-        const uint32_t lo = __ldg(tp), hi = __ldg(tp + 1);
-        if (j == row) { self_lo = lo; self_hi = hi; }
-        const uint32_t* mi = dv.msg_idx + (int64_t)j * dv.kpitch;
-        const float* mv = dv.msg_val + (int64_t)j * dv.kpitch;
-        for (uint32_t p = lo + threadIdx.x; p < hi; p += kThreads) {
-            const uint32_t lc = __ldg(mi + p) - (uint32_t)c0;
-            acc[lc] = __fadd_rn(acc[lc], __fmul_rn(w, __ldg(mv + p)));
-            atomicOr(&touched[lc >> 5], 1u << (lc & 31));
+    // Up to kMaxNb neighbours at a time: first every neighbour's range in this tile (one
+    // round trip), then all their entries at once (a second one), then the additions,
+    // neighbour by neighbour, out of registers.
+    for (int eb = e0; eb < e1; eb += kMaxNb) {
+        const int nb = (e1 - eb) < kMaxNb ? (e1 - eb) : kMaxNb;
+        if (threadIdx.x < nb) {
+            const int j = dv.col[eb + threadIdx.x];
+            const uint32_t* tp = dv.tile_ptr + (int64_t)j * (dv.ntiles + 1) + tile;
+            const uint32_t lo = __ldg(tp), hi = __ldg(tp + 1);
+            nbr->lo[threadIdx.x] = lo;
+            nbr->len[threadIdx.x] = hi - lo;
+            nbr->j[threadIdx.x] = j;
+            nbr->w[threadIdx.x] = dv.wval[eb + threadIdx.x];
+            if (j == row) { nbr->self[0] = lo; nbr->self[1] = hi; }
         }
         __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (int r = 0; r < nb; ++r) { nbr->pref[r] = run; run += nbr->len[r]; }
+            nbr->pref[nb] = run;
+        }
+        __syncthreads();
+        const uint32_t total = nbr->pref[nb];
+        for (uint32_t f0 = 0; f0 < total; f0 += kThreads * kMaxE) {
+            int er[kMaxE];
+            uint32_t elc[kMaxE];
+            float ev[kMaxE];
+#pragma unroll
+            for (int q = 0; q < kMaxE; ++q) {
+                const uint32_t f = f0 + q * kThreads + threadIdx.x;
+                er[q] = -1;
+                if (f < total) {
+                    int r = 0;
+                    while (nbr->pref[r + 1] <= f) ++r;
+                    const uint32_t p = nbr->lo[r] + (f - nbr->pref[r]);
+                    const int64_t mrow = (int64_t)nbr->j[r] * dv.kpitch;
+                    er[q] = r;
+                    elc[q] = __ldg(dv.msg_idx + mrow + p) - (uint32_t)c0;
+                    ev[q] = __fmul_rn(nbr->w[r], __ldg(dv.msg_val + mrow + p));
+                }
+            }
+            // neighbours present in this batch of entries: [r_first, r_last]
+            int r_first = 0;
+            while (nbr->pref[r_first + 1] <= f0) ++r_first;
+            const uint32_t f_last = (f0 + kThreads * kMaxE < total ? f0 + kThreads * kMaxE : total) - 1;
+            int r_last = r_first;
+            while (nbr->pref[r_last + 1] <= f_last) ++r_last;
+            for (int r = r_first; r <= r_last; ++r) {
+                if (nbr->len[r] == 0) continue;
+#pragma unroll
+                for (int q = 0; q < kMaxE; ++q)
+                    if (er[q] == r) {
+                        acc[elc[q]] = __fadd_rn(acc[elc[q]], ev[q]);
+                        atomicOr(&touched[elc[q] >> 5], 1u << (elc[q] & 31));
+                    }
+                __syncthreads();
+            }
+        }
+        __syncthreads(); // the neighbour table is reused by the next batch
     }
+    const uint32_t self_lo = nbr->self[0], self_hi = nbr->self[1];
 
     // every thread polls (so that each sees the copied data); the verdict is made uniform
     const int arrived = __syncthreads_and(mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0);
