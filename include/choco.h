@@ -175,6 +175,30 @@ int choco_read_message(choco_ctx* ctx, int32_t worker, int32_t plane, void* host
  * X: DEVICE pointer.  Synchronises `stream`; *out is a HOST double. */
 int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* stream);
 
+/*
+ * choco_consensus_error_noalloc -- the same quantity as choco_consensus_error for callers
+ * that are not allowed to allocate device memory.  (The paper has no counterpart to this
+ * call; it exists for the sake of such callers only.)  Examples: code that runs while a
+ * memory pool or a capture session owns all allocation on the device, monitoring hooks
+ * inside a training loop whose allocator must not be disturbed, or a process that has
+ * handed its whole memory budget to someone else.  It needs no context: choco_init is
+ * itself an allocating call.
+ *   X        DEVICE pointer, float32 [n, ld], read-only; n >= 1, 1 <= d <= ld.
+ *   out_dev  DEVICE pointer to one double, caller-owned; receives sum_i ||x_i - xbar||^2
+ *            when the work enqueued on `stream` has finished (no host synchronisation).
+ * Limit: d <= 4 194 304.  The per-block partial sums (one double per 256 coordinates) are
+ * kept in a fixed 128 KiB array that is part of the library image on every GPU that loads
+ * it, for the life of the process; larger d returns CHOCO_ERR_TOO_LARGE and enqueues nothing.
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ * First use on a device looks up the address of that array (a one-time query, done with that
+ * device current); make this first call before starting any stream capture.
+ * All calls on a device share the array.  Each call overwrites every partial it later reads,
+ * so nothing carries over from one call to the next, but two calls whose kernels overlap on
+ * the GPU (different streams, no ordering between them) race on it: order them.
+ */
+int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t ld,
+                                  double* out_dev, void* stream);
+
 /* Counters since choco_init (HOST struct filled after synchronising `stream`). */
 typedef struct {
     uint64_t steps;            /* step calls enqueued                                         */

@@ -23,7 +23,7 @@ EXPORTS = [
     "choco_sgd_momentum_step", "choco_sgd_step_host", "choco_invalidate", "choco_set_carry",
     "choco_get_step",
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
-    "choco_consensus_error",
+    "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_read", "choco_strerror",
     "choco_last_cuda_error",
 ]
@@ -72,6 +72,7 @@ def load() -> ctypes.CDLL:
         lib.choco_get_message.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(i64)]
         lib.choco_read_message.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
         lib.choco_consensus_error.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), vp]
+        lib.choco_consensus_error_noalloc.argtypes = [vp, i32, i64, i64, vp, vp]
         lib.choco_get_stats.argtypes = [vp, ctypes.POINTER(choco_stats), vp]
         lib.choco_profile_enable.argtypes = [vp, i32]
         lib.choco_profile_read.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double), vp]
@@ -199,6 +200,13 @@ def choco_consensus_error(ctx, X, stream=None) -> float:
     out = ctypes.c_double()
     _check(load().choco_consensus_error(ctx, _ptr(X), ctypes.byref(out), _stream(stream)), ctx)
     return out.value
+
+
+def choco_consensus_error_noalloc(X, n: int, d: int, ld: int, out_dev, stream=None) -> None:
+    """Consensus distance into `out_dev` (a device tensor holding one float64) without any
+    allocation by the library: for callers that must not allocate device memory, e.g. while
+    a pool or a capture session owns allocation.  d is limited to 4 194 304; asynchronous."""
+    _check(load().choco_consensus_error_noalloc(_ptr(X), n, d, ld, _ptr(out_dev), _stream(stream)))
 
 
 def choco_get_stats(ctx, stream=None) -> dict:
