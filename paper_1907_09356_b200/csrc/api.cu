@@ -1,5 +1,6 @@
 // C entry points of libchoco: argument checks, allocation, and the order in which one step
 // enqueues its kernels.  No arithmetic of the method lives here.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -164,6 +165,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
     dv.ntiles = (d + kTile - 1) / kTile;
+    dv.nspans = (d + kSpan - 1) / kSpan;
     dv.nchunks = (d + kChunk - 1) / kChunk;
 
     cudaError_t e = cudaGetDevice(&ctx->device);
@@ -176,6 +178,28 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     if (e == cudaSuccess) e = cudaMemcpy(col, w_col, sizeof(int32_t) * nnz, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(wv, w_val, sizeof(float) * nnz, cudaMemcpyHostToDevice);
     dv.row_ptr = rp; dv.col = col; dv.wval = wv;
+    {
+        // for every CSR entry (j -> i): where j sits in row i, and the weight row i holds for it
+        std::vector<int32_t> pos(nnz);
+        std::vector<float> rw(nnz);
+        int32_t maxdeg = 0;
+        for (int32_t j = 0; j < n; ++j) {
+            maxdeg = std::max(maxdeg, w_row_ptr[j + 1] - w_row_ptr[j]);
+            for (int32_t e2 = w_row_ptr[j]; e2 < w_row_ptr[j + 1]; ++e2) {
+                const int32_t i = w_col[e2];
+                for (int32_t f = w_row_ptr[i]; f < w_row_ptr[i + 1]; ++f)
+                    if (w_col[f] == j) { pos[e2] = f - w_row_ptr[i]; rw[e2] = w_val[f]; break; }
+            }
+        }
+        dv.maxdeg = maxdeg;
+        int32_t* dpos = nullptr;
+        float* drw = nullptr;
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dpos, nnz);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &drw, nnz);
+        if (e == cudaSuccess) e = cudaMemcpy(dpos, pos.data(), sizeof(int32_t) * nnz, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(drw, rw.data(), sizeof(float) * nnz, cudaMemcpyHostToDevice);
+        dv.rd_pos = dpos; dv.rd_w = drw;
+    }
     if (e == cudaSuccess) e = dev_alloc(ctx, &dv.stats, 1);
 
     const int64_t nwords = (d + 31) / 32;
@@ -188,6 +212,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_idx, n * dv.kpitch);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_val, n * dv.kpitch);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_ptr, n * (dv.ntiles + 1));
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.rec, (int64_t)n * dv.ntiles * dv.maxdeg);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.hist, (int64_t)n * kHistBins);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_lo, n);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_count, n);

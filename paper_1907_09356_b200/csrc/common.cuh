@@ -14,9 +14,13 @@ namespace choco {
 
 constexpr int kThreads = 256;            // threads per block of the streaming kernels
 constexpr int kQuad = 4;                 // coordinates per thread per iteration (one 128-bit access)
-constexpr int kChunk = kThreads * kQuad; // 1024 coordinates: one block iteration, one tree leaf group
-constexpr int kIters = 2;                // iterations per block
-constexpr int kTile = kChunk * kIters;   // coordinates per block (2048)
+constexpr int kChunk = kThreads * kQuad; // 2048 coordinates: one block iteration, one tree leaf group
+constexpr int kDenseIters = 4;           // dense kernels: iterations per block
+constexpr int kSpan = kChunk * kDenseIters; // dense kernels: coordinates per block (4096)
+// sparse path (top-k, random-k): one block owns one tile of one row
+constexpr int kTileThreads = 128;
+constexpr int kTileIters = 4;            // quads per thread
+constexpr int kTile = kTileThreads * kQuad * kTileIters; // 2048 coordinates
 
 constexpr uint32_t kStreamRandK = 0;     // generator stream of the random-k selection keys
 constexpr uint32_t kStreamDither = 1;    // generator stream of the QSGD dither

@@ -37,12 +37,12 @@ __device__ __forceinline__ uint32_t sign_nibble(const float4& v)
 template <bool VEC, int MODE, bool PACK_SIGN>
 __global__ void __launch_bounds__(kThreads) norm_partial_kernel(Dev dv, StepArgs a)
 {
-    __shared__ float ws[kIters][8];
+    __shared__ float ws[kDenseIters][8];
     const int row = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t c0 = (int64_t)blockIdx.x * kTile;
+    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
+    for (int it = 0; it < kDenseIters; ++it) {
         const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
         const float4 v = diff_quad<VEC>(dv, a, row, c);
         float t;
@@ -57,8 +57,8 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(Dev dv, StepArgs
         }
     }
     __syncthreads();
-    if (threadIdx.x < kIters) {
-        const int64_t chunk = (int64_t)blockIdx.x * kIters + threadIdx.x;
+    if (threadIdx.x < kDenseIters) {
+        const int64_t chunk = (int64_t)blockIdx.x * kDenseIters + threadIdx.x;
         if (chunk < dv.nchunks) dv.partial[(int64_t)row * dv.nchunks + chunk] = tree8(ws[threadIdx.x]);
     }
 }
@@ -95,13 +95,13 @@ __global__ void __launch_bounds__(1024) norm_finish_kernel(Dev dv)
 template <bool VEC, int WBITS, int BUCKET>
 __global__ void __launch_bounds__(kThreads) qsgd_pack_kernel(Dev dv, StepArgs a)
 {
-    __shared__ float ws[kIters][8];
+    __shared__ float ws[kDenseIters][8];
     const int row = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t c0 = (int64_t)blockIdx.x * kTile;
-    float4 v[kIters];
+    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
+    float4 v[kDenseIters];
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
+    for (int it = 0; it < kDenseIters; ++it) {
         const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
         v[it] = diff_quad<VEC>(dv, a, row, c);
         if constexpr (BUCKET > 0) {
@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(kThreads) qsgd_pack_kernel(Dev dv, StepArgs a)
     if (BUCKET > 0) __syncthreads();
     const float sf = (float)dv.s;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
+    for (int it = 0; it < kDenseIters; ++it) {
         const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
         float nu;
         int64_t bucket = 0;
@@ -172,9 +172,9 @@ template <bool VEC>
 __global__ void __launch_bounds__(kThreads) identity_kernel(Dev dv, StepArgs a)
 {
     const int row = blockIdx.y;
-    const int64_t c0 = (int64_t)blockIdx.x * kTile;
+    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
+    for (int it = 0; it < kDenseIters; ++it) {
         const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
         if (c < dv.d) {
             const float4 v = diff_quad<VEC>(dv, a, row, c);
@@ -203,7 +203,7 @@ static void launch_qsgd_pack(const Dev& dv, const StepArgs& a, dim3 grid, cudaSt
 template <bool VEC>
 static cudaError_t compress_impl(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
+    const dim3 grid((unsigned)dv.nspans, (unsigned)dv.n);
     switch (dv.kind) {
     case CHOCO_Q_SIGN:
         norm_partial_kernel<VEC, NORM_L1, true><<<grid, kThreads, 0, st>>>(dv, a);

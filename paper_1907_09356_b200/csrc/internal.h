@@ -26,12 +26,20 @@ struct Dev {
     int32_t kind;
     int64_t d;
     int64_t ld;
-    int64_t ntiles;              // ceil(d / 4096)
+    int64_t ntiles;              // ceil(d / kTile): tiles of the sparse path
+    int64_t nspans;              // ceil(d / kSpan): blocks per row of the dense kernels
     int64_t nchunks;             // ceil(d / 1024)
     // W (CSR)
     const int32_t* row_ptr;
     const int32_t* col;
     const float* wval;
+    // reader-oriented view of the messages (sparse Q): for worker i, tile t and position r in
+    // i's CSR row, rec[(i * ntiles + t) * maxdeg + r] = {j, first entry of j's message in the
+    // tile, number of entries, bits of w_ij}; unused positions keep a zero count
+    int32_t maxdeg;              // longest CSR row (diagonal included)
+    const int32_t* rd_pos;       // [nnz] for entry (j, i): position of j in row i
+    const float* rd_w;           // [nnz] for entry (j, i): w_ij as row i stores it
+    uint4* rec;                  // [n, ntiles, maxdeg]
     // generator
     uint64_t seed;
     // sparse messages: idx / val [n, kpitch], tile_ptr [n, ntiles + 1]
@@ -95,6 +103,8 @@ cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cud
 cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st);
 // update kernel; emit: also collect the next step's top-k candidates (if apply_can_emit)
 bool apply_can_emit(const Dev& dv, const StepArgs& a);
+bool update_bulk_usable(const Dev& dv, const StepArgs& a);
+cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 // metrics
 cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,

@@ -47,9 +47,9 @@ __global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a)
     const int row = blockIdx.y;
     for (int b = threadIdx.x; b < kHistBins; b += kThreads) h[b] = 0u;
     __syncthreads();
-    const int64_t c0 = (int64_t)blockIdx.x * kTile;
+    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
+    for (int it = 0; it < kDenseIters; ++it) {
         const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
         if (c < dv.d) {
             uint32_t bits[4];
@@ -106,21 +106,21 @@ __global__ void randk_bound_kernel(Dev dv, uint32_t lo)
 // prepare 3: collect candidates, ascending inside each tile
 // ---------------------------------------------------------------------------------------
 template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
+__global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs a)
 {
-    __shared__ uint32_t sm[2][9];
+    __shared__ uint32_t sm[2][kTileThreads / 32 + 1];
     __shared__ uint32_t s_base;
     const int row = blockIdx.y;
     if (dv.row_flags[row] & kRowExact) return;
     const uint32_t lo = dv.row_lo[row];
     const int64_t c0 = (int64_t)blockIdx.x * kTile;
 
-    uint32_t bits[kIters][4];
+    uint32_t bits[kTileIters][4];
     uint32_t take = 0; // bit (4 it + e)
-    uint32_t cnt[kIters];
+    uint32_t cnt[kTileIters];
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
+    for (int it = 0; it < kTileIters; ++it) {
+        const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
         cnt[it] = 0;
         if (c < dv.d) {
             quad_bits<KIND, VEC>(dv, a, row, c, bits[it]);
@@ -132,8 +132,8 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
                 }
         }
     }
-    uint32_t start[kIters], total;
-    ordered_starts(cnt, sm, start, &total);
+    uint32_t start[kTileIters], total;
+    ordered_starts<kTileThreads, kTileIters>(cnt, sm, start, &total);
     if (threadIdx.x == 0) {
         const uint32_t base = total ? atomicAdd(&dv.row_count[row], total) : 0u;
         dv.seg_off[(int64_t)row * dv.ntiles + blockIdx.x] = base;
@@ -146,8 +146,8 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(Dev dv, StepArgs a)
     uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + s_base;
     uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + s_base;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
+    for (int it = 0; it < kTileIters; ++it) {
+        const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
         uint32_t p = start[it];
 #pragma unroll
         for (int e = 0; e < 4; ++e)
@@ -191,6 +191,23 @@ __device__ __forceinline__ void rank_key(const uint32_t* cv, uint32_t ncand, uin
     }
     *key_out = prefix;
     *above_out = above_total;
+}
+
+// Tell every reader of worker `row` where row's message enters each tile (tp[t] .. tp[t+1]),
+// in the reader's own CSR position, with the reader's own weight.  Called by all threads of
+// the block after tp[] is complete and visible.
+__device__ __forceinline__ void publish_ranges(const Dev& dv, int row, const uint32_t* tp)
+{
+    for (int e = dv.row_ptr[row]; e < dv.row_ptr[row + 1]; ++e) {
+        const int64_t reader = dv.col[e];
+        const int pos = dv.rd_pos[e];
+        const uint32_t wbits = __float_as_uint(dv.rd_w[e]);
+        uint4* rec = dv.rec + (reader * dv.ntiles) * dv.maxdeg + pos;
+        for (int64_t t = threadIdx.x; t < dv.ntiles; t += blockDim.x) {
+            const uint32_t lo = tp[t];
+            rec[t * dv.maxdeg] = make_uint4((uint32_t)row, lo, tp[t + 1] - lo, wbits);
+        }
+    }
 }
 
 // Lower a key bound by `eighths` eighths of an octave (about 8 % of the value each).
@@ -289,6 +306,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     }
     if (threadIdx.x == 0) tp[dv.ntiles] = k;
     __syncthreads();
+    publish_ranges(dv, row, tp);
     // ordered compaction, one warp per tile
     uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch;
     float* mv = dv.msg_val + (int64_t)row * dv.kpitch;
@@ -408,8 +426,10 @@ __global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
         run_gt += tot & 0xFFFFu;
         run_eq += tot >> 16;
     }
+    if (threadIdx.x == 0) tp[dv.ntiles] = k;
+    __syncthreads();
+    publish_ranges(dv, row, tp);
     if (threadIdx.x == 0) {
-        tp[dv.ntiles] = k;
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
         if (KIND == SEL_TOPK) dv.row_lo[row] = lower_bound_key(T, 3u);
@@ -426,8 +446,9 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
 {
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
     if (KIND == SEL_TOPK) {
-        if (a.vec) hist_kernel<true><<<grid, kThreads, 0, st>>>(dv, a);
-        else hist_kernel<false><<<grid, kThreads, 0, st>>>(dv, a);
+        const dim3 hgrid((unsigned)dv.nspans, (unsigned)dv.n);
+        if (a.vec) hist_kernel<true><<<hgrid, kThreads, 0, st>>>(dv, a);
+        else hist_kernel<false><<<hgrid, kThreads, 0, st>>>(dv, a);
         bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv);
         *a.launches += 2;
     } else {
@@ -438,8 +459,8 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
         randk_bound_kernel<<<(dv.n + 127) / 128, 128, 0, st>>>(dv, ~hi);
         *a.launches += 1;
     }
-    if (a.vec) collect_kernel<KIND, true><<<grid, kThreads, 0, st>>>(dv, a);
-    else collect_kernel<KIND, false><<<grid, kThreads, 0, st>>>(dv, a);
+    if (a.vec) collect_kernel<KIND, true><<<grid, kTileThreads, 0, st>>>(dv, a);
+    else collect_kernel<KIND, false><<<grid, kTileThreads, 0, st>>>(dv, a);
     *a.launches += 1;
     return cudaGetLastError();
 }

@@ -77,42 +77,57 @@ __device__ __forceinline__ void block_find_digit(const uint32_t* hist, int nbins
     *above = sm[35];
 }
 
-// A 256-thread block holds, per thread and per iteration `it` < kIters, cnt[it] <= 4 chosen
+// A block of NT threads holds, per thread and per iteration `it` < NIT, cnt[it] <= 4 chosen
 // coordinates of its tile; thread t's quad in iteration it covers coordinates
-// (it * 256 + t) * 4 ... + 3.  Computes the slot of each thread's first chosen coordinate in
+// (it * NT + t) * 4 ... + 3.  Computes the slot of each thread's first chosen coordinate in
 // ascending coordinate order (start[it]) and the number chosen in the whole tile.
-// `sm` needs 2 x 9 words; contains two block barriers.
-__device__ __forceinline__ void ordered_starts(const uint32_t cnt[kIters], uint32_t (*sm)[9],
-                                               uint32_t start[kIters], uint32_t* total)
+// NIT is 2 or 4 (16-bit fields: a tile holds fewer than 65536 coordinates).
+// `sm` needs 2 x (NT / 32 + 1) words; contains two block barriers.
+template <int NT, int NIT>
+__device__ __forceinline__ void ordered_starts(const uint32_t cnt[NIT], uint32_t (*sm)[NT / 32 + 1],
+                                               uint32_t start[NIT], uint32_t* total)
 {
-    static_assert(kIters == 2 || kIters == 4, "two 16-bit fields per word");
+    static_assert(NIT == 2 || NIT == 4, "two 16-bit fields per word");
+    static_assert(NT * NIT * 4 < 65536, "per-iteration totals must fit 16 bits");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t wa = cnt[0] | (cnt[1] << 16);
-    const uint32_t wb = kIters == 4 ? (cnt[kIters - 2] | (cnt[kIters - 1] << 16)) : 0u;
+    uint32_t wb = 0u;
+    if constexpr (NIT == 4) wb = cnt[2] | (cnt[3] << 16);
     uint32_t ia = wa, ib = wb;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o);
-        const uint32_t tb = __shfl_up_sync(0xffffffffu, ib, o);
-        if (lane >= o) { ia += ta; ib += tb; }
+        if (lane >= o) ia += ta;
+        if constexpr (NIT == 4) {
+            const uint32_t tb = __shfl_up_sync(0xffffffffu, ib, o);
+            if (lane >= o) ib += tb;
+        }
     }
     __syncthreads(); // protect sm from the previous use
-    if (lane == 31) { sm[0][warp] = ia; sm[1][warp] = ib; }
+    if (lane == 31) {
+        sm[0][warp] = ia;
+        if constexpr (NIT == 4) sm[1][warp] = ib;
+    }
     __syncthreads();
     uint32_t pa = 0, pb = 0, ta = 0, tb = 0; // exclusive over warps, totals
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) {
-        const uint32_t xa = sm[0][w], xb = sm[1][w];
-        if (w < warp) { pa += xa; pb += xb; }
-        ta += xa; tb += xb;
+    for (int w = 0; w < NT / 32; ++w) {
+        const uint32_t xa = sm[0][w];
+        if (w < warp) pa += xa;
+        ta += xa;
+        if constexpr (NIT == 4) {
+            const uint32_t xb = sm[1][w];
+            if (w < warp) pb += xb;
+            tb += xb;
+        }
     }
     const uint32_t ea = pa + ia - wa, eb = pb + ib - wb; // exclusive, per thread
     const uint32_t t0 = ta & 0xFFFFu, t1 = ta >> 16, t2 = tb & 0xFFFFu, t3 = tb >> 16;
     start[0] = ea & 0xFFFFu;
     start[1] = t0 + (ea >> 16);
-    if (kIters == 4) {
-        start[kIters - 2] = t0 + t1 + (eb & 0xFFFFu);
-        start[kIters - 1] = t0 + t1 + t2 + (eb >> 16);
+    if constexpr (NIT == 4) {
+        start[2] = t0 + t1 + (eb & 0xFFFFu);
+        start[3] = t0 + t1 + t2 + (eb >> 16);
     }
     *total = t0 + t1 + t2 + t3;
 }
