@@ -18,8 +18,8 @@ constexpr int kChunk = kThreads * kQuad; // 2048 coordinates: one block iteratio
 constexpr int kDenseIters = 4;           // dense kernels: iterations per block
 constexpr int kSpan = kChunk * kDenseIters; // dense kernels: coordinates per block (4096)
 // sparse path (top-k, random-k): one block owns one tile of one row
-constexpr int kTileThreads = 128;
-constexpr int kTileIters = 4;            // quads per thread
+constexpr int kTileThreads = 256;
+constexpr int kTileIters = 2;            // quads per thread
 constexpr int kTile = kTileThreads * kQuad * kTileIters; // 2048 coordinates
 
 constexpr uint32_t kStreamRandK = 0;     // generator stream of the random-k selection keys

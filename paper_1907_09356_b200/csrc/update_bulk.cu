@@ -5,9 +5,10 @@
 //
 // Requirements: rows 16-byte aligned, d a multiple of 4.  The x, x^, s, g (and momentum)
 // tiles are fetched into shared memory by asynchronous bulk copies that complete on an
-// mbarrier, so no registers are tied up while they are in flight; warp 0 meanwhile gathers the
-// neighbours' message entries that fall into the tile and is the only one that polls the
-// barrier.  With EMIT the kernel also collects the candidates of the next step's top-k
+// mbarrier, so no registers are tied up while they are in flight.  Meanwhile the block reads
+// the range records of its neighbours (one round trip), then all their entries that fall
+// into the tile (a second one), and adds them into a shared accumulator tile neighbour by
+// neighbour.  With EMIT the kernel also collects the candidates of the next step's top-k
 // selection from x' - x^', which it holds anyway.
 #include "select.cuh"
 
@@ -81,25 +82,38 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     return false;
 }
 
-constexpr int kPrefetch = 6; // neighbours whose first 32 entries are fetched together
+constexpr int NT = kTileThreads;
+constexpr int NIT = kTileIters;
+constexpr int kMaxNb = 32; // neighbours handled per batch (one lane each)
+constexpr int kMaxE = 2;   // message entries a thread holds per pass
+
+struct NbrTable {
+    uint32_t lo[kMaxNb];       // first entry of neighbour r's message inside this tile
+    uint32_t len[kMaxNb];      // number of such entries
+    uint32_t pref[kMaxNb + 1]; // exclusive prefix of len
+    uint32_t j[kMaxNb];        // the neighbour's row
+    float w[kMaxNb];           // w_ij
+    uint32_t self;             // position of this worker in the batch, or kMaxNb
+    uint32_t pad;
+};
 
 template <bool HAS_G, bool HAS_M>
 __host__ __device__ constexpr int bulk_arrays() { return 3 + (HAS_G ? 1 : 0) + (HAS_M ? 1 : 0); }
 
-template <int NT, bool HAS_G, bool HAS_M>
+template <bool HAS_G, bool HAS_M>
 constexpr size_t bulk_smem_bytes()
 {
     return (size_t)(bulk_arrays<HAS_G, HAS_M>() + 1) * kTile * sizeof(float) // tiles + acc
            + 2 * (kTile / 32) * sizeof(uint32_t)                              // touched, self
            + 8                                                                // barrier
-           + 2 * (NT / 32 + 1) * sizeof(uint32_t) + 8;                        // scan scratch, base
+           + 2 * (NT / 32 + 1) * sizeof(uint32_t) + 8                         // scan scratch, base
+           + sizeof(NbrTable);
 }
 
-template <int NT, bool HAS_G, bool HAS_M, bool EMIT>
+template <bool HAS_G, bool HAS_M, bool EMIT>
 __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepArgs a)
 {
-    constexpr int NIT = kTile / (NT * kQuad); // quads per thread
-    static_assert(NT >= kTile / 32, "one thread per mask word");
+    static_assert(NT >= kTile / 32 && NT >= kMaxNb, "one thread per mask word / neighbour");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* hs = xs + kTile;
@@ -112,18 +126,18 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     uint64_t* bar = reinterpret_cast<uint64_t*>(tself + kTile / 32);
     uint32_t(*scan)[NT / 32 + 1] = reinterpret_cast<uint32_t(*)[NT / 32 + 1]>(bar + 1);
     uint32_t* s_base = reinterpret_cast<uint32_t*>(scan) + 2 * (NT / 32 + 1);
+    NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
 
     const int row = blockIdx.y;
     const int64_t tile = blockIdx.x;
     const int64_t c0 = tile * kTile;
     const int nvalid = (int)((dv.d - c0) < kTile ? (dv.d - c0) : kTile); // multiple of 4
+    const int lane = threadIdx.x & 31;
     float* xr = a.X + (int64_t)row * dv.ld + c0;
     float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
     float* sr = a.S + (int64_t)row * dv.ld + c0;
+    const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
 
-    // Thread 0 starts the tile copies; warp 0 looks up where each neighbour's message enters
-    // this tile (lane r holds neighbour r of the current batch of 32) while all threads clear
-    // the accumulator tile.
     if (threadIdx.x == 0) {
         mbar_init(bar, 1);
         const uint32_t bytes = (uint32_t)nvalid * sizeof(float);
@@ -134,100 +148,114 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
         if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, bytes, bar);
         if (HAS_M) bulk_load(ms, a.M + (int64_t)row * dv.ld + c0, bytes, bar);
     }
-    const int lane = threadIdx.x & 31;
-    const uint32_t lo_key = EMIT ? __ldg(dv.row_lo + row) : 0u; // needed only at the end: fetch early
-    // lane r of warp 0: where neighbour r's message enters this tile (one 16-byte record)
-    const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
-    int nj = 0;
-    float nw = 0.f;
-    uint32_t nlo = 0, nlen = 0;
-    if (threadIdx.x < 32 && lane < dv.maxdeg) {
-        const uint4 rc = __ldg(recs + lane);
-        nj = (int)rc.x; nlo = rc.y; nlen = rc.z; nw = __uint_as_float(rc.w);
-    }
+    const uint32_t lo_key = EMIT ? __ldg(dv.row_lo + row) : 0u; // used at the end: fetch early
+    // warp 1 builds the neighbour table of the first batch while the others clear the tile
+    uint4 rc = make_uint4(0u, 0u, 0u, 0u);
+    if ((threadIdx.x >> 5) == 1 && lane < dv.maxdeg) rc = __ldg(recs + lane);
 #pragma unroll
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (threadIdx.x < kTile / 32) { touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; }
-    __syncthreads();
 
-    // Warp 0 alone adds the neighbours' entries, in CSR order; program order inside the warp
-    // (plus __syncwarp between neighbours) is what orders two neighbours that hit the same
-    // coordinate.  The first 32 entries of up to kPrefetch neighbours are fetched together.
-    int ok = 1;
-    if (threadIdx.x < 32) {
-        uint32_t self_lo = 0, self_len = 0, self_idx = 0; // own entries: first 32 kept in registers
-        float self_val = 0.f;
-        for (int eb = 0; eb < dv.maxdeg; eb += 32) {
+    bool self_in_regs = false;  // this worker's own entries are held by threads (er == self)
+    uint32_t self_lo = 0, self_len = 0;
+    int er[kMaxE];
+    uint32_t elc[kMaxE];
+    float ev[kMaxE];
+#pragma unroll
+    for (int q = 0; q < kMaxE; ++q) er[q] = -1;
+
+    for (int eb = 0; eb < dv.maxdeg; eb += kMaxNb) {
+        const int nb = (dv.maxdeg - eb) < kMaxNb ? (dv.maxdeg - eb) : kMaxNb;
+        if ((threadIdx.x >> 5) == 1) {
             if (eb != 0) {
-                nlen = 0;
-                if (eb + lane < dv.maxdeg) {
-                    const uint4 rc = __ldg(recs + eb + lane);
-                    nj = (int)rc.x; nlo = rc.y; nlen = rc.z; nw = __uint_as_float(rc.w);
-                }
+                rc = make_uint4(0u, 0u, 0u, 0u);
+                if (lane < nb) rc = __ldg(recs + eb + lane);
             }
-            const int nb = (dv.maxdeg - eb) < 32 ? (dv.maxdeg - eb) : 32;
-            for (int rc = 0; rc < nb; rc += kPrefetch) {
-                uint32_t pidx[kPrefetch];
-                float pval[kPrefetch];
+            // inclusive prefix of the lengths over the lanes
+            uint32_t inc = rc.z;
 #pragma unroll
-                for (int q = 0; q < kPrefetch; ++q) {
-                    const int r = (rc + q) & 31;
-                    const int jr = __shfl_sync(0xffffffffu, nj, r);
-                    const uint32_t lor = __shfl_sync(0xffffffffu, nlo, r);
-                    const uint32_t lenr = __shfl_sync(0xffffffffu, nlen, r);
-                    pidx[q] = 0u;
-                    pval[q] = 0.f;
-                    if (rc + q < nb && (uint32_t)lane < lenr) {
-                        pidx[q] = __ldg(dv.msg_idx + (int64_t)jr * dv.kpitch + lor + lane);
-                        pval[q] = __ldg(dv.msg_val + (int64_t)jr * dv.kpitch + lor + lane);
-                    }
-                }
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += t;
+            }
+            nbr->lo[lane] = rc.y;
+            nbr->len[lane] = rc.z;
+            nbr->j[lane] = rc.x;
+            nbr->w[lane] = __uint_as_float(rc.w);
+            nbr->pref[lane + 1] = inc;
+            if (lane == 0) { nbr->pref[0] = 0u; nbr->self = kMaxNb; }
+            __syncwarp();
+            if (lane < nb && (int)rc.x == row && rc.z != 0u) nbr->self = (uint32_t)lane;
+        }
+        __syncthreads();
+        const uint32_t total = nbr->pref[nb];
+        const uint32_t selfr = nbr->self;
+        if (selfr < (uint32_t)nb) { self_lo = nbr->lo[selfr]; self_len = nbr->len[selfr]; }
+        for (uint32_t f0 = 0; f0 < total; f0 += NT * kMaxE) {
 #pragma unroll
-                for (int q = 0; q < kPrefetch; ++q) {
-                    if (rc + q >= nb) break;
-                    const int r = rc + q;
-                    const int jr = __shfl_sync(0xffffffffu, nj, r);
-                    const float wr = __shfl_sync(0xffffffffu, nw, r);
-                    const uint32_t lor = __shfl_sync(0xffffffffu, nlo, r);
-                    const uint32_t lenr = __shfl_sync(0xffffffffu, nlen, r);
-                    if (jr == row && lenr) { self_lo = lor; self_len = lenr; self_idx = pidx[q]; self_val = pval[q]; }
-                    if ((uint32_t)lane < lenr) {
-                        const uint32_t lc = pidx[q] - (uint32_t)c0;
-                        acc[lc] = __fadd_rn(acc[lc], __fmul_rn(wr, pval[q]));
-                        atomicOr(&touched[lc >> 5], 1u << (lc & 31));
-                    }
-                    for (uint32_t p = 32 + lane; p < lenr; p += 32) { // beyond the prefetched 32
-                        const uint32_t lc = __ldg(dv.msg_idx + (int64_t)jr * dv.kpitch + lor + p) - (uint32_t)c0;
-                        const float val = __ldg(dv.msg_val + (int64_t)jr * dv.kpitch + lor + p);
-                        acc[lc] = __fadd_rn(acc[lc], __fmul_rn(wr, val));
-                        atomicOr(&touched[lc >> 5], 1u << (lc & 31));
-                    }
-                    __syncwarp();
+            for (int q = 0; q < kMaxE; ++q) {
+                const uint32_t f = f0 + q * NT + threadIdx.x;
+                er[q] = -1;
+                if (f < total) {
+                    int r = 0;
+                    while (nbr->pref[r + 1] <= f) ++r;
+                    const uint32_t p = nbr->lo[r] + (f - nbr->pref[r]);
+                    const int64_t mrow = (int64_t)nbr->j[r] * dv.kpitch;
+                    er[q] = r;
+                    elc[q] = __ldg(dv.msg_idx + mrow + p) - (uint32_t)c0;
+                    ev[q] = __ldg(dv.msg_val + mrow + p);
                 }
             }
-        }
-        // wait (bounded) for the tiles, then x^ += q_i in place on the staged tile
-        ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
-        if (ok) {
-            if ((uint32_t)lane < self_len) {
-                const uint32_t lc = self_idx - (uint32_t)c0;
-                hs[lc] = __fadd_rn(hs[lc], self_val);
-                atomicOr(&tself[lc >> 5], 1u << (lc & 31));
+            // neighbours present in this pass: [r_first, r_last]; one round per neighbour
+            int r_first = 0;
+            while (nbr->pref[r_first + 1] <= f0) ++r_first;
+            const uint32_t f_last = (f0 + NT * kMaxE < total ? f0 + NT * kMaxE : total) - 1;
+            int r_last = r_first;
+            while (nbr->pref[r_last + 1] <= f_last) ++r_last;
+            for (int r = r_first; r <= r_last; ++r) {
+                if (nbr->len[r] == 0) continue;
+                const float wr = nbr->w[r];
+#pragma unroll
+                for (int q = 0; q < kMaxE; ++q)
+                    if (er[q] == r) {
+                        acc[elc[q]] = __fadd_rn(acc[elc[q]], __fmul_rn(wr, ev[q]));
+                        atomicOr(&touched[elc[q] >> 5], 1u << (elc[q] & 31));
+                    }
+                __syncthreads();
             }
-            const uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch + self_lo;
-            const float* mv = dv.msg_val + (int64_t)row * dv.kpitch + self_lo;
-            for (uint32_t p = 32 + lane; p < self_len; p += 32) { // beyond the 32 kept in registers
-                const uint32_t lc = __ldg(mi + p) - (uint32_t)c0;
-                hs[lc] = __fadd_rn(hs[lc], __ldg(mv + p));
-                atomicOr(&tself[lc >> 5], 1u << (lc & 31));
-            }
+            // a single pass over a single batch keeps this worker's own entries in registers
+            self_in_regs = (f0 == 0 && total <= NT * kMaxE && dv.maxdeg <= kMaxNb);
         }
+        if (eb + kMaxNb < dv.maxdeg) __syncthreads(); // the table is rebuilt for the next batch
     }
-    // the other warps wait here without polling; afterwards each thread observes the
-    // completed barrier phase itself so that the copied tiles are visible to it
+
+    // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
+    // completed phase itself so that the copied tiles are visible to it
+    int ok = 1;
+    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
     if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
     if (!mbar_wait_bounded(bar, 0, dv.stats)) return;
+
+    // x^ += q_i in place on the staged tile
+    if (self_in_regs) {
+        const int selfr = (int)nbr->self;
+#pragma unroll
+        for (int q = 0; q < kMaxE; ++q)
+            if (er[q] == selfr) {
+                hs[elc[q]] = __fadd_rn(hs[elc[q]], ev[q]);
+                atomicOr(&tself[elc[q] >> 5], 1u << (elc[q] & 31));
+            }
+    } else {
+        const uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch + self_lo;
+        const float* mv = dv.msg_val + (int64_t)row * dv.kpitch + self_lo;
+        for (uint32_t p = threadIdx.x; p < self_len; p += NT) {
+            const uint32_t lc = __ldg(mi + p) - (uint32_t)c0;
+            hs[lc] = __fadd_rn(hs[lc], __ldg(mv + p));
+            atomicOr(&tself[lc >> 5], 1u << (lc & 31));
+        }
+    }
+    __syncthreads();
 
     const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
     uint32_t take = 0, cnt[NIT];
@@ -312,7 +340,7 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
 template <bool HAS_G, bool HAS_M, bool EMIT>
 cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    constexpr size_t smem = bulk_smem_bytes<kTileThreads, HAS_G, HAS_M>();
+    constexpr size_t smem = bulk_smem_bytes<HAS_G, HAS_M>();
     // Once per device and instantiation: allow the dynamic shared memory size and ask for the
     // largest shared-memory carve-out, so that as many tiles as possible are in flight per SM.
     static bool configured[64] = {};
@@ -320,7 +348,7 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        auto kern = update_sparse_bulk_kernel<kTileThreads, HAS_G, HAS_M, EMIT>;
+        auto kern = update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -329,7 +357,7 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
-    update_sparse_bulk_kernel<kTileThreads, HAS_G, HAS_M, EMIT><<<grid, kTileThreads, smem, st>>>(dv, a);
+    update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT><<<grid, NT, smem, st>>>(dv, a);
     return cudaSuccess;
 }
 
