@@ -223,6 +223,21 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.seg_cnt, n * dv.ntiles);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_a, n * dv.ntiles);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_b, n * dv.ntiles);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_c, n * dv.ntiles);
+        {
+            // the emit kernel keeps in shared memory, in this order of preference and as far
+            // as the budget allows: slab prefixes, per-tile arrays, a cache of the keys
+            dv.slab_pitch = dv.cap / 32 + 2;
+            int64_t left = kEmitSmemBudget;
+            dv.emit_slabs_smem = 2 * dv.slab_pitch * 4 <= left ? 1 : 0;
+            if (dv.emit_slabs_smem) left -= 2 * dv.slab_pitch * 4;
+            dv.emit_tiles_smem = 3 * dv.ntiles * 4 <= left ? 1 : 0;
+            if (dv.emit_tiles_smem) left -= 3 * dv.ntiles * 4;
+            dv.emit_keys_cap = std::min<int64_t>(dv.cap, left / 4);
+            dv.emit_smem_bytes = kEmitSmemBudget - left + dv.emit_keys_cap * 4;
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);
+        }
         ctx->msg_bytes_per_worker = (p->kind == CHOCO_Q_TOPK ? 8 : 4) * p->k;
     } else if (p->kind == CHOCO_Q_SIGN) {
         dv.wpitch = round_up(nwords, 4);

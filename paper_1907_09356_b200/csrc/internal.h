@@ -11,6 +11,7 @@ namespace choco {
 // Row flags of the selection pipeline (top-k, random-k).
 constexpr uint32_t kRowExact = 1u;    // candidates unusable: run the exact one-block selection
 
+constexpr int64_t kEmitSmemBudget = 200 * 1024; // dynamic shared memory the emit kernel may use
 constexpr int kHistBins = 2048;       // first radix digit: top 11 bits of the ordering key
 
 struct Stats {
@@ -60,6 +61,15 @@ struct Dev {
     uint32_t* seg_cnt;           // [n, ntiles]
     uint32_t* tile_a;            // [n, ntiles] scratch
     uint32_t* tile_b;            // [n, ntiles] scratch
+    uint32_t* tile_c;            // [n, ntiles] scratch
+    // emit kernel: where its working arrays live (shared memory as far as it fits)
+    int64_t slab_pitch;          // cap / 32 + 2: slabs of 32 candidates per row
+    uint32_t* slab_a;            // [n, slab_pitch] scratch (used when not in shared memory)
+    uint32_t* slab_b;            // [n, slab_pitch]
+    int32_t emit_slabs_smem;     // slab arrays in shared memory
+    int32_t emit_tiles_smem;     // per-tile arrays in shared memory
+    int64_t emit_keys_cap;       // candidate keys cached in shared memory up to this many
+    int64_t emit_smem_bytes;     // dynamic shared memory of the emit kernel
     Stats* stats;
     // dense messages
     int64_t wpitch;              // sign-plane words per row (multiple of 4)

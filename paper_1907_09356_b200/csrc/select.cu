@@ -77,8 +77,8 @@ __global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv)
         g[b] = 0u; // ready for the next use
     }
     __syncthreads();
-    // keep down to rank 3.5 k (not just k) so that emit can place the next step's bound
-    const uint64_t want = 3 * (uint64_t)dv.k + (uint64_t)dv.k / 2;
+    // keep down to rank 2.5 k (not just k) so that emit can place the next step's bound
+    const uint64_t want = 2 * (uint64_t)dv.k + (uint64_t)dv.k / 2;
     const uint32_t need = (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d);
     uint32_t digit, above;
     block_find_digit<kSelThreads>(h, kHistBins, need, sm, &digit, &above);
@@ -163,33 +163,57 @@ __global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs 
 // emit: exact selection among the candidates of a row, ordered output
 // ---------------------------------------------------------------------------------------
 
-// Radix refinement over the candidate values cv[0..ncand): the key of rank `rank`
-// (1 = largest) and how many candidates are strictly above it.
-template <int KIND>
-__device__ __forceinline__ void rank_key(const uint32_t* cv, uint32_t ncand, uint32_t rank,
-                                         uint32_t* h, uint32_t* sm, uint32_t* key_out,
-                                         uint32_t* above_out)
+// The key of rank `rank` (1 = largest) among key(0..ncand) and how many keys are strictly
+// above it.  `key` is any callable p -> uint32_t.  Histogram refinement over the range the
+// keys actually span: candidates share their leading bits, so a fixed radix digit would pile
+// them into a handful of bins (and serialise the shared-memory atomics); bins spread over
+// [min, max] instead, then over the chosen bin, until a bin is one key wide.
+template <typename KeyFn>
+__device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t rank, uint32_t* h,
+                                         uint32_t* sm, uint32_t* key_out, uint32_t* above_out)
 {
-    uint32_t prefix = 0, pmask = 0, need = rank, above_total = 0;
-    const int shifts[3] = {21, 10, 0};
-    const int nbins[3] = {2048, 2048, 1024};
-    for (int pass = 0; pass < 3; ++pass) {
+    // range of the keys
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+    for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+        const uint32_t kk = key(p);
+        lo = kk < lo ? kk : lo;
+        hi = kk > hi ? kk : hi;
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    __syncthreads(); // protect sm from the previous use
+    if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = lo; h[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    for (int w = 0; w < kSelThreads / 32; ++w) {
+        lo = sm[w] < lo ? sm[w] : lo;
+        hi = h[w] > hi ? h[w] : hi;
+    }
+    __syncthreads();
+    uint32_t need = rank, above_total = 0;
+    for (;;) {
+        const uint32_t width = hi - lo;
+        const int shift = width < (uint32_t)kHistBins ? 0 : (32 - __clz(width)) - 11;
+        const int nbins = (int)(width >> shift) + 1; // <= kHistBins
         for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
         __syncthreads();
         for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
-            const uint32_t key = order_key<KIND>(cv[p]);
-            if ((key & pmask) == prefix) atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
+            const uint32_t kk = key(p);
+            if (kk >= lo && kk <= hi) atomicAdd(&h[(kk - lo) >> shift], 1u);
         }
         __syncthreads();
         uint32_t digit, above;
-        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
+        block_find_digit<kSelThreads>(h, nbins, need, sm, &digit, &above);
         need -= above;
         above_total += above;
-        prefix |= digit << shifts[pass];
-        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
+        const uint32_t nlo = lo + (digit << shift);
+        const uint32_t span = shift ? ((1u << shift) - 1u) : 0u;
+        const uint32_t nhi = (hi - nlo) < span ? hi : nlo + span;
+        lo = nlo;
+        hi = nhi;
         __syncthreads();
+        if (shift == 0) break;
     }
-    *key_out = prefix;
+    *key_out = lo;
     *above_out = above_total;
 }
 
@@ -217,24 +241,64 @@ __device__ __forceinline__ uint32_t lower_bound_key(uint32_t key, uint32_t eight
     return key > dec ? key - dec : 0u;
 }
 
-// Rank aimed at by the candidate bound: 3.5 k (the k chosen leave, about 2.5 k stay)
-__host__ __device__ __forceinline__ uint64_t target_rank(uint64_t k) { return 3 * k + k / 2; }
+// Rank aimed at by the candidate bound: 2.5 k (the k chosen leave, about 1.5 k stay)
+__host__ __device__ __forceinline__ uint64_t target_rank(uint64_t k) { return 2 * k + k / 2; }
 
 // lo: bound the ncand candidates were collected with (their rank-ncand key, roughly);
-// T: key of rank k.  Linear in the key between the two ranks, at most half an octave down.
+// T: key of rank k.  The key is read off a line in (log rank, key) through the two points
+// (tails fall off roughly like that; a line in the rank itself sits above a convex tail and
+// would keep too few), at most half an octave below the old bound.
 __device__ __forceinline__ uint32_t next_bound(uint32_t lo, uint32_t T, uint32_t ncand, uint32_t k)
 {
     if (ncand <= k || T < lo) return lower_bound_key(lo, 4u);
-    const uint64_t span = T - lo, want = target_rank(k), den = ncand - k;
-    if (ncand >= want) return lo + (uint32_t)((ncand - want) * span / den);
-    uint64_t dec = (want - ncand) * span / den;
-    if (dec > (4ull << 21)) dec = 4ull << 21;
-    return lo > dec ? (uint32_t)(lo - dec) : 0u;
+    const float span = (float)(T - lo);
+    const float want = (float)target_rank(k);
+    const float frac = __log2f(want / (float)k) / __log2f((float)ncand / (float)k); // 1 at rank ncand
+    const float drop = span * frac;                                                // below T
+    if (drop <= span) return T - (uint32_t)drop;
+    float dec = drop - span;
+    if (dec > (float)(4u << 21)) dec = (float)(4u << 21);
+    return lo > (uint32_t)dec ? lo - (uint32_t)dec : 0u;
 }
 
+// Exclusive prefix sums, in place, of two arrays of length n (one block, kSelThreads threads).
+// `carry` is two words of shared memory; totals are returned through tot_a / tot_b.
+__device__ __forceinline__ void block_scan_pair(uint32_t* a, uint32_t* b, int64_t n, uint32_t* sm,
+                                                uint32_t* carry, uint32_t* tot_a, uint32_t* tot_b)
+{
+    if (threadIdx.x == 0) { carry[0] = 0u; carry[1] = 0u; }
+    __syncthreads();
+    for (int64_t i0 = 0; i0 < n; i0 += kSelThreads) {
+        const int64_t i = i0 + threadIdx.x;
+        const uint32_t va = i < n ? a[i] : 0u, vb = i < n ? b[i] : 0u;
+        uint32_t ta, tb;
+        const uint32_t ea = block_scan_excl<kSelThreads>(va, sm, &ta);
+        const uint32_t eb = block_scan_excl<kSelThreads>(vb, sm, &tb);
+        const uint32_t ca = carry[0], cb = carry[1];
+        if (i < n) { a[i] = ca + ea; b[i] = cb + eb; }
+        __syncthreads();
+        if (threadIdx.x == 0) { carry[0] = ca + ta; carry[1] = cb + tb; }
+        __syncthreads();
+    }
+    *tot_a = carry[0];
+    *tot_b = carry[1];
+}
+
+// Layout of the emit kernel's dynamic shared memory, fixed at choco_init from the sizes:
+// slab prefix arrays, per-tile arrays and a cache of the candidate keys go to shared memory
+// as far as they fit (in that order); what does not fit lives in global scratch.
+//
+// One block per row.  All passes over the candidates are flat (candidate p = slab * 32 + lane)
+// so that their loads are independent of each other:
+//   1. keys into shared memory, k-th key T by radix refinement, next bound;
+//   2. per tile: number of keys above T and equal to T (atomics); per 32-candidate slab too;
+//   3. prefix over tiles -> tile_ptr and the number of equal keys before each tile; prefix
+//      over slabs; per tile the two prefixes at its first candidate;
+//   4. every chosen candidate computes its own output position and writes itself.
 template <int KIND>
 __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused)
 {
+    extern __shared__ uint32_t dyn[];
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t sm[36];
     __shared__ uint32_t s_carry[2];
@@ -253,88 +317,131 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     }
     const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
     const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
+    const int64_t nslab = ((int64_t)ncand + 31) >> 5;
+
+    // carve the dynamic shared memory
+    uint32_t* cursor = dyn;
+    uint32_t *slab_g, *slab_e, *t_gt, *t_eq, *t_sbe;
+    if (dv.emit_slabs_smem) { slab_g = cursor; slab_e = cursor + dv.slab_pitch; cursor += 2 * dv.slab_pitch; }
+    else { slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch; }
+    if (dv.emit_tiles_smem) { t_gt = cursor; t_eq = cursor + dv.ntiles; t_sbe = cursor + 2 * dv.ntiles; cursor += 3 * dv.ntiles; }
+    else { t_gt = dv.tile_a + (int64_t)row * dv.ntiles; t_eq = dv.tile_b + (int64_t)row * dv.ntiles; t_sbe = dv.tile_c + (int64_t)row * dv.ntiles; }
+    uint32_t* sbits = cursor; // the candidates' value bits, when they fit
+    const bool cached = ncand <= (uint32_t)dv.emit_keys_cap;
+    if (cached)
+        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) sbits[p] = __ldg(cv + p);
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
+    __syncthreads();
+    auto bits_at = [&](uint32_t p) -> uint32_t { return cached ? sbits[p] : __ldg(cv + p); };
+    auto key_at = [&](uint32_t p) -> uint32_t { return order_key<KIND>(bits_at(p)); };
 
     uint32_t T, above;
-    rank_key<KIND>(cv, ncand, k, h, sm, &T, &above);
+    rank_key(key_at, ncand, k, h, sm, &T, &above);
     const uint32_t r = k - above; // how many coordinates with key == T are kept (lowest first)
 
     if (KIND == SEL_TOPK) {
         // Candidate bound for the next step: only a guess (the next step verifies that it kept
         // at least k coordinates and otherwise selects exactly from the dense row).  The k
-        // chosen coordinates drop to ~0, so aim the bound at today's rank 3.5 k, reading the
+        // chosen coordinates drop to ~0, so aim the bound at today's rank 2.5 k, reading the
         // key of that rank off a straight line through (rank k, T) and (rank ncand, bound).
         if (threadIdx.x == 0) dv.row_lo[row] = next_bound(dv.row_lo[row], T, ncand, k);
     }
 
-    // per tile: candidates above T, candidates equal to T
+    // 2. counts per tile and per slab.  kBatch slabs at a time so that the index loads of a
+    // batch are in flight together.
+    constexpr int kBatch = 8;
+    for (int64_t s0 = warp; s0 < nslab; s0 += (kSelThreads / 32) * kBatch) {
+        uint32_t idx[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
+            const uint32_t p = (uint32_t)(sl << 5) + lane;
+            idx[u] = (sl < nslab && p < ncand) ? __ldg(ci + p) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
+            if (sl >= nslab) break;
+            const uint32_t p = (uint32_t)(sl << 5) + lane;
+            bool gt = false, eq = false;
+            if (p < ncand) {
+                const uint32_t kk = key_at(p);
+                gt = kk > T;
+                eq = kk == T;
+                if (gt | eq) atomicAdd(gt ? &t_gt[idx[u] / kTile] : &t_eq[idx[u] / kTile], 1u);
+            }
+            const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+            if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); }
+        }
+    }
+    __syncthreads();
+
+    // 3. prefixes.  Tiles: t_gt <- keys above T before the tile, t_eq <- equal keys before it.
+    uint32_t tot_a, tot_b;
+    block_scan_pair(t_gt, t_eq, dv.ntiles, sm, s_carry, &tot_a, &tot_b);
+    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_a, &tot_b);
+    uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
     const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
     const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
-    uint32_t* tgt = dv.tile_a + (int64_t)row * dv.ntiles;
-    uint32_t* teq = dv.tile_b + (int64_t)row * dv.ntiles;
-    for (int64_t t = warp; t < dv.ntiles; t += kSelThreads / 32) {
-        const uint32_t off = so[t], cnt = sc[t];
-        uint32_t gt = 0, eq = 0;
-        for (uint32_t p = lane; p < cnt; p += 32) {
-            const uint32_t key = order_key<KIND>(cv[off + p]);
-            gt += key > T;
-            eq += key == T;
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
+        const uint32_t gb = t_gt[t], eb = t_eq[t];
+        tp[t] = gb + (eb < r ? eb : r);
+        // the two flat prefixes at the tile's first candidate: t_gt <- above, t_sbe <- equal
+        uint32_t pg = 0, pe = 0;
+        if (sc[t]) {
+            const uint32_t first = so[t], s0 = first >> 5;
+            pg = slab_g[s0];
+            pe = slab_e[s0];
+            for (uint32_t p = s0 << 5; p < first; ++p) {
+                const uint32_t kk = key_at(p);
+                pg += kk > T;
+                pe += kk == T;
+            }
         }
-        gt = __reduce_add_sync(0xffffffffu, gt);
-        eq = __reduce_add_sync(0xffffffffu, eq);
-        if (lane == 0) { tgt[t] = gt; teq[t] = eq; }
-    }
-    if (threadIdx.x == 0) { s_carry[0] = 0u; s_carry[1] = 0u; }
-    __syncthreads();
-    // prefix over tiles: tile_ptr = (#above before) + min(#equal before, r); teq <- #equal before
-    uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
-    for (int64_t t0 = 0; t0 < dv.ntiles; t0 += kSelThreads) {
-        const int64_t t = t0 + threadIdx.x;
-        const uint32_t gt = t < dv.ntiles ? tgt[t] : 0u;
-        const uint32_t eq = t < dv.ntiles ? teq[t] : 0u;
-        uint32_t tot_gt, tot_eq;
-        const uint32_t ex_gt = block_scan_excl<kSelThreads>(gt, sm, &tot_gt);
-        const uint32_t ex_eq = block_scan_excl<kSelThreads>(eq, sm, &tot_eq);
-        const uint32_t cg = s_carry[0], ce = s_carry[1];
-        if (t < dv.ntiles) {
-            const uint32_t eqb = ce + ex_eq;
-            tp[t] = cg + ex_gt + (eqb < r ? eqb : r);
-            teq[t] = eqb;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) { s_carry[0] = cg + tot_gt; s_carry[1] = ce + tot_eq; }
-        __syncthreads();
+        t_gt[t] = pg;
+        t_sbe[t] = pe;
     }
     if (threadIdx.x == 0) tp[dv.ntiles] = k;
     __syncthreads();
-    publish_ranges(dv, row, tp);
-    // ordered compaction, one warp per tile
+    // 4. every chosen candidate writes itself
     uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch;
     float* mv = dv.msg_val + (int64_t)row * dv.kpitch;
     const float* xr = a.X + (int64_t)row * dv.ld;
     const float* hr = a.Xhat + (int64_t)row * dv.ld;
     const uint32_t lt = (1u << lane) - 1u;
-    for (int64_t t = warp; t < dv.ntiles; t += kSelThreads / 32) {
-        const uint32_t off = so[t], cnt = sc[t];
-        uint32_t out = tp[t], eqrank = teq[t];
-        for (uint32_t p0 = 0; p0 < cnt; p0 += 32) {
-            const uint32_t p = p0 + lane;
-            const bool act = p < cnt;
-            const uint32_t idx = act ? ci[off + p] : 0u;
-            const uint32_t bits = act ? cv[off + p] : 0u;
-            const uint32_t key = order_key<KIND>(bits);
-            const bool iseq = act && key == T;
-            const uint32_t eqb = __ballot_sync(0xffffffffu, iseq);
-            const bool sel = act && (key > T || (iseq && eqrank + __popc(eqb & lt) < r));
-            const uint32_t sb = __ballot_sync(0xffffffffu, sel);
-            if (sel) {
-                const uint32_t pos = out + __popc(sb & lt);
-                mi[pos] = idx;
-                mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits) : __fsub_rn(xr[idx], hr[idx]);
+    for (int64_t s0 = warp; s0 < nslab; s0 += (kSelThreads / 32) * kBatch) {
+        uint32_t idx[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
+            const uint32_t p = (uint32_t)(sl << 5) + lane;
+            idx[u] = (sl < nslab && p < ncand) ? __ldg(ci + p) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
+            if (sl >= nslab) break;
+            const uint32_t p = (uint32_t)(sl << 5) + lane;
+            const bool act = p < ncand;
+            const uint32_t bits = act ? bits_at(p) : 0u;
+            const uint32_t kk = order_key<KIND>(bits);
+            const bool gt = act && kk > T, eq = act && kk == T;
+            const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+            if (gt | eq) {
+                const uint32_t tile = idx[u] / kTile;
+                const uint32_t g_in = slab_g[sl] + __popc(bg & lt) - t_gt[tile];  // above T, earlier in the tile
+                const uint32_t e_in = slab_e[sl] + __popc(be & lt) - t_sbe[tile]; // equal to T, earlier in the tile
+                const uint32_t eqb = t_eq[tile];                                  // equal to T, in earlier tiles
+                const uint32_t room = r > eqb ? r - eqb : 0u;                     // equal keys this tile may keep
+                if (gt || e_in < room) {
+                    const uint32_t pos = tp[tile] + g_in + (e_in < room ? e_in : room);
+                    mi[pos] = idx[u];
+                    mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits) : __fsub_rn(xr[idx[u]], hr[idx[u]]);
+                }
             }
-            out += __popc(sb);
-            eqrank += __popc(eqb);
         }
     }
+    publish_ranges(dv, row, tp);
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
@@ -474,7 +581,17 @@ cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t
 template <int KIND>
 static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
 {
-    emit_kernel<KIND><<<dv.n, kSelThreads, 0, st>>>(dv, a, fused ? 1 : 0);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(emit_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kEmitSmemBudget);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    emit_kernel<KIND><<<dv.n, kSelThreads, (size_t)dv.emit_smem_bytes, st>>>(dv, a, fused ? 1 : 0);
     if (a.vec) exact_kernel<KIND, true><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     else exact_kernel<KIND, false><<<dv.n, kSelThreads, 0, st>>>(dv, a);
     *a.launches += 2;
