@@ -77,6 +77,35 @@ float qsgd_tau(int64_t len, int32_t s, bool biased)
     return (float)(1.0 + (a < b ? a : b));
 }
 
+// Ask the L2 cache to keep the context's hot arena resident for work on `st` (best effort:
+// failures are ignored, the results do not depend on it).  Raises the persisting-L2 carve-out
+// of the current context if it is smaller than the arena needs; it is never lowered here.
+void keep_hot_in_l2(choco_ctx* ctx, cudaStream_t st)
+{
+    ctx->hot_set = true;
+    ctx->hot_stream = st;
+    int dev = 0, max_persist = 0, max_window = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
+    cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev);
+    cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev);
+    if (max_persist <= 0 || max_window <= 0) { cudaGetLastError(); return; }
+    const size_t want = std::min<size_t>((size_t)ctx->hot_bytes, (size_t)max_persist / 4 * 3);
+    size_t have = 0;
+    cudaDeviceGetLimit(&have, cudaLimitPersistingL2CacheSize);
+    if (have < want) cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want);
+    cudaDeviceGetLimit(&have, cudaLimitPersistingL2CacheSize);
+    cudaStreamAttrValue av;
+    std::memset(&av, 0, sizeof(av));
+    av.accessPolicyWindow.base_ptr = ctx->hot_base;
+    av.accessPolicyWindow.num_bytes = std::min<size_t>((size_t)ctx->hot_bytes, (size_t)max_window);
+    const double ratio = (double)have / (double)av.accessPolicyWindow.num_bytes;
+    av.accessPolicyWindow.hitRatio = ratio >= 1.0 ? 1.0f : (float)ratio;
+    av.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+    av.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+    cudaStreamSetAttribute(st, cudaStreamAttributeAccessPolicyWindow, &av);
+    cudaGetLastError(); // best effort
+}
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
 
@@ -96,6 +125,7 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     a.vec = (dv.ld % 4 == 0) && aligned16(X) && aligned16(Xhat) && aligned16(S) &&
             (!G || aligned16(G)) && (!M || aligned16(M));
     if (ctx->last_x != X || ctx->last_xhat != Xhat) ctx->prepared = false;
+    if (ctx->hot_base && (!ctx->hot_set || ctx->hot_stream != st)) keep_hot_in_l2(ctx, st);
 
     cudaError_t e = cudaSuccess;
     const bool sparse = dv.kind == CHOCO_Q_TOPK || dv.kind == CHOCO_Q_RANDK;
@@ -206,21 +236,40 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     if (p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK) {
         dv.k = p->k;
         dv.kpitch = round_up(p->k, 4);
-        // candidates per row: aimed at 2.5-3.5 k, with room for a bound that was guessed low
-        int64_t cap = 8 * p->k > p->k + 8192 ? 8 * p->k : p->k + 8192;
+        // candidates per row: aimed at 2.5 k, with room for a bound that was guessed low
+        int64_t cap = 6 * p->k > p->k + 8192 ? 6 * p->k : p->k + 8192;
         dv.cap = cap < d ? cap : d;
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_idx, n * dv.kpitch);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_val, n * dv.kpitch);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_ptr, n * (dv.ntiles + 1));
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.rec, (int64_t)n * dv.ntiles * dv.maxdeg);
+        {
+            // One arena for what one kernel writes and the next reads back within a step.  Its
+            // head (range records, messages, per-tile tables) is read with dependent loads by
+            // the update kernel: steps ask the L2 cache to keep that part resident while the
+            // dense arrays stream past it (measured: keeping the candidates too does not pay).
+            const int64_t b_rec = round_up((int64_t)n * dv.ntiles * dv.maxdeg * 16, 256);
+            const int64_t b_msg = round_up(n * dv.kpitch * 4, 256);
+            const int64_t b_tp = round_up(n * (dv.ntiles + 1) * 4, 256);
+            const int64_t b_cand = round_up(n * dv.cap * 4, 256);
+            const int64_t b_seg = round_up(n * dv.ntiles * 4, 256);
+            const int64_t b_row = round_up((int64_t)n * 4, 256);
+            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 3 * b_row;
+            unsigned char* arena = nullptr;
+            if (e == cudaSuccess) e = dev_alloc(ctx, &arena, total);
+            unsigned char* q = arena;
+            dv.rec = (uint4*)q; q += b_rec;
+            dv.msg_idx = (uint32_t*)q; q += b_msg;
+            dv.msg_val = (float*)q; q += b_msg;
+            dv.tile_ptr = (uint32_t*)q; q += b_tp;
+            dv.seg_off = (uint32_t*)q; q += b_seg;
+            dv.seg_cnt = (uint32_t*)q; q += b_seg;
+            dv.row_lo = (uint32_t*)q; q += b_row;
+            dv.row_count = (uint32_t*)q; q += b_row;
+            dv.row_flags = (uint32_t*)q; q += b_row;
+            const int64_t hot = q - arena; // the candidates behind it are written once, read once
+            dv.cand_idx = (uint32_t*)q; q += b_cand;
+            dv.cand_val = (uint32_t*)q; q += b_cand;
+            ctx->hot_base = arena;
+            ctx->hot_bytes = hot;
+        }
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.hist, (int64_t)n * kHistBins);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_lo, n);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_count, n);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.row_flags, n);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.cand_idx, n * dv.cap);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.cand_val, n * dv.cap);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.seg_off, n * dv.ntiles);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.seg_cnt, n * dv.ntiles);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_a, n * dv.ntiles);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_b, n * dv.ntiles);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_c, n * dv.ntiles);

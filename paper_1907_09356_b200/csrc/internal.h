@@ -134,6 +134,11 @@ struct choco_ctx {
     const float* last_x;
     const float* last_xhat;
     int64_t msg_bytes_per_worker;
+    // arena that steps ask the L2 cache to keep resident (messages, records, candidates)
+    void* hot_base;
+    int64_t hot_bytes;
+    bool hot_set;
+    cudaStream_t hot_stream;
     // host staging for choco_sgd_step_host
     float* stage[4];
     // consensus scratch
