@@ -13,8 +13,8 @@
 //   emit    : one block per row: exact k-th key by radix refinement over the candidates,
 //             tie ranks, ordered compaction into the message; the candidate bound for the
 //             next step.
-//   exact   : rows whose candidates are unusable (too many, too few, overflow) run a
-//             one-block exact selection straight from the dense row.
+//   exact   : rows whose candidates are unusable (too many, too few, overflow) are selected
+//             exactly, by the same block, straight from the dense row.
 #include "select.cuh"
 
 namespace choco {
@@ -284,6 +284,97 @@ __device__ __forceinline__ void block_scan_pair(uint32_t* a, uint32_t* b, int64_
     *tot_b = carry[1];
 }
 
+// ---------------------------------------------------------------------------------------
+// exact: one block selects straight from the dense row (three radix passes and an ordered
+// compaction pass).  Slow; only for rows whose candidates could not be used.
+// ---------------------------------------------------------------------------------------
+template <int KIND, bool VEC>
+__device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int row, uint32_t* h, uint32_t* sm)
+{
+    const uint32_t k = (uint32_t)dv.k;
+    const int64_t span = (int64_t)kSelThreads * kQuad; // coordinates per block iteration
+    const int64_t nspan = (dv.d + span - 1) / span;
+    constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
+    uint32_t prefix = 0, pmask = 0, need = k;
+    const int shifts[3] = {21, 10, 0};
+    const int nbins[3] = {2048, 2048, 1024};
+    for (int pass = 0; pass < 3; ++pass) {
+        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
+        __syncthreads();
+        for (int64_t c = (int64_t)threadIdx.x * kQuad; c < dv.d; c += span) {
+            uint32_t bits[4];
+            quad_bits<KIND, VEC>(dv, a, row, c, bits);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t key = order_key<KIND>(bits[e]);
+                if (c + e < dv.d && (key & pmask) == prefix)
+                    atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
+            }
+        }
+        __syncthreads();
+        uint32_t digit, above;
+        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
+        need -= above;
+        prefix |= digit << shifts[pass];
+        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
+        __syncthreads();
+    }
+    const uint32_t T = prefix, r = need;
+    uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch;
+    float* mv = dv.msg_val + (int64_t)row * dv.kpitch;
+    uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
+    const float* xr = a.X + (int64_t)row * dv.ld;
+    const float* hr = a.Xhat + (int64_t)row * dv.ld;
+    uint32_t run_gt = 0, run_eq = 0; // coordinates above / equal to T before this span
+    for (int64_t sp = 0; sp < nspan; ++sp) {
+        const int64_t c = sp * span + (int64_t)threadIdx.x * kQuad;
+        uint32_t bits[4] = {0u, 0u, 0u, 0u};
+        uint32_t gtm = 0, eqm = 0;
+        if (c < dv.d) {
+            quad_bits<KIND, VEC>(dv, a, row, c, bits);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t key = order_key<KIND>(bits[e]);
+                if (c + e < dv.d) {
+                    gtm |= (uint32_t)(key > T) << e;
+                    eqm |= (uint32_t)(key == T) << e;
+                }
+            }
+        }
+        uint32_t tot;
+        const uint32_t ex = block_scan_excl<kSelThreads>(__popc(gtm) | (__popc(eqm) << 16), sm, &tot);
+        uint32_t g = run_gt + (ex & 0xFFFFu), q = run_eq + (ex >> 16);
+        // the first thread of every tile records how many coordinates were chosen before it
+        if ((threadIdx.x % (kTile / kQuad)) == 0) {
+            const int64_t t = sp * kTilesPerSpan + threadIdx.x / (kTile / kQuad);
+            if (t < dv.ntiles) tp[t] = g + (q < r ? q : r);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool isgt = (gtm >> e) & 1u, iseq = (eqm >> e) & 1u;
+            if (isgt || (iseq && q < r)) {
+                const uint32_t pos = g + (q < r ? q : r);
+                mi[pos] = (uint32_t)(c + e);
+                mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits[e])
+                                           : __fsub_rn(xr[c + e], hr[c + e]);
+            }
+            g += isgt;
+            q += iseq;
+        }
+        run_gt += tot & 0xFFFFu;
+        run_eq += tot >> 16;
+    }
+    if (threadIdx.x == 0) tp[dv.ntiles] = k;
+    __syncthreads();
+    publish_ranges(dv, row, tp);
+    if (threadIdx.x == 0) {
+        dv.row_flags[row] = 0u;
+        dv.row_count[row] = 0u;
+        if (KIND == SEL_TOPK) dv.row_lo[row] = lower_bound_key(T, 3u);
+        atomicAdd(&dv.stats->exact_rows, 1ull);
+    }
+}
+
 // Layout of the emit kernel's dynamic shared memory, fixed at choco_init from the sizes:
 // slab prefix arrays, per-tile arrays and a cache of the candidate keys go to shared memory
 // as far as they fit (in that order); what does not fit lives in global scratch.
@@ -295,7 +386,7 @@ __device__ __forceinline__ void block_scan_pair(uint32_t* a, uint32_t* b, int64_
 //   3. prefix over tiles -> tile_ptr and the number of equal keys before each tile; prefix
 //      over slabs; per tile the two prefixes at its first candidate;
 //   4. every chosen candidate computes its own output position and writes itself.
-template <int KIND>
+template <int KIND, bool VEC>
 __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused)
 {
     extern __shared__ uint32_t dyn[];
@@ -309,10 +400,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const uint32_t k = (uint32_t)dv.k;
     __syncthreads();
     if ((flags & kRowExact) || ncand > (uint32_t)dv.cap || ncand < k) {
-        if (threadIdx.x == 0) {
-            dv.row_flags[row] = kRowExact;
-            dv.row_count[row] = 0u;
-        }
+        exact_row<KIND, VEC>(dv, a, row, h, sm); // the candidates cannot be used
         return;
     }
     const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
@@ -450,101 +538,6 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
 }
 
 // ---------------------------------------------------------------------------------------
-// exact: one block selects straight from the dense row (three radix passes and an ordered
-// compaction pass).  Slow; only for rows whose candidates could not be used.
-// ---------------------------------------------------------------------------------------
-template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kSelThreads) exact_kernel(Dev dv, StepArgs a)
-{
-    __shared__ uint32_t h[kHistBins];
-    __shared__ uint32_t sm[36];
-    const int row = blockIdx.x;
-    if (!(dv.row_flags[row] & kRowExact)) return;
-    const uint32_t k = (uint32_t)dv.k;
-    const int64_t span = (int64_t)kSelThreads * kQuad; // coordinates per block iteration
-    const int64_t nspan = (dv.d + span - 1) / span;
-    constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
-    uint32_t prefix = 0, pmask = 0, need = k;
-    const int shifts[3] = {21, 10, 0};
-    const int nbins[3] = {2048, 2048, 1024};
-    for (int pass = 0; pass < 3; ++pass) {
-        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
-        __syncthreads();
-        for (int64_t c = (int64_t)threadIdx.x * kQuad; c < dv.d; c += span) {
-            uint32_t bits[4];
-            quad_bits<KIND, VEC>(dv, a, row, c, bits);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t key = order_key<KIND>(bits[e]);
-                if (c + e < dv.d && (key & pmask) == prefix)
-                    atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
-            }
-        }
-        __syncthreads();
-        uint32_t digit, above;
-        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
-        need -= above;
-        prefix |= digit << shifts[pass];
-        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
-        __syncthreads();
-    }
-    const uint32_t T = prefix, r = need;
-    uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch;
-    float* mv = dv.msg_val + (int64_t)row * dv.kpitch;
-    uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
-    const float* xr = a.X + (int64_t)row * dv.ld;
-    const float* hr = a.Xhat + (int64_t)row * dv.ld;
-    uint32_t run_gt = 0, run_eq = 0; // coordinates above / equal to T before this span
-    for (int64_t sp = 0; sp < nspan; ++sp) {
-        const int64_t c = sp * span + (int64_t)threadIdx.x * kQuad;
-        uint32_t bits[4] = {0u, 0u, 0u, 0u};
-        uint32_t gtm = 0, eqm = 0;
-        if (c < dv.d) {
-            quad_bits<KIND, VEC>(dv, a, row, c, bits);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t key = order_key<KIND>(bits[e]);
-                if (c + e < dv.d) {
-                    gtm |= (uint32_t)(key > T) << e;
-                    eqm |= (uint32_t)(key == T) << e;
-                }
-            }
-        }
-        uint32_t tot;
-        const uint32_t ex = block_scan_excl<kSelThreads>(__popc(gtm) | (__popc(eqm) << 16), sm, &tot);
-        uint32_t g = run_gt + (ex & 0xFFFFu), q = run_eq + (ex >> 16);
-        // the first thread of every tile records how many coordinates were chosen before it
-        if ((threadIdx.x % (kTile / kQuad)) == 0) {
-            const int64_t t = sp * kTilesPerSpan + threadIdx.x / (kTile / kQuad);
-            if (t < dv.ntiles) tp[t] = g + (q < r ? q : r);
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const bool isgt = (gtm >> e) & 1u, iseq = (eqm >> e) & 1u;
-            if (isgt || (iseq && q < r)) {
-                const uint32_t pos = g + (q < r ? q : r);
-                mi[pos] = (uint32_t)(c + e);
-                mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits[e])
-                                           : __fsub_rn(xr[c + e], hr[c + e]);
-            }
-            g += isgt;
-            q += iseq;
-        }
-        run_gt += tot & 0xFFFFu;
-        run_eq += tot >> 16;
-    }
-    if (threadIdx.x == 0) tp[dv.ntiles] = k;
-    __syncthreads();
-    publish_ranges(dv, row, tp);
-    if (threadIdx.x == 0) {
-        dv.row_flags[row] = 0u;
-        dv.row_count[row] = 0u;
-        if (KIND == SEL_TOPK) dv.row_lo[row] = lower_bound_key(T, 3u);
-        atomicAdd(&dv.stats->exact_rows, 1ull);
-    }
-}
-
-// ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
 
@@ -581,20 +574,18 @@ cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t
 template <int KIND>
 static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
 {
-    static bool configured[64] = {};
+    auto kern = a.vec ? emit_kernel<KIND, true> : emit_kernel<KIND, false>;
+    static bool configured[64][2] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(emit_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kEmitSmemBudget);
+    if (dev < 0 || dev >= 64 || !configured[dev][a.vec ? 1 : 0]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmitSmemBudget);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
+        if (dev >= 0 && dev < 64) configured[dev][a.vec ? 1 : 0] = true;
     }
-    emit_kernel<KIND><<<dv.n, kSelThreads, (size_t)dv.emit_smem_bytes, st>>>(dv, a, fused ? 1 : 0);
-    if (a.vec) exact_kernel<KIND, true><<<dv.n, kSelThreads, 0, st>>>(dv, a);
-    else exact_kernel<KIND, false><<<dv.n, kSelThreads, 0, st>>>(dv, a);
-    *a.launches += 2;
+    kern<<<dv.n, kSelThreads, (size_t)dv.emit_smem_bytes, st>>>(dv, a, fused ? 1 : 0);
+    *a.launches += 1;
     return cudaGetLastError();
 }
 
