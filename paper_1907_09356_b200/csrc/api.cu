@@ -250,7 +250,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             const int64_t b_cand = round_up(n * dv.cap * 4, 256);
             const int64_t b_seg = round_up(n * dv.ntiles * 4, 256);
             const int64_t b_row = round_up((int64_t)n * 4, 256);
-            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 3 * b_row;
+            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 4 * b_row;
             unsigned char* arena = nullptr;
             if (e == cudaSuccess) e = dev_alloc(ctx, &arena, total);
             unsigned char* q = arena;
@@ -263,6 +263,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             dv.row_lo = (uint32_t*)q; q += b_row;
             dv.row_count = (uint32_t*)q; q += b_row;
             dv.row_flags = (uint32_t*)q; q += b_row;
+            dv.row_aim = (uint32_t*)q; q += b_row;
             const int64_t hot = q - arena; // the candidates behind it are written once, read once
             dv.cand_idx = (uint32_t*)q; q += b_cand;
             dv.cand_val = (uint32_t*)q; q += b_cand;

@@ -54,6 +54,7 @@ struct Dev {
     uint32_t* hist;              // [n, kHistBins]
     uint32_t* row_lo;            // [n] lower bound of the ordering key for candidates
     uint32_t* row_count;         // [n] candidates collected
+    uint32_t* row_aim;           // [n] rank the next bound aims at, in units of k / 256
     uint32_t* row_flags;         // [n]
     uint32_t* cand_idx;          // [n, cap]
     uint32_t* cand_val;          // [n, cap] value bits (top-k) or random word (random-k)

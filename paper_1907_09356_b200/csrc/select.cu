@@ -19,6 +19,11 @@
 
 namespace choco {
 
+// Rank the candidate bound aims at, in units of k / 256, kept per row: it starts at 2.5 k,
+// creeps down to 1.75 k while the guesses keep holding (fewer candidates = less work in the
+// emit kernel) and jumps back to 3 k when a row had to be selected exactly.
+constexpr uint32_t kAimStart = 640u, kAimMin = 448u, kAimAfterMiss = 768u, kAimStep = 8u;
+
 // value bits of the four coordinates of a quad (top-k: x - x^; random-k: Philox words)
 template <int KIND, bool VEC>
 __device__ __forceinline__ void quad_bits(const Dev& dv, const StepArgs& a, int row, int64_t c,
@@ -84,6 +89,7 @@ __global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv)
     block_find_digit<kSelThreads>(h, kHistBins, need, sm, &digit, &above);
     if (threadIdx.x == 0) {
         dv.row_lo[row] = digit << 21;
+        dv.row_aim[row] = kAimStart;
         dv.row_count[row] = 0u;
         // every coordinate with this digit or a higher one becomes a candidate
         dv.row_flags[row] = ((int64_t)above + (int64_t)h[digit] > dv.cap) ? kRowExact : 0u;
@@ -241,18 +247,18 @@ __device__ __forceinline__ uint32_t lower_bound_key(uint32_t key, uint32_t eight
     return key > dec ? key - dec : 0u;
 }
 
-// Rank aimed at by the candidate bound: 2.5 k (the k chosen leave, about 1.5 k stay)
-__host__ __device__ __forceinline__ uint64_t target_rank(uint64_t k) { return 2 * k + k / 2; }
 
 // lo: bound the ncand candidates were collected with (their rank-ncand key, roughly);
 // T: key of rank k.  The key is read off a line in (log rank, key) through the two points
 // (tails fall off roughly like that; a line in the rank itself sits above a convex tail and
 // would keep too few), at most half an octave below the old bound.
-__device__ __forceinline__ uint32_t next_bound(uint32_t lo, uint32_t T, uint32_t ncand, uint32_t k)
+__device__ __forceinline__ uint32_t next_bound(uint32_t lo, uint32_t T, uint32_t ncand, uint32_t k,
+                                               uint32_t aim)
 {
     if (ncand <= k || T < lo) return lower_bound_key(lo, 4u);
     const float span = (float)(T - lo);
-    const float want = (float)target_rank(k);
+    const float want = (float)k * (float)aim * (1.0f / 256.0f);
+    if (want <= (float)k) return T;
     const float frac = __log2f(want / (float)k) / __log2f((float)ncand / (float)k); // 1 at rank ncand
     const float drop = span * frac;                                                // below T
     if (drop <= span) return T - (uint32_t)drop;
@@ -370,7 +376,10 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     if (threadIdx.x == 0) {
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
-        if (KIND == SEL_TOPK) dv.row_lo[row] = lower_bound_key(T, 3u);
+        if (KIND == SEL_TOPK) {
+            dv.row_lo[row] = lower_bound_key(T, 3u);
+            dv.row_aim[row] = kAimAfterMiss;
+        }
         atomicAdd(&dv.stats->exact_rows, 1ull);
     }
 }
@@ -432,7 +441,12 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         // at least k coordinates and otherwise selects exactly from the dense row).  The k
         // chosen coordinates drop to ~0, so aim the bound at today's rank 2.5 k, reading the
         // key of that rank off a straight line through (rank k, T) and (rank ncand, bound).
-        if (threadIdx.x == 0) dv.row_lo[row] = next_bound(dv.row_lo[row], T, ncand, k);
+        if (threadIdx.x == 0) {
+            uint32_t aim = dv.row_aim[row];
+            aim = aim > kAimMin + kAimStep ? aim - kAimStep : kAimMin;
+            dv.row_aim[row] = aim;
+            dv.row_lo[row] = next_bound(dv.row_lo[row], T, ncand, k, aim);
+        }
     }
 
     // 2. counts per tile and per slab.  kBatch slabs at a time so that the index loads of a
