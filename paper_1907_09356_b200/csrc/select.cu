@@ -174,27 +174,29 @@ __global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs 
 // keys actually span: candidates share their leading bits, so a fixed radix digit would pile
 // them into a handful of bins (and serialise the shared-memory atomics); bins spread over
 // [min, max] instead, then over the chosen bin, until a bin is one key wide.
-template <typename KeyFn>
-__device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t rank, uint32_t* h,
-                                         uint32_t* sm, uint32_t* key_out, uint32_t* above_out)
+// Block-wide minimum and maximum of per-thread values (kSelThreads threads); `sm` needs 64 words.
+__device__ __forceinline__ void block_min_max(uint32_t& lo, uint32_t& hi, uint32_t* sm)
 {
-    // range of the keys
-    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
-    for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
-        const uint32_t kk = key(p);
-        lo = kk < lo ? kk : lo;
-        hi = kk > hi ? kk : hi;
-    }
     lo = __reduce_min_sync(0xffffffffu, lo);
     hi = __reduce_max_sync(0xffffffffu, hi);
     __syncthreads(); // protect sm from the previous use
-    if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = lo; h[threadIdx.x >> 5] = hi; }
+    if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = lo; sm[32 + (threadIdx.x >> 5)] = hi; }
     __syncthreads();
     for (int w = 0; w < kSelThreads / 32; ++w) {
         lo = sm[w] < lo ? sm[w] : lo;
-        hi = h[w] > hi ? h[w] : hi;
+        hi = sm[32 + w] > hi ? sm[32 + w] : hi;
     }
     __syncthreads();
+}
+
+constexpr int kListCap = 1024; // a histogram bin this small is resolved by direct comparison
+
+template <typename KeyFn>
+__device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t rank, uint32_t lo,
+                                         uint32_t hi, uint32_t* h, uint32_t* sm, uint32_t* key_out,
+                                         uint32_t* above_out)
+{
+    // [lo, hi] is the range of the keys (block_min_max)
     uint32_t need = rank, above_total = 0;
     for (;;) {
         const uint32_t width = hi - lo;
@@ -209,6 +211,7 @@ __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t ran
         __syncthreads();
         uint32_t digit, above;
         block_find_digit<kSelThreads>(h, nbins, need, sm, &digit, &above);
+        const uint32_t inbin = h[digit];
         need -= above;
         above_total += above;
         const uint32_t nlo = lo + (digit << shift);
@@ -218,6 +221,33 @@ __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t ran
         hi = nhi;
         __syncthreads();
         if (shift == 0) break;
+        if (inbin <= (uint32_t)kListCap) {
+            // few keys left in [lo, hi]: list them (h is free now) and rank them directly
+            uint32_t* list = h;          // kListCap keys
+            uint32_t* count = sm + 40;   // one word
+            if (threadIdx.x == 0) { *count = 0u; sm[41] = lo; sm[42] = 0u; }
+            __syncthreads();
+            for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+                const uint32_t kk = key(p);
+                if (kk >= lo && kk <= hi) list[atomicAdd(count, 1u)] = kk;
+            }
+            __syncthreads();
+            const uint32_t m = *count; // == inbin
+            if (threadIdx.x < m) {
+                const uint32_t mine = list[threadIdx.x];
+                uint32_t g = 0, e = 0;
+                for (uint32_t q = 0; q < m; ++q) {
+                    g += list[q] > mine;
+                    e += list[q] == mine;
+                }
+                if (g < need && need <= g + e) { sm[41] = mine; sm[42] = g; } // same values from every such thread
+            }
+            __syncthreads();
+            lo = sm[41];
+            above_total += sm[42];
+            __syncthreads();
+            break;
+        }
     }
     *key_out = lo;
     *above_out = above_total;
@@ -400,7 +430,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
 {
     extern __shared__ uint32_t dyn[];
     __shared__ uint32_t h[kHistBins];
-    __shared__ uint32_t sm[36];
+    __shared__ uint32_t sm[64];
     __shared__ uint32_t s_carry[2];
     const int row = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -425,15 +455,21 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     else { t_gt = dv.tile_a + (int64_t)row * dv.ntiles; t_eq = dv.tile_b + (int64_t)row * dv.ntiles; t_sbe = dv.tile_c + (int64_t)row * dv.ntiles; }
     uint32_t* sbits = cursor; // the candidates' value bits, when they fit
     const bool cached = ncand <= (uint32_t)dv.emit_keys_cap;
-    if (cached)
-        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) sbits[p] = __ldg(cv + p);
+    uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
+    for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+        const uint32_t bits = __ldg(cv + p);
+        if (cached) sbits[p] = bits;
+        const uint32_t kk = order_key<KIND>(bits);
+        klo = kk < klo ? kk : klo;
+        khi = kk > khi ? kk : khi;
+    }
     for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
-    __syncthreads();
+    block_min_max(klo, khi, sm);
     auto bits_at = [&](uint32_t p) -> uint32_t { return cached ? sbits[p] : __ldg(cv + p); };
     auto key_at = [&](uint32_t p) -> uint32_t { return order_key<KIND>(bits_at(p)); };
 
     uint32_t T, above;
-    rank_key(key_at, ncand, k, h, sm, &T, &above);
+    rank_key(key_at, ncand, k, klo, khi, h, sm, &T, &above);
     const uint32_t r = k - above; // how many coordinates with key == T are kept (lowest first)
 
     if (KIND == SEL_TOPK) {
