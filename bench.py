@@ -184,6 +184,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-stride", type=int, default=8,
+                    help="time the update kernel with CUDA events on every Nth timed step")
     ap.add_argument("--pool", type=int, default=8, help="gradient tensors cycled through (>= 2)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -254,6 +256,7 @@ def main():
     barrier()
     st0 = choco.choco_get_stats(ch.ctx)
     choco.choco_profile_enable(ch.ctx, args.steps)
+    choco.choco_profile_set_stride(ch.ctx, args.profile_stride)   # events between kernels cost time
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -317,7 +320,8 @@ def main():
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None,
                          "traffic": None, "algorithmic_bytes_per_launch": upd_bytes,
-                         "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec},
+                         "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec,
+                         "timed_every": args.profile_stride},
             "gpu_launches": int(st1["kernel_launches"] - st0["kernel_launches"]),
             "selection": {k: int(st1[k] - st0[k]) for k in ("prepared_rows", "recompressed_rows", "exact_rows")},
             "finite": finite,

@@ -218,6 +218,9 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
  * milliseconds, then clears the record.  Not part of the method; used by benchmarks.
  */
 int choco_profile_enable(choco_ctx* ctx, int32_t max_steps);
+/* Record only every `stride`-th step call (default 1): the events sit between the step's
+ * kernels and keep them from overlapping, so timing every step slows the steps down. */
+int choco_profile_set_stride(choco_ctx* ctx, int32_t stride);
 int choco_profile_read(choco_ctx* ctx, int32_t* steps_recorded, double* update_ms_total,
                        void* stream);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "choco_get_step",
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error", "choco_consensus_error_noalloc",
-    "choco_get_stats", "choco_profile_enable", "choco_profile_read", "choco_strerror",
+    "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
     "choco_last_cuda_error",
 ]
 
@@ -75,6 +75,7 @@ def load() -> ctypes.CDLL:
         lib.choco_consensus_error_noalloc.argtypes = [vp, i32, i64, i64, vp, vp]
         lib.choco_get_stats.argtypes = [vp, ctypes.POINTER(choco_stats), vp]
         lib.choco_profile_enable.argtypes = [vp, i32]
+        lib.choco_profile_set_stride.argtypes = [vp, i32]
         lib.choco_profile_read.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double), vp]
         lib.choco_strerror.argtypes = [ctypes.c_int]
         lib.choco_strerror.restype = ctypes.c_char_p
@@ -217,6 +218,10 @@ def choco_get_stats(ctx, stream=None) -> dict:
 
 def choco_profile_enable(ctx, max_steps: int) -> None:
     _check(load().choco_profile_enable(ctx, max_steps), ctx)
+
+
+def choco_profile_set_stride(ctx, stride: int) -> None:
+    _check(load().choco_profile_set_stride(ctx, stride), ctx)
 
 
 def choco_profile_read(ctx, stream=None) -> tuple[int, float]:

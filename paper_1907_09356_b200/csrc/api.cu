@@ -138,7 +138,8 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     }
     // the update kernel can collect the next step's candidates from the x' - x^' it holds
     const bool emit = ctx->carry_enabled && apply_can_emit(dv, a);
-    const bool prof = ctx->prof_ev && ctx->prof_n < ctx->prof_cap;
+    const bool prof = ctx->prof_ev && ctx->prof_n < ctx->prof_cap &&
+                      (ctx->prof_stride <= 1 || ctx->steps_enqueued % (uint64_t)ctx->prof_stride == 0);
     if (e == cudaSuccess && prof) e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], st);
     if (e == cudaSuccess) e = launch_apply(dv, a, emit, st);
     if (e == cudaSuccess && prof) {
@@ -538,6 +539,13 @@ int choco_profile_enable(choco_ctx* ctx, int32_t max_steps)
         }
     }
     ctx->prof_cap = max_steps;
+    return CHOCO_OK;
+}
+
+int choco_profile_set_stride(choco_ctx* ctx, int32_t stride)
+{
+    if (!ctx || stride < 1) return CHOCO_ERR_INVALID_ARG;
+    ctx->prof_stride = stride;
     return CHOCO_OK;
 }
 

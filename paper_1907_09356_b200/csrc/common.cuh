@@ -143,6 +143,36 @@ __device__ __forceinline__ uint32_t gather_sign_word(uint32_t nib, int lane)
     return w;
 }
 
+// Programmatic dependent launch: a kernel launched with launch_overlapped() may be scheduled
+// while the kernel before it on the stream is still draining.  It must call
+// wait_for_previous_kernel() before it touches anything that kernel wrote; calling
+// allow_next_kernel() lets the one after it be scheduled early in the same way.
+__device__ __forceinline__ void wait_for_previous_kernel()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void allow_next_kernel()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 __device__ __forceinline__ uint32_t abs_key(float v)
 {
     return __float_as_uint(v) & 0x7FFFFFFFu;

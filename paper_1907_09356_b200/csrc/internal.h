@@ -149,7 +149,7 @@ struct choco_ctx {
     unsigned long long launches;
     // optional event pairs around the update kernel
     cudaEvent_t* prof_ev;
-    int prof_cap, prof_n;
+    int prof_cap, prof_n, prof_stride;
     // all device allocations, for choco_destroy
     void* allocs[64];
     int nallocs;

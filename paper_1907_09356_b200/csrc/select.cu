@@ -432,6 +432,8 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t sm[64];
     __shared__ uint32_t s_carry[2];
+    wait_for_previous_kernel(); // the candidates come from the kernel before this one
+    allow_next_kernel();
     const int row = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ncand = dv.row_count[row];
@@ -634,7 +636,9 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaS
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev][a.vec ? 1 : 0] = true;
     }
-    kern<<<dv.n, kSelThreads, (size_t)dv.emit_smem_bytes, st>>>(dv, a, fused ? 1 : 0);
+    e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st, dv, a,
+                          fused ? 1 : 0);
+    if (e != cudaSuccess) return e;
     *a.launches += 1;
     return cudaGetLastError();
 }

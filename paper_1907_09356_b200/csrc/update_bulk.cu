@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     uint32_t* s_base = reinterpret_cast<uint32_t*>(scan) + 2 * (NT / 32 + 1);
     NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
 
+    wait_for_previous_kernel(); // messages and range records come from the kernel before this one
+    allow_next_kernel();
     const int row = blockIdx.y;
     const int64_t tile = blockIdx.x;
     const int64_t c0 = tile * kTile;
@@ -357,8 +359,7 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
-    update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT><<<grid, NT, smem, st>>>(dv, a);
-    return cudaSuccess;
+    return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT>, grid, dim3(NT), smem, st, dv, a);
 }
 
 } // namespace
