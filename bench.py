@@ -30,6 +30,9 @@ import workloads  # noqa: E402
 L2_BYTES = 126 * 2 ** 20
 NOMINAL_HBM_GBS = 8000.0           # the figure the 60 % target is quoted against
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, from the ncu
+# capture summarised under profiles/ (None for workloads that were not captured)
+NCU_TRAFFIC = {("c4_torus64_topk", "update"): 1.365e9}
 
 
 def measured_peak():
@@ -319,7 +322,8 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "update (apply) kernel", "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None,
-                         "traffic": None, "algorithmic_bytes_per_launch": upd_bytes,
+                         "traffic": NCU_TRAFFIC.get((wl.name, "update")),
+                         "algorithmic_bytes_per_launch": upd_bytes,
                          "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec,
                          "timed_every": args.profile_stride},
             "gpu_launches": int(st1["kernel_launches"] - st0["kernel_launches"]),
