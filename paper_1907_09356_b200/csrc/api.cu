@@ -116,7 +116,14 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     if (!aligned4(X) || !aligned4(Xhat) || !aligned4(S) || !aligned4(G) || !aligned4(M))
         return CHOCO_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
-    const Dev& dv = ctx->dv;
+    Dev dv = ctx->dv; // by value: the dense message buffers are swapped per step
+    {
+        const choco_ctx::DenseBuf &cur = ctx->dbuf[ctx->msg_cur], &nxt = ctx->dbuf[ctx->msg_cur ^ 1];
+        dv.msg_bits = cur.bits; dv.msg_scale = cur.scale; dv.msg_norms = cur.norms;
+        dv.msg_levels = cur.levels; dv.msg_dense = cur.dense;
+        dv.nxt_bits = nxt.bits; dv.nxt_scale = nxt.scale; dv.nxt_norms = nxt.norms;
+        dv.nxt_levels = nxt.levels; dv.nxt_dense = nxt.dense;
+    }
     StepArgs a;
     a.X = X; a.Xhat = Xhat; a.S = S; a.G = G; a.M = M;
     a.eta = eta; a.gamma = gamma; a.lambda = lambda; a.beta = beta;
@@ -133,7 +140,7 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     if (sparse) {
         if (!was_prepared) e = launch_select_prepare(dv, a, st);
         if (e == cudaSuccess) e = launch_select_emit(dv, a, was_prepared, st);
-    } else {
+    } else if (!was_prepared) {
         e = launch_compress_dense(dv, a, st);
     }
     // the update kernel can collect the next step's candidates from the x' - x^' it holds
@@ -146,7 +153,13 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
         e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], st);
         ctx->prof_n += 1;
     }
+    if (e == cudaSuccess && emit && dv.kind == CHOCO_Q_SIGN) {
+        e = launch_next_sign_scale(dv, st);
+        ctx->launches += 1;
+    }
     if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->msg_last = ctx->msg_cur;
+    if (emit && !sparse) ctx->msg_cur ^= 1; // the next step's messages sit in the other buffer
     ctx->prepared = emit;
     ctx->last_x = X;
     ctx->last_xhat = Xhat;
@@ -292,8 +305,10 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         ctx->msg_bytes_per_worker = (p->kind == CHOCO_Q_TOPK ? 8 : 4) * p->k;
     } else if (p->kind == CHOCO_Q_SIGN) {
         dv.wpitch = round_up(nwords, 4);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_bits, n * dv.wpitch);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_scale, n);
+        for (int b = 0; b < 2; ++b) {
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].bits, n * dv.wpitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].scale, n);
+        }
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial, n * dv.nchunks);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial2, n * dv.nchunks);
         ctx->msg_bytes_per_worker = 4 * nwords + 4;
@@ -306,20 +321,26 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         const int64_t blen = p->bucket > 0 ? p->bucket : d;
         dv.nbuckets = (d + blen - 1) / blen;
         dv.npitch = round_up(dv.nbuckets, 4);
+        dv.bucket_shift = 0;
+        while (p->bucket > 0 && (1 << dv.bucket_shift) < p->bucket) ++dv.bucket_shift;
+        dv.tail_bucket = (p->bucket > 0 && d % blen != 0) ? dv.nbuckets - 1 : -1;
         dv.tau_full = qsgd_tau(blen, p->s, p->qsgd_biased != 0);
         dv.tau_tail = qsgd_tau(d % blen ? d % blen : blen, p->s, p->qsgd_biased != 0);
         dv.wpitch = round_up(nwords, 4);
         const int64_t lbytes = (d * w + 7) / 8;
         dv.lpitch = round_up(lbytes, 16) + 16;
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_bits, n * dv.wpitch);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_norms, n * dv.npitch);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_levels, n * dv.lpitch);
+        for (int b = 0; b < 2; ++b) {
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].bits, n * dv.wpitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].norms, n * dv.npitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].levels, n * dv.lpitch);
+        }
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial, n * dv.nchunks);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.partial2, n * dv.nchunks);
         ctx->msg_bytes_per_worker = 4 * dv.nbuckets + 4 * nwords + lbytes;
     } else {
         dv.dpitch = round_up(d, 4);
-        if (e == cudaSuccess) e = dev_alloc(ctx, &dv.msg_dense, n * dv.dpitch);
+        for (int b = 0; b < 2; ++b)
+            if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->dbuf[b].dense, n * dv.dpitch);
         ctx->msg_bytes_per_worker = 4 * d;
     }
     ctx->cons_blocks = (d + 255) / 256;
@@ -449,7 +470,12 @@ int choco_get_message(const choco_ctx* ctx, int32_t worker, int32_t plane, const
 {
     if (!ctx || !dev_ptr || !nbytes || worker < 0 || worker >= ctx->dv.n || plane < 0 || plane > 2)
         return CHOCO_ERR_INVALID_ARG;
-    const Dev& dv = ctx->dv;
+    Dev dv = ctx->dv;
+    {
+        const choco_ctx::DenseBuf& last = ctx->dbuf[ctx->msg_last];
+        dv.msg_bits = last.bits; dv.msg_scale = last.scale; dv.msg_norms = last.norms;
+        dv.msg_levels = last.levels; dv.msg_dense = last.dense;
+    }
     const int64_t nwords = (dv.d + 31) / 32;
     *dev_ptr = nullptr;
     *nbytes = 0;

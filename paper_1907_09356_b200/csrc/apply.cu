@@ -27,88 +27,6 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
 }
 
 // ---------------------------------------------------------------------------------------
-// dense Q: decode each neighbour's message on the fly
-// ---------------------------------------------------------------------------------------
-template <int KIND>
-__device__ __forceinline__ float4 decode_quad(const Dev& dv, int j, int64_t c)
-{
-    if (KIND == CHOCO_Q_IDENTITY)
-        return __ldg(reinterpret_cast<const float4*>(dv.msg_dense + (int64_t)j * dv.dpitch + c));
-    const uint32_t word = __ldg(dv.msg_bits + (int64_t)j * dv.wpitch + (c >> 5));
-    const uint32_t nib = (word >> (c & 31)) & 0xFu;
-    float m[4];
-    if (KIND == CHOCO_Q_SIGN) {
-        const float sc = __ldg(dv.msg_scale + j);
-        m[0] = m[1] = m[2] = m[3] = sc;
-    } else {
-        const int64_t b = dv.bucket > 0 ? c / dv.bucket : 0;
-        const float nu = __ldg(dv.msg_norms + (int64_t)j * dv.npitch + b);
-        const bool tail = dv.bucket > 0 && b == dv.nbuckets - 1 && (dv.d % dv.bucket) != 0;
-        const float scale = __fdiv_rn(nu, __fmul_rn(tail ? dv.tau_tail : dv.tau_full, (float)dv.s));
-        const uint8_t* lrow = dv.msg_levels + (int64_t)j * dv.lpitch;
-        uint32_t packed, width = (uint32_t)dv.wbits;
-        if (width == 8) packed = __ldg(reinterpret_cast<const uint32_t*>(lrow + c));
-        else if (width == 4) packed = __ldg(reinterpret_cast<const uint16_t*>(lrow + (c >> 1)));
-        else if (width == 2) packed = __ldg(lrow + (c >> 2));
-        else packed = (__ldg(lrow + (c >> 3)) >> (c & 7)) & 0xFu;
-        const uint32_t mask = (1u << width) - 1u;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) m[e] = __fmul_rn(scale, (float)((packed >> (e * width)) & mask));
-    }
-    return make_float4(nib & 1u ? -m[0] : m[0], nib & 2u ? -m[1] : m[1], nib & 4u ? -m[2] : m[2],
-                       nib & 8u ? -m[3] : m[3]);
-}
-
-template <bool VEC, int KIND, bool HAS_G, bool HAS_M>
-__global__ void __launch_bounds__(kThreads) apply_dense_kernel(Dev dv, StepArgs a)
-{
-    const int row = blockIdx.y;
-    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
-    const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
-    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
-    float* xr = a.X + (int64_t)row * dv.ld;
-    float* hr = a.Xhat + (int64_t)row * dv.ld;
-    float* sr = a.S + (int64_t)row * dv.ld;
-    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld : nullptr;
-    float* mr = HAS_M ? a.M + (int64_t)row * dv.ld : nullptr;
-#pragma unroll
-    for (int it = 0; it < kDenseIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
-        if (c >= dv.d) continue;
-        const float4 x = load_quad<VEC>(xr, c, dv.d);
-        const float4 h = load_quad<VEC>(hr, c, dv.d);
-        const float4 s = load_quad<VEC>(sr, c, dv.d);
-        float4 g = make_float4(0.f, 0.f, 0.f, 0.f), m = g;
-        if (HAS_G) g = load_quad_stream<VEC>(gr, c, dv.d);
-        if (HAS_M) m = load_quad<VEC>(mr, c, dv.d);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), qs = acc;
-        for (int e = e0; e < e1; ++e) {
-            const int j = dv.col[e];
-            const float w = dv.wval[e];
-            const float4 q = decode_quad<KIND>(dv, j, c);
-            acc.x = __fadd_rn(acc.x, __fmul_rn(w, q.x));
-            acc.y = __fadd_rn(acc.y, __fmul_rn(w, q.y));
-            acc.z = __fadd_rn(acc.z, __fmul_rn(w, q.z));
-            acc.w = __fadd_rn(acc.w, __fmul_rn(w, q.w));
-            if (j == row) qs = q;
-        }
-        const float4 hn = make_float4(__fadd_rn(h.x, qs.x), __fadd_rn(h.y, qs.y),
-                                      __fadd_rn(h.z, qs.z), __fadd_rn(h.w, qs.w));
-        const float4 sn = make_float4(__fadd_rn(s.x, acc.x), __fadd_rn(s.y, acc.y),
-                                      __fadd_rn(s.z, acc.z), __fadd_rn(s.w, acc.w));
-        float4 xn;
-        xn.x = next_x<HAS_G, HAS_M>(x.x, sn.x, hn.x, g.x, m.x, u);
-        xn.y = next_x<HAS_G, HAS_M>(x.y, sn.y, hn.y, g.y, m.y, u);
-        xn.z = next_x<HAS_G, HAS_M>(x.z, sn.z, hn.z, g.z, m.z, u);
-        xn.w = next_x<HAS_G, HAS_M>(x.w, sn.w, hn.w, g.w, m.w, u);
-        store_quad<VEC>(hr, c, dv.d, hn);
-        store_quad<VEC>(sr, c, dv.d, sn);
-        store_quad<VEC>(xr, c, dv.d, xn);
-        if (HAS_M) store_quad<VEC>(mr, c, dv.d, m);
-    }
-}
-
-// ---------------------------------------------------------------------------------------
 // sparse Q, register-staged variant (any alignment, any d): the neighbours' (index, value)
 // lists are scattered into a shared-memory tile, one neighbour after the other so that the
 // additions happen in CSR order, then the tile is streamed against x, x^, s and g.  x^ and s
@@ -211,22 +129,14 @@ template <bool VEC, bool HAS_G, bool HAS_M>
 static cudaError_t apply_pick(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);  // sparse: one block per tile
-    const dim3 dgrid((unsigned)dv.nspans, (unsigned)dv.n); // dense: one block per span
     switch (dv.kind) {
     case CHOCO_Q_TOPK:
     case CHOCO_Q_RANDK:
         if (update_bulk_usable(dv, a)) return launch_update_bulk(dv, a, emit, st);
         apply_sparse_kernel<VEC, HAS_G, HAS_M><<<grid, kTileThreads, 0, st>>>(dv, a);
         break;
-    case CHOCO_Q_SIGN:
-        apply_dense_kernel<VEC, CHOCO_Q_SIGN, HAS_G, HAS_M><<<dgrid, kThreads, 0, st>>>(dv, a);
-        break;
-    case CHOCO_Q_QSGD:
-        apply_dense_kernel<VEC, CHOCO_Q_QSGD, HAS_G, HAS_M><<<dgrid, kThreads, 0, st>>>(dv, a);
-        break;
     default:
-        apply_dense_kernel<VEC, CHOCO_Q_IDENTITY, HAS_G, HAS_M><<<dgrid, kThreads, 0, st>>>(dv, a);
-        break;
+        return launch_update_dense(dv, a, emit, st);
     }
     return cudaSuccess;
 }
@@ -241,7 +151,9 @@ static cudaError_t apply_vec(const Dev& dv, const StepArgs& a, bool emit, cudaSt
 
 bool apply_can_emit(const Dev& dv, const StepArgs& a)
 {
-    return dv.kind == CHOCO_Q_TOPK && update_bulk_usable(dv, a);
+    if (dv.kind == CHOCO_Q_TOPK) return update_bulk_usable(dv, a);
+    if (dv.kind == CHOCO_Q_RANDK) return false;
+    return update_dense_can_emit(dv);
 }
 
 cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)

@@ -232,6 +232,14 @@ static cudaError_t compress_impl(const Dev& dv, const StepArgs& a, cudaStream_t 
     return cudaGetLastError();
 }
 
+cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st)
+{
+    Dev dn = dv;
+    dn.msg_scale = dv.nxt_scale;
+    norm_finish_kernel<NORM_L1><<<dv.n, 1024, 0, st>>>(dn);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
     return a.vec ? compress_impl<true>(dv, a, st) : compress_impl<false>(dv, a, st);

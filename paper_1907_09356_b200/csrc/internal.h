@@ -83,10 +83,19 @@ struct Dev {
     uint8_t* msg_levels;         // qsgd: [n, lpitch]
     int64_t dpitch;              // identity: floats per row of msg_dense
     float* msg_dense;            // identity: [n, dpitch]
+    // the other message buffer of the dense operators: the update kernel writes the next
+    // step's messages there while it reads this step's from msg_* (the host swaps them)
+    uint32_t* nxt_bits;
+    float* nxt_scale;
+    float* nxt_norms;
+    uint8_t* nxt_levels;
+    float* nxt_dense;
     // qsgd parameters
     int32_t s;
     int32_t bucket;              // 0 = whole row
     int32_t wbits;               // level field width
+    int32_t bucket_shift;        // log2(bucket) when bucket > 0
+    int64_t tail_bucket;         // index of the ragged last block, or -1 if the last one is full
     float tau_full;              // tau of a full block (or of the whole row)
     float tau_tail;              // tau of the ragged last block
     // norm workspace
@@ -116,6 +125,10 @@ cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t
 bool apply_can_emit(const Dev& dv, const StepArgs& a);
 bool update_bulk_usable(const Dev& dv, const StepArgs& a);
 cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
+bool update_dense_can_emit(const Dev& dv);
+cudaError_t launch_update_dense(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
+// sign: finish the tree over the partial sums the update kernel left and set nxt_scale
+cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st);
 cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 // metrics
 cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,
@@ -135,6 +148,10 @@ struct choco_ctx {
     const float* last_x;
     const float* last_xhat;
     int64_t msg_bytes_per_worker;
+    // dense operators: two sets of message buffers; msg_cur is read by the next update
+    // kernel, msg_last holds the message applied most recently (choco_get_message)
+    struct DenseBuf { uint32_t* bits; float* scale; float* norms; uint8_t* levels; float* dense; } dbuf[2];
+    int msg_cur, msg_last;
     // arena that steps ask the L2 cache to keep resident (messages, records, candidates)
     void* hot_base;
     int64_t hot_bytes;
