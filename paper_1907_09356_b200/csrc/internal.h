@@ -127,6 +127,8 @@ bool update_bulk_usable(const Dev& dv, const StepArgs& a);
 cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 bool update_dense_can_emit(const Dev& dv);
 cudaError_t launch_update_dense(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
+bool update_dense_bulk_usable(const Dev& dv, const StepArgs& a);
+cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 // sign: finish the tree over the partial sums the update kernel left and set nxt_scale
 cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st);
 cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);

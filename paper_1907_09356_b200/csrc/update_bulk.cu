@@ -10,6 +10,7 @@
 // into the tile (a second one), and adds them into a shared accumulator tile neighbour by
 // neighbour.  With EMIT the kernel also collects the candidates of the next step's top-k
 // selection from x' - x^', which it holds anyway.
+#include "bulk.cuh"
 #include "select.cuh"
 
 namespace choco {
@@ -32,54 +33,6 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
         xn = __fsub_rn(x, __fmul_rn(u.eta, g));
     }
     return __fadd_rn(xn, __fmul_rn(u.gamma, cons));
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-                 : "memory");
-}
-// global -> this block's shared memory; both addresses 16-byte aligned, bytes % 16 == 0
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok)
-                 : "r"(smem_u32(bar)), "r"(parity)
-                 : "memory");
-    return ok != 0;
-}
-// Wait for phase `parity` with a bound: after kSpinLimit polls the wait is recorded as timed
-// out; the copies in flight are then given a second bounded grace period so that the block
-// does not retire under them.  Returns false on a timeout.
-constexpr uint32_t kSpinLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, Stats* stats)
-{
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    if ((threadIdx.x & 31) == 0) atomicAdd(&stats->timeouts, 1ull);
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) break;
-        __nanosleep(256);
-    }
-    return false;
 }
 
 constexpr int NT = kTileThreads;

@@ -242,6 +242,7 @@ bool update_dense_can_emit(const Dev& dv)
 
 cudaError_t launch_update_dense(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {
+    if (update_dense_bulk_usable(dv, a)) return launch_update_dense_bulk(dv, a, emit, st);
     if (a.vec) { if (emit) pick_terms<true, true>(dv, a, st); else pick_terms<true, false>(dv, a, st); }
     else { if (emit) pick_terms<false, true>(dv, a, st); else pick_terms<false, false>(dv, a, st); }
     return cudaGetLastError();
