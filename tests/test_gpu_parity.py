@@ -188,6 +188,33 @@ def test_topk_carry_across_steps():
     ch2.close()
 
 
+@pytest.mark.parametrize("kind,kw", [("sign", {}), ("qsgd", dict(s=16, bucket=512)), ("identity", {})])
+def test_dense_carry_across_steps(kind, kw):
+    """For dense operators the update kernel writes the next step's messages; switching that
+    off (every step compresses from X and Xhat again) must give the same state."""
+    w = workloads.ring(6)
+    n, d, steps = 6, 30000, 6
+    X0 = workloads.normal_rows(n, d, 1.0, 31)
+    G = [_dev(workloads.normal_rows(n, d, 0.01, 700 + t)) for t in range(steps)]
+    out = []
+    for carry in (True, False):
+        ch = choco.Choco(w, d, kind, seed=4, **kw)
+        choco.choco_set_carry(ch.ctx, carry)
+        st = [_dev(X0), torch.zeros(n, d, device=DEV), torch.zeros(n, d, device=DEV)]
+        for t in range(steps):
+            ch.sgd_step(st[0], st[1], st[2], G[t], 0.05, 0.2)
+            if t == 2:      # an external change of X in the middle, announced to the library
+                st[0].mul_(1.5)
+                choco.choco_invalidate(ch.ctx)
+        torch.cuda.synchronize()
+        launches = choco.choco_get_stats(ch.ctx)["kernel_launches"]
+        out.append((st, launches))
+        ch.close()
+    for a, b in zip(out[0][0], out[1][0]):
+        assert torch.equal(a, b)
+    assert out[0][1] < out[1][1]     # carrying saves the separate compression kernels
+
+
 def test_invalidate_after_external_change():
     w = workloads.ring(4)
     n, d, k = 4, 20000, 200
