@@ -455,12 +455,13 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     else { slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch; }
     if (dv.emit_tiles_smem) { t_gt = cursor; t_eq = cursor + dv.ntiles; t_sbe = cursor + 2 * dv.ntiles; cursor += 3 * dv.ntiles; }
     else { t_gt = dv.tile_a + (int64_t)row * dv.ntiles; t_eq = dv.tile_b + (int64_t)row * dv.ntiles; t_sbe = dv.tile_c + (int64_t)row * dv.ntiles; }
-    uint32_t* sbits = cursor; // the candidates' value bits, when they fit
+    uint32_t* sbits = cursor;                      // the candidates' value bits and
+    uint32_t* sidx = cursor + dv.emit_keys_cap;    // coordinates, when they fit
     const bool cached = ncand <= (uint32_t)dv.emit_keys_cap;
     uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
     for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
         const uint32_t bits = __ldg(cv + p);
-        if (cached) sbits[p] = bits;
+        if (cached) { sbits[p] = bits; sidx[p] = __ldg(ci + p); }
         const uint32_t kk = order_key<KIND>(bits);
         klo = kk < klo ? kk : klo;
         khi = kk > khi ? kk : khi;
@@ -468,6 +469,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
     block_min_max(klo, khi, sm);
     auto bits_at = [&](uint32_t p) -> uint32_t { return cached ? sbits[p] : __ldg(cv + p); };
+    auto idx_at = [&](uint32_t p) -> uint32_t { return cached ? sidx[p] : __ldg(ci + p); };
     auto key_at = [&](uint32_t p) -> uint32_t { return order_key<KIND>(bits_at(p)); };
 
     uint32_t T, above;
@@ -496,7 +498,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         for (int u = 0; u < kBatch; ++u) {
             const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
             const uint32_t p = (uint32_t)(sl << 5) + lane;
-            idx[u] = (sl < nslab && p < ncand) ? __ldg(ci + p) : 0u;
+            idx[u] = (sl < nslab && p < ncand) ? idx_at(p) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
@@ -555,7 +557,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         for (int u = 0; u < kBatch; ++u) {
             const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
             const uint32_t p = (uint32_t)(sl << 5) + lane;
-            idx[u] = (sl < nslab && p < ncand) ? __ldg(ci + p) : 0u;
+            idx[u] = (sl < nslab && p < ncand) ? idx_at(p) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
