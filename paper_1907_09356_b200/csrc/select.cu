@@ -458,13 +458,33 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     uint32_t* sbits = cursor;                      // the candidates' value bits and
     uint32_t* sidx = cursor + dv.emit_keys_cap;    // coordinates, when they fit
     const bool cached = ncand <= (uint32_t)dv.emit_keys_cap;
+    // a thread's own tile segment, fetched now so that the wait overlaps the copy below
+    const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
+    const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
+    const bool own_tile = dv.ntiles <= kSelThreads;
+    uint32_t my_so = 0u, my_sc = 0u;
+    if (own_tile && threadIdx.x < dv.ntiles) { my_so = __ldg(so + threadIdx.x); my_sc = __ldg(sc + threadIdx.x); }
     uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
-    for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
-        const uint32_t bits = __ldg(cv + p);
-        if (cached) { sbits[p] = bits; sidx[p] = __ldg(ci + p); }
-        const uint32_t kk = order_key<KIND>(bits);
-        klo = kk < klo ? kk : klo;
-        khi = kk > khi ? kk : khi;
+    for (uint32_t p0 = threadIdx.x; p0 < ncand; p0 += 4 * kSelThreads) {
+        uint32_t bits[4], idx[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t p = p0 + j * kSelThreads;
+            if (p < ncand) {
+                bits[j] = __ldg(cv + p);
+                if (cached) idx[j] = __ldg(ci + p);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t p = p0 + j * kSelThreads;
+            if (p < ncand) {
+                if (cached) { sbits[p] = bits[j]; sidx[p] = idx[j]; }
+                const uint32_t kk = order_key<KIND>(bits[j]);
+                klo = kk < klo ? kk : klo;
+                khi = kk > khi ? kk : khi;
+            }
+        }
     }
     for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
     block_min_max(klo, khi, sm);
@@ -523,15 +543,13 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     block_scan_pair(t_gt, t_eq, dv.ntiles, sm, s_carry, &tot_a, &tot_b);
     block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_a, &tot_b);
     uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
-    const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
-    const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
     for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
         const uint32_t gb = t_gt[t], eb = t_eq[t];
         tp[t] = gb + (eb < r ? eb : r);
         // the two flat prefixes at the tile's first candidate: t_gt <- above, t_sbe <- equal
         uint32_t pg = 0, pe = 0;
-        if (sc[t]) {
-            const uint32_t first = so[t], s0 = first >> 5;
+        if (own_tile ? my_sc : sc[t]) {
+            const uint32_t first = own_tile ? my_so : so[t], s0 = first >> 5;
             pg = slab_g[s0];
             pe = slab_e[s0];
             for (uint32_t p = s0 << 5; p < first; ++p) {
