@@ -178,6 +178,20 @@ def rows_for_budget(wl) -> int:
 # ------------------------------------------------------------------------------------------
 
 
+def max_over_ranks(values, device):
+    """The slowest rank's figure for each entry: every replica must have finished."""
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return [float(v) for v in tt]
+
+
+def whole_job_rate(world: int, coords_per_replica_step: int, steps: int, seconds: float) -> float:
+    """Coordinates per second over all replicas: each of `world` ranks ran `steps` steps."""
+    return world * coords_per_replica_step * steps / seconds
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -294,16 +308,14 @@ def main():
         e2e = {"seconds": e2e_s, "steps": args.e2e_steps}
 
     if world > 1:
-        tt = torch.tensor([ms, e2e["seconds"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt[0]);
+        ms, e2e_s = max_over_ranks([ms, e2e["seconds"] if e2e else 0.0], dev)
         if e2e:
-            e2e["seconds"] = float(tt[1])
+            e2e["seconds"] = e2e_s
 
     if rank == 0:
         peak, peak_src = measured_peak()
         ms_step = ms / args.steps
-        value = world * N * args.steps / (ms * 1e-3)
+        value = whole_job_rate(world, N, args.steps, ms * 1e-3)
         upd_bytes = update_kernel_bytes(wl, w)
         upd_avg_s = (upd_ms / max(nrec, 1)) * 1e-3
         achieved = upd_bytes / upd_avg_s / 1e9 if nrec else None
@@ -332,7 +344,7 @@ def main():
             "clocks": clocks,
         }
         if e2e:
-            out["e2e"] = {"value": world * N * e2e["steps"] / e2e["seconds"], "unit": "coords/s",
+            out["e2e"] = {"value": whole_job_rate(world, N, e2e["steps"], e2e["seconds"]), "unit": "coords/s",
                           "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,
                           "steps": e2e["steps"], "api": "choco_sgd_step_host, pinned host buffers"}
         if not args.no_cpu_baseline and world == 1:
