@@ -81,8 +81,6 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     uint32_t* s_base = reinterpret_cast<uint32_t*>(scan) + 2 * (NT / 32 + 1);
     NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
 
-    wait_for_previous_kernel(); // messages and range records come from the kernel before this one
-    allow_next_kernel();
     const int row = blockIdx.y;
     const int64_t tile = blockIdx.x;
     const int64_t c0 = tile * kTile;
@@ -103,14 +101,20 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
         if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, bytes, bar);
         if (HAS_M) bulk_load(ms, a.M + (int64_t)row * dv.ld + c0, bytes, bar);
     }
-    const uint32_t lo_key = EMIT ? __ldg(dv.row_lo + row) : 0u; // used at the end: fetch early
-    // warp 1 builds the neighbour table of the first batch while the others clear the tile
-    uint4 rc = make_uint4(0u, 0u, 0u, 0u);
-    if ((threadIdx.x >> 5) == 1 && lane < dv.maxdeg) rc = __ldg(recs + lane);
 #pragma unroll
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (threadIdx.x < kTile / 32) { touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; }
+    // Messages, range records and the candidate bound come from the kernel before this one.
+    // The dense arrays requested above do not: the kernel before either ran to completion
+    // before this one started, or is the emit kernel, which lets its successor start only
+    // after it has itself seen the previous update complete.
+    wait_for_previous_kernel();
+    allow_next_kernel();
+    const uint32_t lo_key = EMIT ? __ldg(dv.row_lo + row) : 0u; // used at the end: fetch early
+    // warp 1 builds the neighbour table of the first batch
+    uint4 rc = make_uint4(0u, 0u, 0u, 0u);
+    if ((threadIdx.x >> 5) == 1 && lane < dv.maxdeg) rc = __ldg(recs + lane);
 
     bool self_in_regs = false;  // this worker's own entries are held by threads (er == self)
     uint32_t self_lo = 0, self_len = 0;

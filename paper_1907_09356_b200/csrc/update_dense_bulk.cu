@@ -33,23 +33,21 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
     return __fadd_rn(xn, __fmul_rn(u.gamma, cons));
 }
 
-// the pieces of worker j's message that cover coordinates [c, c+4)
+// The pieces of worker j's message that cover coordinates [c, c+4): the quad's four sign
+// bits and (gsgd_b) its packed level fields.  The magnitude that goes with them -- the row's
+// scale, or norm / (tau s) of the block -- is the same for many quads and is kept apart.
 struct Piece {
-    uint32_t word;   // sign plane word holding the quad's bits
-    uint32_t packed; // the quad's level fields (gsgd_b)
-    float mag;       // sign: the scale; gsgd_b: the block norm
+    uint32_t nib;    // bit e: coordinate c + e is negative
+    uint32_t packed; // level fields, wbits each (gsgd_b)
 };
 
 template <int KIND>
 __device__ __forceinline__ Piece load_piece(const Dev& dv, int j, int64_t c)
 {
     Piece p;
-    p.word = __ldg(dv.msg_bits + (int64_t)j * dv.wpitch + (c >> 5));
+    p.nib = __ldg(dv.msg_bits + (int64_t)j * dv.wpitch + (c >> 5));
     p.packed = 0u;
-    if (KIND == CHOCO_Q_SIGN) {
-        p.mag = __ldg(dv.msg_scale + j);
-    } else {
-        p.mag = __ldg(dv.msg_norms + (int64_t)j * dv.npitch + (c >> dv.bucket_shift));
+    if (KIND == CHOCO_Q_QSGD) {
         const uint8_t* lrow = dv.msg_levels + (int64_t)j * dv.lpitch;
         const uint32_t width = (uint32_t)dv.wbits;
         if (width == 8) p.packed = __ldg(reinterpret_cast<const uint32_t*>(lrow + c));
@@ -60,22 +58,41 @@ __device__ __forceinline__ Piece load_piece(const Dev& dv, int j, int64_t c)
     return p;
 }
 
+// magnitude shared by the coordinates of one block of worker j's message
 template <int KIND>
-__device__ __forceinline__ float4 decode_piece(const Dev& dv, const Piece& p, int64_t c)
+__device__ __forceinline__ float load_mag(const Dev& dv, int j, int64_t bucket)
 {
-    const uint32_t nib = (p.word >> (c & 31)) & 0xFu;
+    if (KIND == CHOCO_Q_SIGN) return __ldg(dv.msg_scale + j);
+    const float nu = __ldg(dv.msg_norms + (int64_t)j * dv.npitch + bucket);
+    return __fdiv_rn(nu, __fmul_rn(bucket == dv.tail_bucket ? dv.tau_tail : dv.tau_full, (float)dv.s));
+}
+
+// small non-negative integer -> float without the conversion unit: exact below 2^23
+__device__ __forceinline__ float small_uint_to_float(uint32_t v)
+{
+    return __fsub_rn(__uint_as_float(0x4B000000u | v), 8388608.f);
+}
+
+// mag is >= 0, so setting the sign bit negates it
+__device__ __forceinline__ float with_sign(float mag, uint32_t nib, int e)
+{
+    return __uint_as_float(__float_as_uint(mag) | ((nib << (31 - e)) & 0x80000000u));
+}
+
+template <int KIND>
+__device__ __forceinline__ float4 decode_piece(const Dev& dv, const Piece& pp, float mag, int64_t c)
+{
+    Piece p = pp; p.nib = (pp.nib >> (c & 31)) & 0xFu;
     float m[4];
     if (KIND == CHOCO_Q_SIGN) {
-        m[0] = m[1] = m[2] = m[3] = p.mag;
+        m[0] = m[1] = m[2] = m[3] = mag;
     } else {
-        const bool tail = (c >> dv.bucket_shift) == dv.tail_bucket;
-        const float scale = __fdiv_rn(p.mag, __fmul_rn(tail ? dv.tau_tail : dv.tau_full, (float)dv.s));
         const uint32_t width = (uint32_t)dv.wbits, mask = (1u << width) - 1u;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) m[e] = __fmul_rn(scale, (float)((p.packed >> (e * width)) & mask));
+        for (int e = 0; e < 4; ++e) m[e] = __fmul_rn(mag, small_uint_to_float((p.packed >> (e * width)) & mask));
     }
-    return make_float4(nib & 1u ? -m[0] : m[0], nib & 2u ? -m[1] : m[1], nib & 4u ? -m[2] : m[2],
-                       nib & 8u ? -m[3] : m[3]);
+    return make_float4(with_sign(m[0], p.nib, 0), with_sign(m[1], p.nib, 1), with_sign(m[2], p.nib, 2),
+                       with_sign(m[3], p.nib, 3));
 }
 
 __device__ __forceinline__ uint32_t sign_nibble4(const float4& v)
@@ -123,14 +140,16 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     // message pieces of the first kPre neighbours, fetched while the tiles are in flight
     Piece pre[NIT][kPre];
     int prej[kPre];
-    float prew[kPre];
+    float prew[kPre], pmag[kPre];
 #pragma unroll
     for (int q = 0; q < kPre; ++q) {
         prej[q] = -1;
         prew[q] = 0.f;
+        pmag[q] = 0.f;
         if (e0 + q < e1) {
             prej[q] = dv.col[e0 + q];
             prew[q] = dv.wval[e0 + q];
+            if (KIND == CHOCO_Q_SIGN) pmag[q] = load_mag<KIND>(dv, prej[q], 0);
         }
     }
 #pragma unroll
@@ -138,8 +157,23 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         const int li = (it * NT + threadIdx.x) * kQuad;
 #pragma unroll
         for (int q = 0; q < kPre; ++q) {
-            pre[it][q].word = 0u; pre[it][q].packed = 0u; pre[it][q].mag = 0.f;
+            pre[it][q].nib = 0u; pre[it][q].packed = 0u;
             if (prej[q] >= 0 && li < nvalid) pre[it][q] = load_piece<KIND>(dv, prej[q], c0 + li);
+        }
+    }
+    // gsgd_b: the 128 coordinates of a warp's quads lie in one block, so lane q fetches the
+    // norm of neighbour q's block and the warp shares norm / (tau s) by shuffles later
+    float nraw[NIT];
+    bool ntail[NIT];
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        nraw[it] = 0.f;
+        ntail[it] = false;
+        if (KIND == CHOCO_Q_QSGD) {
+            const int64_t bucket = (c0 + (int64_t)(it * NT + warp * 32) * kQuad) >> dv.bucket_shift;
+            ntail[it] = bucket == dv.tail_bucket;
+            if (lane < kPre && e0 + lane < e1 && bucket < dv.nbuckets)
+                nraw[it] = __ldg(dv.msg_norms + (int64_t)dv.col[e0 + lane] * dv.npitch + bucket);
         }
     }
     // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
@@ -156,6 +190,13 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         const int li = q4 * kQuad;
         const int64_t c = c0 + li;
         vn[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float lane_mag = 0.f; // lane q: norm / (tau s) of neighbour q's block
+        if (KIND == CHOCO_Q_QSGD)
+            lane_mag = __fdiv_rn(nraw[it], __fmul_rn(ntail[it] ? dv.tau_tail : dv.tau_full, (float)dv.s));
+        float qmag[kPre];
+#pragma unroll
+        for (int q = 0; q < kPre; ++q)
+            qmag[q] = KIND == CHOCO_Q_SIGN ? pmag[q] : __shfl_sync(0xffffffffu, lane_mag, q);
         if (li < nvalid) {
             const float4 x = reinterpret_cast<const float4*>(xs)[q4];
             const float4 h = reinterpret_cast<const float4*>(hs)[q4];
@@ -167,7 +208,7 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
 #pragma unroll
             for (int q = 0; q < kPre; ++q) {
                 if (prej[q] < 0) continue;
-                const float4 qv = decode_piece<KIND>(dv, pre[it][q], c);
+                const float4 qv = decode_piece<KIND>(dv, pre[it][q], qmag[q], c);
                 acc.x = __fadd_rn(acc.x, __fmul_rn(prew[q], qv.x));
                 acc.y = __fadd_rn(acc.y, __fmul_rn(prew[q], qv.y));
                 acc.z = __fadd_rn(acc.z, __fmul_rn(prew[q], qv.z));
@@ -178,7 +219,7 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
                 const int j = dv.col[e];
                 const float w = dv.wval[e];
                 const Piece p = load_piece<KIND>(dv, j, c);
-                const float4 qv = decode_piece<KIND>(dv, p, c);
+                const float4 qv = decode_piece<KIND>(dv, p, load_mag<KIND>(dv, j, c >> dv.bucket_shift), c);
                 acc.x = __fadd_rn(acc.x, __fmul_rn(w, qv.x));
                 acc.y = __fadd_rn(acc.y, __fmul_rn(w, qv.y));
                 acc.z = __fadd_rn(acc.z, __fmul_rn(w, qv.z));
@@ -246,16 +287,14 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         const uint4 rw = coord_words(dv.seed, a.step + 1, (uint32_t)row, kStreamDither, c);
         const float uu[4] = {word_to_unit(rw.x), word_to_unit(rw.y), word_to_unit(rw.z), word_to_unit(rw.w)};
         const float vv[4] = {vn[it].x, vn[it].y, vn[it].z, vn[it].w};
-        uint32_t lev[4];
+        uint32_t lev[4] = {0u, 0u, 0u, 0u};
+        if (nu != 0.f) { // the same for every lane of the warp
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            int l = 0;
-            if (nu != 0.f) {
+            for (int e = 0; e < 4; ++e) {
                 const float r = __fdiv_rn(__fmul_rn(sf, fabsf(vv[e])), nu);
-                l = (int)floorf(__fadd_rn(r, uu[e]));
-                l = l > dv.s - 1 ? dv.s - 1 : l;
+                const int l = __float2int_rz(__fadd_rn(r, uu[e])); // r + u >= 0: truncation is the floor
+                lev[e] = (uint32_t)(l > dv.s - 1 ? dv.s - 1 : l);
             }
-            lev[e] = (uint32_t)l;
         }
         uint8_t* lrow = dv.nxt_levels + (int64_t)row * dv.lpitch;
         const bool in = li < nvalid;
@@ -276,7 +315,8 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
 template <int KIND, bool HAS_G, bool HAS_M, bool EMIT>
 cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    constexpr size_t smem = (size_t)n_arrays<HAS_G, HAS_M>() * kDTile * sizeof(float) + NIT * 8 * sizeof(float) + 16;
+    constexpr size_t smem = (size_t)n_arrays<HAS_G, HAS_M>() * kDTile * sizeof(float) +
+                            NIT * 8 * sizeof(float) + 16;
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);

@@ -169,6 +169,8 @@ class Workload:
         if self.graph.startswith("torus"):
             r, c = self.graph[5:].split("x")
             return torus(int(r), int(c))
+        if self.graph == "social32":
+            return random_graph(32, 14, 1)
         raise ValueError(self.graph)
 
 
@@ -195,6 +197,21 @@ WORKLOADS = {
     "c5_ring32_topk": Workload("c5_ring32_topk", 32, 25_557_032, "ring", "topk",
                                k=k_of(1, 1000, 25_557_032), eta=0.1, gamma=0.1, steps=200,
                                x_var=0.01, g_var=1e-3),
+    # irregular 32-node graph (max degree 14), scaled sign as in the paper's on-device
+    # runs: a ResNet-20-sized and an LSTM-sized (28.95 M) flat vector; and top-1 %
+    "c6_social32_sign": Workload("c6_social32_sign", 32, 272474, "social32", "sign", eta=0.1,
+                                 gamma=0.5, steps=1000, x_var=0.01, g_var=1e-2),
+    "c6_social32_sign_lstm": Workload("c6_social32_sign_lstm", 32, 28_950_000, "social32", "sign",
+                                      eta=0.1, gamma=0.6, steps=100, x_var=0.01, g_var=1e-3),
+    "c6_social32_topk": Workload("c6_social32_topk", 32, 272474, "social32", "topk",
+                                 k=k_of(1, 100, 272474), eta=0.1, gamma=0.04, steps=1000,
+                                 x_var=0.01, g_var=1e-2),
+    # mid-sized dense cases (1 GB of state): small enough for a full counter capture,
+    # larger than L2
+    "p_ring8_qsgd": Workload("p_ring8_qsgd", 8, 8 * 1024 * 1024, "ring", "qsgd", s=16, bucket=512,
+                             eta=0.1, gamma=0.1, steps=100, x_var=0.01, g_var=1e-3),
+    "p_ring8_sign": Workload("p_ring8_sign", 8, 8 * 1024 * 1024, "ring", "sign", eta=0.1,
+                             gamma=0.4, steps=100, x_var=0.01, g_var=1e-3),
 }
 
 
