@@ -123,7 +123,6 @@ cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cud
 cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st);
 // update kernel; emit: also collect the next step's top-k candidates (if apply_can_emit)
 bool apply_can_emit(const Dev& dv, const StepArgs& a);
-bool update_bulk_usable(const Dev& dv, const StepArgs& a);
 cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
 bool update_dense_can_emit(const Dev& dv);
 cudaError_t launch_update_dense(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);

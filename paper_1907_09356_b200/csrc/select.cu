@@ -332,6 +332,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     const int64_t nspan = (dv.d + span - 1) / span;
     constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
     uint32_t prefix = 0, pmask = 0, need = k;
+    uint32_t aim_lo = 0, aim_count = 0;
     const int shifts[3] = {21, 10, 0};
     const int nbins[3] = {2048, 2048, 1024};
     for (int pass = 0; pass < 3; ++pass) {
@@ -350,6 +351,16 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
         __syncthreads();
         uint32_t digit, above;
         block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
+        if (KIND == SEL_TOPK && pass == 0) {
+            // a second point for the next step's bound: the eighth-of-an-octave bin that holds
+            // the rank the bound aims at, and how many keys lie at or above its lower edge
+            const uint64_t want = (uint64_t)k * kAimAfterMiss / 256u;
+            uint32_t d2, a2;
+            block_find_digit<kSelThreads>(h, nbins[0], (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d), sm,
+                                          &d2, &a2);
+            aim_lo = d2 << shifts[0];
+            aim_count = a2 + h[d2];
+        }
         need -= above;
         prefix |= digit << shifts[pass];
         pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
@@ -407,7 +418,8 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
         if (KIND == SEL_TOPK) {
-            dv.row_lo[row] = lower_bound_key(T, 3u);
+            // between (rank k, key T) and (rank aim_count, key aim_lo), as after a usable step
+            dv.row_lo[row] = next_bound(aim_lo, T, aim_count, k, kAimAfterMiss);
             dv.row_aim[row] = kAimAfterMiss;
         }
         atomicAdd(&dv.stats->exact_rows, 1ull);

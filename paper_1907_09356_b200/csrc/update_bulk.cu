@@ -3,9 +3,13 @@
 //     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
 //     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i).
 //
-// Requirements: rows 16-byte aligned, d a multiple of 4.  The x, x^, s, g (and momentum)
-// tiles are fetched into shared memory by asynchronous bulk copies that complete on an
-// mbarrier, so no registers are tied up while they are in flight.  Meanwhile the block reads
+// The x, x^, s, g (and momentum) tiles are fetched into shared memory by asynchronous bulk
+// copies that complete on an mbarrier, so no registers are tied up while they are in flight.
+// A bulk copy needs 16-byte aligned addresses and sizes.  With AL (rows 16-byte aligned, d a
+// multiple of 4) a tile is copied as it is; otherwise each copy starts at the 16-byte
+// boundary at or below the tile's first element and ends at the one at or above its last
+// (never touching a 16-byte unit that holds no element of the tile), and the tile is read
+// from shared memory at the resulting offset of 0..3 elements.  Meanwhile the block reads
 // the range records of its neighbours (one round trip), then all their entries that fall
 // into the tile (a second one), and adds them into a shared accumulator tile neighbour by
 // neighbour.  With EMIT the kernel also collects the candidates of the next step's top-k
@@ -53,27 +57,34 @@ struct NbrTable {
 template <bool HAS_G, bool HAS_M>
 __host__ __device__ constexpr int bulk_arrays() { return 3 + (HAS_G ? 1 : 0) + (HAS_M ? 1 : 0); }
 
-template <bool HAS_G, bool HAS_M>
+constexpr int kShiftPad = 4; // floats of slack per staged tile when it may start mid-unit
+
+template <bool HAS_G, bool HAS_M, bool AL>
 constexpr size_t bulk_smem_bytes()
 {
     return (size_t)(bulk_arrays<HAS_G, HAS_M>() + 1) * kTile * sizeof(float) // tiles + acc
+           + (AL ? 0 : bulk_arrays<HAS_G, HAS_M>() * kShiftPad * sizeof(float))
            + 2 * (kTile / 32) * sizeof(uint32_t)                              // touched, self
            + 8                                                                // barrier
            + 2 * (NT / 32 + 1) * sizeof(uint32_t) + 8                         // scan scratch, base
            + sizeof(NbrTable);
 }
 
-template <bool HAS_G, bool HAS_M, bool EMIT>
+// element offset of p inside its 16-byte unit
+__device__ __forceinline__ uint32_t unit_shift(const float* p) { return (uint32_t)(((uintptr_t)p & 15u) >> 2); }
+
+template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepArgs a)
 {
     static_assert(NT >= kTile / 32 && NT >= kMaxNb, "one thread per mask word / neighbour");
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    constexpr int kStage = kTile + (AL ? 0 : kShiftPad);
     float* xs = reinterpret_cast<float*>(smem_raw);
-    float* hs = xs + kTile;
-    float* ss = hs + kTile;
-    float* gs = ss + kTile;                             // used when HAS_G
-    float* ms = gs + (HAS_G ? kTile : 0);               // used when HAS_M
-    float* acc = ms + (HAS_M ? kTile : 0);
+    float* hs = xs + kStage;
+    float* ss = hs + kStage;
+    float* gs = ss + kStage;                            // used when HAS_G
+    float* ms = gs + (HAS_G ? kStage : 0);              // used when HAS_M
+    float* acc = ms + (HAS_M ? kStage : 0);
     uint32_t* touched = reinterpret_cast<uint32_t*>(acc + kTile);
     uint32_t* tself = touched + kTile / 32;
     uint64_t* bar = reinterpret_cast<uint64_t*>(tself + kTile / 32);
@@ -84,23 +95,29 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     const int row = blockIdx.y;
     const int64_t tile = blockIdx.x;
     const int64_t c0 = tile * kTile;
-    const int nvalid = (int)((dv.d - c0) < kTile ? (dv.d - c0) : kTile); // multiple of 4
+    const int nvalid = (int)((dv.d - c0) < kTile ? (dv.d - c0) : kTile); // AL: a multiple of 4
     const int lane = threadIdx.x & 31;
     float* xr = a.X + (int64_t)row * dv.ld + c0;
     float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
     float* sr = a.S + (int64_t)row * dv.ld + c0;
     const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
 
+    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld + c0 : nullptr;
+    float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
+    // where each staged tile's first element sits in its shared-memory buffer
+    const uint32_t shx = AL ? 0u : unit_shift(xr), shh = AL ? 0u : unit_shift(hr), shs = AL ? 0u : unit_shift(sr);
+    const uint32_t shg = (AL || !HAS_G) ? 0u : unit_shift(gr), shm = (AL || !HAS_M) ? 0u : unit_shift(mrow);
     if (threadIdx.x == 0) {
         mbar_init(bar, 1);
-        const uint32_t bytes = (uint32_t)nvalid * sizeof(float);
-        mbar_expect_tx(bar, bytes * bulk_arrays<HAS_G, HAS_M>());
-        bulk_load(xs, xr, bytes, bar);
-        bulk_load(hs, hr, bytes, bar);
-        bulk_load(ss, sr, bytes, bar);
-        if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, bytes, bar);
-        if (HAS_M) bulk_load(ms, a.M + (int64_t)row * dv.ld + c0, bytes, bar);
+        auto span = [&](uint32_t sh) { return (((uint32_t)nvalid + sh) * (uint32_t)sizeof(float) + 15u) & ~15u; };
+        mbar_expect_tx(bar, span(shx) + span(shh) + span(shs) + (HAS_G ? span(shg) : 0u) + (HAS_M ? span(shm) : 0u));
+        bulk_load(xs, xr - shx, span(shx), bar);
+        bulk_load(hs, hr - shh, span(shh), bar);
+        bulk_load(ss, sr - shs, span(shs), bar);
+        if (HAS_G) bulk_load(gs, gr - shg, span(shg), bar);
+        if (HAS_M) bulk_load(ms, mrow - shm, span(shm), bar);
     }
+    hs += shh; // the in-place x^ update below addresses the tile by coordinate
 #pragma unroll
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -219,19 +236,25 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
     uint32_t take = 0, cnt[NIT];
     uint32_t vbits[NIT][4];
-    float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
+    // a staged quad: one 128-bit read when the tile sits aligned, else element by element
+    auto staged_quad = [&](const float* buf, uint32_t sh, int q4) {
+        if (AL) return reinterpret_cast<const float4*>(buf)[q4];
+        const float* p = buf + sh + q4 * kQuad;
+        const int left = nvalid - q4 * kQuad;
+        return make_float4(p[0], left > 1 ? p[1] : 0.f, left > 2 ? p[2] : 0.f, left > 3 ? p[3] : 0.f);
+    };
 #pragma unroll
     for (int it = 0; it < NIT; ++it) {
         const int q4 = it * NT + threadIdx.x;
         const int li = q4 * kQuad;
         cnt[it] = 0;
         if (li >= nvalid) continue;
-        const float4 x = reinterpret_cast<const float4*>(xs)[q4];
-        const float4 h = reinterpret_cast<const float4*>(hs)[q4];
-        const float4 s = reinterpret_cast<const float4*>(ss)[q4];
+        const float4 x = staged_quad(xs, shx, q4);
+        const float4 h = staged_quad(hs, 0u, q4);
+        const float4 s = staged_quad(ss, shs, q4);
         float4 g = make_float4(0.f, 0.f, 0.f, 0.f), m = g;
-        if (HAS_G) g = reinterpret_cast<const float4*>(gs)[q4];
-        if (HAS_M) m = reinterpret_cast<const float4*>(ms)[q4];
+        if (HAS_G) g = staged_quad(gs, shg, q4);
+        if (HAS_M) m = staged_quad(ms, shm, q4);
         const uint32_t tb = (touched[li >> 5] >> (li & 31)) & 0xFu;
         const uint32_t sb = (tself[li >> 5] >> (li & 31)) & 0xFu;
         const float xv[4] = {x.x, x.y, x.z, x.w};
@@ -257,14 +280,23 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
             xn[e] = next_x<HAS_G, HAS_M>(xv[e], sv[e], hv[e], gv[e], mv4[e], u);
             if (EMIT) {
                 vbits[it][e] = __float_as_uint(__fsub_rn(xn[e], hv[e]));
-                if (order_key<SEL_TOPK>(vbits[it][e]) >= lo_key) {
+                if ((AL || li + e < nvalid) && order_key<SEL_TOPK>(vbits[it][e]) >= lo_key) {
                     take |= 1u << (4 * it + e);
                     ++cnt[it];
                 }
             }
         }
-        *reinterpret_cast<float4*>(xr + li) = make_float4(xn[0], xn[1], xn[2], xn[3]);
-        if (HAS_M) *reinterpret_cast<float4*>(mrow + li) = make_float4(mv4[0], mv4[1], mv4[2], mv4[3]);
+        if (AL) {
+            *reinterpret_cast<float4*>(xr + li) = make_float4(xn[0], xn[1], xn[2], xn[3]);
+            if (HAS_M) *reinterpret_cast<float4*>(mrow + li) = make_float4(mv4[0], mv4[1], mv4[2], mv4[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (li + e < nvalid) {
+                    xr[li + e] = xn[e];
+                    if (HAS_M) mrow[li + e] = mv4[e];
+                }
+        }
     }
 
     if (EMIT) {
@@ -296,10 +328,10 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     }
 }
 
-template <bool HAS_G, bool HAS_M, bool EMIT>
+template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    constexpr size_t smem = bulk_smem_bytes<HAS_G, HAS_M>();
+    constexpr size_t smem = bulk_smem_bytes<HAS_G, HAS_M, AL>();
     // Once per device and instantiation: allow the dynamic shared memory size and ask for the
     // largest shared-memory carve-out, so that as many tiles as possible are in flight per SM.
     static bool configured[64] = {};
@@ -307,7 +339,7 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        auto kern = update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT>;
+        auto kern = update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT, AL>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -316,21 +348,23 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
-    return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT>, grid, dim3(NT), smem, st, dv, a);
+    return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT, AL>, grid, dim3(NT), smem, st, dv, a);
+}
+
+template <bool AL>
+cudaError_t launch_terms(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
+{
+    if (a.M) return emit ? launch_bulk<true, true, true, AL>(dv, a, st) : launch_bulk<true, true, false, AL>(dv, a, st);
+    if (a.G) return emit ? launch_bulk<true, false, true, AL>(dv, a, st) : launch_bulk<true, false, false, AL>(dv, a, st);
+    return emit ? launch_bulk<false, false, true, AL>(dv, a, st) : launch_bulk<false, false, false, AL>(dv, a, st);
 }
 
 } // namespace
 
-bool update_bulk_usable(const Dev& dv, const StepArgs& a)
-{
-    return (dv.kind == CHOCO_Q_TOPK || dv.kind == CHOCO_Q_RANDK) && a.vec && dv.d % 4 == 0;
-}
-
 cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {
-    if (a.M) return emit ? launch_bulk<true, true, true>(dv, a, st) : launch_bulk<true, true, false>(dv, a, st);
-    if (a.G) return emit ? launch_bulk<true, false, true>(dv, a, st) : launch_bulk<true, false, false>(dv, a, st);
-    return emit ? launch_bulk<false, false, true>(dv, a, st) : launch_bulk<false, false, false>(dv, a, st);
+    // a.vec: every row of every array starts on a 16-byte boundary
+    return (a.vec && dv.d % 4 == 0) ? launch_terms<true>(dv, a, emit, st) : launch_terms<false>(dv, a, emit, st);
 }
 
 } // namespace choco

@@ -150,6 +150,48 @@ def test_randk_shapes(d, k, ld):
     ch.close()
 
 
+@pytest.mark.parametrize("kind,kw", [("topk", dict(k=300)), ("randk", dict(k=300)), ("sign", {}),
+                                     ("qsgd", dict(s=16, bucket=256))])
+def test_arrays_at_different_offsets_in_a_16_byte_unit(kind, kw):
+    """X, Xhat, S, G start 0, 4, 8 and 12 bytes into a 16-byte unit; rows of 4099 floats move
+    the offset from row to row; the floats around every array stay untouched."""
+    w = workloads.ring(6)
+    n, d, steps = 6, 4099, 3
+    p = oracle.Params(kind, seed=5, **kw)
+    X = workloads.normal_rows(n, d, 1.0, 77)
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    guard = 8
+
+    def place(a, off):
+        flat = torch.full((guard + off + n * d + guard,), float("nan"), dtype=torch.float32, device=DEV)
+        view = flat[guard + off: guard + off + n * d].view(n, d)
+        view.copy_(torch.from_numpy(a))
+        assert view.data_ptr() % 16 == 4 * off
+        return flat, view
+
+    fX, dX = place(X, 0)
+    fXh, dXh = place(Xh, 1)
+    fS, dS = place(S, 2)
+    ch = choco.Choco(w, d, kind, seed=5, **kw)
+    try:
+        for t in range(steps):
+            G = workloads.normal_rows(n, d, 0.01, 900 + t)
+            fG, dG = place(G, 3)
+            msgs = oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, t)
+            ch.sgd_step(dX, dXh, dS, dG, 0.1, 0.2)
+            torch.cuda.synchronize()
+            check_messages(ch.ctx, kind, msgs, d)
+            assert_state(dXh.cpu().numpy(), Xh, f"Xhat after step {t}")
+            assert_state(dS.cpu().numpy(), S, f"S after step {t}")
+            assert_state(dX.cpu().numpy(), X, f"X after step {t}")
+            assert np.array_equal(dG.cpu().numpy(), G)
+            for flat, off in ((fX, 0), (fXh, 1), (fS, 2), (fG, 3)):
+                assert bool(torch.isnan(flat[:guard + off]).all()) and bool(torch.isnan(flat[guard + off + n * d:]).all())
+        assert choco.choco_get_stats(ch.ctx)["device_timeouts"] == 0
+    finally:
+        ch.close()
+
+
 def test_topk_ties_zeros_and_signed_zero():
     n, d, k = 4, 9000, 700
     rng = np.random.default_rng(0)
