@@ -332,7 +332,10 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     const int64_t nspan = (dv.d + span - 1) / span;
     constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
     uint32_t prefix = 0, pmask = 0, need = k;
-    uint32_t aim_lo = 0, aim_count = 0;
+    uint32_t aim_lo = 0, aim_count = 0, aim_above = 0;
+    bool aim_in_bin = false;
+    const uint64_t aim_want = (uint64_t)k * kAimAfterMiss / 256u;
+    const uint32_t aim_rank = (uint32_t)(aim_want < (uint64_t)dv.d ? aim_want : (uint64_t)dv.d);
     const int shifts[3] = {21, 10, 0};
     const int nbins[3] = {2048, 2048, 1024};
     for (int pass = 0; pass < 3; ++pass) {
@@ -354,12 +357,17 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
         if (KIND == SEL_TOPK && pass == 0) {
             // a second point for the next step's bound: the eighth-of-an-octave bin that holds
             // the rank the bound aims at, and how many keys lie at or above its lower edge
-            const uint64_t want = (uint64_t)k * kAimAfterMiss / 256u;
             uint32_t d2, a2;
-            block_find_digit<kSelThreads>(h, nbins[0], (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d), sm,
-                                          &d2, &a2);
+            block_find_digit<kSelThreads>(h, nbins[0], aim_rank, sm, &d2, &a2);
             aim_lo = d2 << shifts[0];
             aim_count = a2 + h[d2];
+            aim_in_bin = d2 == digit; // the same bin as rank k: the next pass resolves it further
+            aim_above = above;
+        } else if (KIND == SEL_TOPK && pass == 1 && aim_in_bin) {
+            uint32_t d2, a2;
+            block_find_digit<kSelThreads>(h, nbins[1], aim_rank - aim_above, sm, &d2, &a2);
+            aim_lo = prefix | (d2 << shifts[1]);
+            aim_count = aim_above + a2 + h[d2];
         }
         need -= above;
         prefix |= digit << shifts[pass];

@@ -230,6 +230,20 @@ def test_topk_carry_across_steps():
     ch2.close()
 
 
+def test_topk_values_in_one_histogram_bin_recover_after_exact_selection():
+    """All |x - x^| within 5 % of each other: the first histogram cannot separate them, the rows
+    are selected exactly, and the bound set there must make the next steps' candidates usable."""
+    n, d, k, steps = 4, 200_000, 2000, 6
+    rng = np.random.default_rng(12)
+    x0 = ((1.0 + 0.05 * rng.random((n, d))) * rng.choice([-1.0, 1.0], size=(n, d))).astype(np.float32)
+    ch, _, _ = run_lockstep(workloads.ring(n), "topk", n, d, steps, k=k, seed=3, gamma=0.01, eta=0.01,
+                            g_var=1e-8, x_init=x0)
+    st = choco.choco_get_stats(ch.ctx)
+    ch.close()
+    assert st["exact_rows"] <= 2 * n, st
+    assert st["prepared_rows"] >= n * (steps - 2), st
+
+
 @pytest.mark.parametrize("kind,kw", [("sign", {}), ("qsgd", dict(s=16, bucket=512)), ("identity", {})])
 def test_dense_carry_across_steps(kind, kw):
     """For dense operators the update kernel writes the next step's messages; switching that
