@@ -31,8 +31,12 @@ L2_BYTES = 126 * 2 ** 20
 NOMINAL_HBM_GBS = 8000.0           # the figure the 60 % target is quoted against
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, from the ncu
-# capture summarised under profiles/ (None for workloads that were not captured)
-NCU_TRAFFIC = {("c4_torus64_topk", "update"): 1.365e9}
+# captures summarised under profiles/ (None for workloads that were not captured).  The
+# 32-ring QSGD figure is the 8-ring capture of the same kernel scaled by the coordinates per
+# launch (29.70 B per coordinate), as the capture of the full-size workload would be too large.
+NCU_TRAFFIC = {("c4_torus64_topk", "update"): 1.366e9,
+               ("p_ring8_qsgd", "update"): 1.993e9,
+               ("c5_ring32_qsgd", "update"): 29.70 * 32 * 25_557_032}
 
 
 def measured_peak():
