@@ -53,21 +53,38 @@ def measured_peak():
 # ------------------------------------------------------------------------------------------
 
 
-def message_bytes(wl) -> int:
-    d = wl.d
-    if wl.q == "topk":
-        return 8 * wl.k
-    if wl.q == "randk":
-        return 4 * wl.k
-    if wl.q == "sign":
+def message_bytes_of(q: str, d: int, k: int, s: int, bucket: int) -> int:
+    if q == "topk":
+        return 8 * k
+    if q == "randk":
+        return 4 * k
+    if q == "sign":
         return 4 * ((d + 31) // 32) + 4
-    if wl.q == "qsgd":
-        blen = wl.bucket or d
+    if q == "qsgd":
+        blen = bucket or d
         wbits = 1
-        while (1 << wbits) < wl.s:
+        while (1 << wbits) < s:
             wbits *= 2
         return 4 * ((d + blen - 1) // blen) + 4 * ((d + 31) // 32) + (d * wbits + 7) // 8
     return 4 * d
+
+
+def layer_k(wl, length: int) -> int:
+    return max(1, (length * wl.a_num) // wl.a_den)
+
+
+def entries_per_row(wl) -> int:
+    """Entries a sparse Q keeps per worker (summed over the layers, if any)."""
+    if wl.layers:
+        return sum(layer_k(wl, dl) for dl in wl.layer_sizes())
+    return wl.k
+
+
+def message_bytes(wl) -> int:
+    """Per worker and step, by the paper's accounting."""
+    if wl.layers:
+        return sum(message_bytes_of(wl.q, dl, layer_k(wl, dl), wl.s, wl.bucket) for dl in wl.layer_sizes())
+    return message_bytes_of(wl.q, wl.d, wl.k, wl.s, wl.bucket)
 
 
 def step_min_bytes(wl, w, sgd=True) -> int:
@@ -79,7 +96,8 @@ def step_min_bytes(wl, w, sgd=True) -> int:
     msg = message_bytes(wl)
     if wl.q in ("topk", "randk"):
         dense = (20 if sgd else 16) * N
-        return dense + msg * wl.n + msg * deg_off + 4 * (wl.n * wl.k + nnz * wl.k)
+        k = entries_per_row(wl)
+        return dense + msg * wl.n + msg * deg_off + 4 * (wl.n * k + nnz * k)
     dense = (28 if sgd else 24) * N
     return dense + msg * wl.n + msg * deg_off
 
@@ -92,7 +110,8 @@ def update_kernel_bytes(wl, w, sgd=True) -> int:
     msg = message_bytes(wl)
     if wl.q in ("topk", "randk"):
         per_entry = 8                                   # index + value as read by the kernel
-        return (20 if sgd else 16) * N + per_entry * wl.k * nnz + 4 * (wl.n * wl.k + nnz * wl.k)
+        k = entries_per_row(wl)
+        return (20 if sgd else 16) * N + per_entry * k * nnz + 4 * (wl.n * k + nnz * k)
     return (28 if sgd else 24) * N + msg * nnz
 
 
@@ -166,7 +185,11 @@ def oracle_sample(wl, w, budget_rows=None):
                               np.asarray(val, np.float32))
     p = oracle.Params(wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=1)
     t0 = time.perf_counter()
-    oracle.step(sub, p, X, Xh, S, G, wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
+    if wl.layers:
+        oracle.step_layers(sub, p, workloads.layer_offsets(wl.layer_sizes()), wl.a_num, wl.a_den, X, Xh, S, G,
+                           wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
+    else:
+        oracle.step(sub, p, X, Xh, S, G, wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
     dt = time.perf_counter() - t0
     text = (f"one oracle step for {len(rows)} of {wl.n} workers of {wl.name} "
             f"(their {len(need)} neighbours' messages formed too), single thread")
@@ -218,7 +241,9 @@ def main():
     w = wl.mixing()
     N = wl.n * wl.d
     config = {"workload": wl.name, "n": wl.n, "d": wl.d, "graph": wl.graph, "Q": wl.q,
-              "k": wl.k, "s": wl.s, "bucket": wl.bucket, "eta": wl.eta, "gamma": wl.gamma,
+              "k": entries_per_row(wl) if wl.q in ("topk", "randk") else 0, "s": wl.s, "bucket": wl.bucket,
+              "layers": (f"{wl.layers}: Q per layer, {len(wl.layer_sizes())} layers" if wl.layers else "none: Q on the whole row"),
+              "eta": wl.eta, "gamma": wl.gamma,
               "parallelism": "replicas only" if args.gpus > 1 else "single GPU",
               "l2": "inputs per step exceed L2" if 20 * N > 2 * L2_BYTES else "state fits L2 (no flush)"}
 
@@ -264,7 +289,27 @@ def main():
     pool_n = int(max(2, min(args.pool, (free_b * 0.5) // (4 * N))))
     pool = [torch.randn(wl.n, wl.d, device=dev, generator=gen) * float(np.sqrt(wl.g_var or 1e-2))
             for _ in range(pool_n)]
-    ch = choco.Choco(w, wl.d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=7)
+    if wl.layers:
+        off = workloads.layer_offsets(wl.layer_sizes())
+        lay = choco.choco_layers_init(wl.n, off, wl.d, w.row_ptr, w.col, w.val, wl.q, wl.a_num, wl.a_den,
+                                      s=wl.s or 16, bucket=wl.bucket, seed=7)
+        ctxs = [choco.choco_layers_get_layer(lay, l)[0] for l in range(len(off) - 1)]
+
+        def do_step(G):
+            choco.choco_layers_sgd_step(lay, X, Xh, S, G, wl.eta, wl.gamma)
+    else:
+        ch = choco.Choco(w, wl.d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=7)
+        ctxs = [ch.ctx]
+
+        def do_step(G):
+            ch.sgd_step(X, Xh, S, G, wl.eta, wl.gamma)
+
+    def stats_sum():
+        tot = {}
+        for c in ctxs:
+            for key, v in choco.choco_get_stats(c).items():
+                tot[key] = tot.get(key, 0) + int(v)
+        return tot
 
     def barrier():
         torch.cuda.synchronize()
@@ -273,11 +318,12 @@ def main():
         torch.cuda.synchronize()
 
     for t in range(args.warmup):
-        ch.sgd_step(X, Xh, S, pool[t % pool_n], wl.eta, wl.gamma)
+        do_step(pool[t % pool_n])
     barrier()
-    st0 = choco.choco_get_stats(ch.ctx)
-    choco.choco_profile_enable(ch.ctx, args.steps)
-    choco.choco_profile_set_stride(ch.ctx, args.profile_stride)   # events between kernels cost time
+    st0 = stats_sum()
+    if not wl.layers:
+        choco.choco_profile_enable(ch.ctx, args.steps)
+        choco.choco_profile_set_stride(ch.ctx, args.profile_stride)   # events between kernels cost time
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -287,14 +333,14 @@ def main():
     t_wall0 = time.time()
     e0.record()
     for t in range(args.steps):
-        ch.sgd_step(X, Xh, S, pool[(args.warmup + t) % pool_n], wl.eta, wl.gamma)
+        do_step(pool[(args.warmup + t) % pool_n])
     e1.record()
     barrier()
     t_wall1 = time.time()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    st1 = choco.choco_get_stats(ch.ctx)
-    nrec, upd_ms = choco.choco_profile_read(ch.ctx)
+    st1 = stats_sum()
+    nrec, upd_ms = (0, 0.0) if wl.layers else choco.choco_profile_read(ch.ctx)
     finite = bool(torch.isfinite(X).all())
 
     # end to end: host buffers in, host buffers out, through choco_sgd_step_host
@@ -302,11 +348,24 @@ def main():
     if args.e2e_steps > 0:
         hX, hXh, hS = (t.cpu().pin_memory() for t in (X, Xh, S))
         hG = pool[0].cpu().pin_memory()
-        choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)      # warm-up, allocates staging
+        if wl.layers:
+            # the layered calls take device arrays: copy in from pinned memory, step, copy out
+            def host_step():
+                for dst, src in ((X, hX), (Xh, hXh), (S, hS), (pool[0], hG)):
+                    dst.copy_(src, non_blocking=True)
+                do_step(pool[0])
+                for dst, src in ((hX, X), (hXh, Xh), (hS, S)):
+                    dst.copy_(src, non_blocking=True)
+                torch.cuda.synchronize()
+            choco.choco_layers_invalidate(lay)
+        else:
+            def host_step():
+                choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)
+        host_step()                                                # warm-up, allocates staging
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
-            choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)
+            host_step()
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
         e2e = {"seconds": e2e_s, "steps": args.e2e_steps}
@@ -325,6 +384,12 @@ def main():
         achieved = upd_bytes / upd_avg_s / 1e9 if nrec else None
         step_bytes = step_min_bytes(wl, w)
         step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
+        roof_kernel = "update (apply) kernel"
+        if wl.layers:
+            # one small set of kernels per layer: no single dominant launch to time, so the
+            # roofline entry is the whole step (all layers' kernels) against its minimum bytes
+            roof_kernel = "whole step: the kernels of all layers"
+            achieved, upd_bytes, upd_avg_s, nrec = step_gbs, step_bytes, ms_step * 1e-3, args.steps
         out = {
             "metric": "coords_per_sec", "value": value, "unit": "coords/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
@@ -335,7 +400,7 @@ def main():
             "step_min_bytes": step_bytes, "step_hbm_gbs": step_gbs,
             "step_frac_of_measured_peak": step_gbs / peak,
             "step_frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
-            "roofline": {"bound": "hbm", "kernel": "update (apply) kernel", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None,
                          "traffic": NCU_TRAFFIC.get((wl.name, "update")),
@@ -350,13 +415,18 @@ def main():
         if e2e:
             out["e2e"] = {"value": whole_job_rate(world, N, e2e["steps"], e2e["seconds"]), "unit": "coords/s",
                           "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,
-                          "steps": e2e["steps"], "api": "choco_sgd_step_host, pinned host buffers"}
+                          "steps": e2e["steps"],
+                          "api": ("pinned host buffers copied in and out around choco_layers_sgd_step" if wl.layers
+                                  else "choco_sgd_step_host, pinned host buffers")}
         if not args.no_cpu_baseline and world == 1:
             coords, dt, text = oracle_sample(wl, w, rows_for_budget(wl))
             out["cpu_baseline"] = {"value": coords / dt, "unit": "coords/s", "cores": 1,
                                    "kind": "oracle", "sample": text, "seconds": dt}
         print(json.dumps(out))
-    ch.close()
+    if wl.layers:
+        choco.choco_layers_destroy(lay)
+    else:
+        ch.close()
     if world > 1:
         dist.destroy_process_group()
 

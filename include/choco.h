@@ -199,6 +199,49 @@ int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* str
 int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t ld,
                                   double* out_dev, void* stream);
 
+/*
+ * Per-layer compression -- Section 5, "Setup": in the paper's experiments every compression
+ * scheme is applied to every layer of the network separately.  The first d = layer_off[n_layers]
+ * coordinates of a row are cut into n_layers consecutive layers, layer l = coordinates
+ * [layer_off[l], layer_off[l+1]), and Q acts on each layer as a vector of its own:
+ *   TOPK / RANDK   k_l = max(1, floor(a d_l)) entries per layer, a = a_num / a_den in (0, 1]
+ *                  (p->k is ignored; floor(a d_l) = 0 would never transmit a small layer, so
+ *                  at least one entry is kept);
+ *   SIGN           one scale ||v_l||_1 / d_l per layer;
+ *   QSGD           norms per block inside each layer (blocks restart at the layer's first
+ *                  coordinate; a layer shorter than p->bucket is one block of its own length);
+ *   the generator of layer l is keyed with seed + l and the coordinate's index inside the layer.
+ * Everything else (Algorithm 1 / 2, arithmetic, determinism) is as for the plain calls: a
+ * layered step gives the same bits as running choco_*_step with d = d_l, seed + l and
+ * pointers advanced by layer_off[l] for every layer.  That is also how it is carried out: one
+ * library context per layer, their kernels spread over a few internal streams that fork from
+ * and join `stream`, so a model of many small layers costs a few kernel launches per layer.
+ *   layer_off[n_layers + 1]   HOST, strictly increasing from 0; ld >= layer_off[n_layers].
+ *   a_num, a_den              used by TOPK / RANDK only.
+ * Errors are those of choco_init; on error nothing is left allocated.
+ */
+typedef struct choco_layers choco_layers;
+int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int64_t* layer_off, int64_t ld,
+                      const int32_t* w_row_ptr, const int32_t* w_col, const float* w_val, const choco_params* p,
+                      int64_t a_num, int64_t a_den, uint64_t seed);
+int choco_layers_destroy(choco_layers* layers);
+/* The three step calls, with the meaning of choco_gossip_step, choco_sgd_step and
+ * choco_sgd_momentum_step; X, Xhat, S, G, M are the whole [n, ld] DEVICE arrays. */
+int choco_layers_gossip_step(choco_layers* layers, float* X, float* Xhat, float* S, float gamma, void* stream);
+int choco_layers_sgd_step(choco_layers* layers, float* X, float* Xhat, float* S, const float* G, float eta,
+                          float gamma, void* stream);
+int choco_layers_sgd_momentum_step(choco_layers* layers, float* X, float* Xhat, float* S, const float* G,
+                                   float* M, float eta, float gamma, float lambda, float beta, void* stream);
+/* Sum over the layers of choco_message_bytes. */
+int choco_layers_message_bytes(const choco_layers* layers, int64_t* per_worker, int64_t* total);
+/* The context that serves one layer (owned by `layers`; for choco_get_message, choco_get_stats
+ * and the like), the layer's first coordinate and its length.  Any output may be NULL. */
+int choco_layers_get_layer(const choco_layers* layers, int32_t layer, choco_ctx** ctx, int64_t* offset,
+                           int64_t* length);
+/* choco_invalidate / choco_set_step for every layer. */
+int choco_layers_invalidate(choco_layers* layers);
+int choco_layers_set_step(choco_layers* layers, uint64_t t);
+
 /* Counters since choco_init (HOST struct filled after synchronising `stream`). */
 typedef struct {
     uint64_t steps;            /* step calls enqueued                                         */

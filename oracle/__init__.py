@@ -292,6 +292,39 @@ def step(w, p: Params, X: np.ndarray, Xhat: np.ndarray, S: np.ndarray,
     return msgs
 
 
+def layer_k(a_num: int, a_den: int, length: int) -> int:
+    """Entries a sparse Q keeps of a layer: floor(a d_l), but at least one (with floor(a d_l)
+    = 0 a small layer would never be transmitted)."""
+    return max(1, (length * a_num) // a_den)
+
+
+def step_layers(w, p: Params, layer_off: Sequence[int], a_num: int, a_den: int,
+                X: np.ndarray, Xhat: np.ndarray, S: np.ndarray, G: Optional[np.ndarray],
+                eta: float, gamma: float, t: int, M: Optional[np.ndarray] = None,
+                lam: float = 0.0, beta: float = 0.0,
+                rows: Optional[Sequence[int]] = None) -> list:
+    """Per-layer compression (Section 5, "Setup": every compression scheme is applied to
+    every layer separately): the columns [layer_off[l], layer_off[l+1]) of the arrays are
+    layer l, and one call of :func:`step` is made on each layer as a problem of its own
+    -- its own k = layer_k(a, d_l) for top-k / random-k, its own scale (sign) or blocks
+    (qsgd), the generator keyed with seed + l and the coordinate's index inside the layer.
+    Returns the per-layer message dictionaries."""
+    out = []
+    for l in range(len(layer_off) - 1):
+        lo, hi = int(layer_off[l]), int(layer_off[l + 1])
+        pl = dataclasses.replace(p, seed=p.seed + l)
+        if p.kind in ("topk", "randk"):
+            pl = dataclasses.replace(pl, k=layer_k(a_num, a_den, hi - lo))
+        parts = [np.ascontiguousarray(A[:, lo:hi]) if A is not None else None
+                 for A in (X, Xhat, S, G, M)]
+        out.append(step(w, pl, parts[0], parts[1], parts[2], parts[3], eta, gamma, t,
+                        rows=rows, M=parts[4], lam=lam, beta=beta))
+        for A, part in ((X, parts[0]), (Xhat, parts[1]), (S, parts[2]), (M, parts[4])):
+            if A is not None:
+                A[:, lo:hi] = part
+    return out
+
+
 def consensus_error(X: np.ndarray) -> float:
     """sum_i ||x_i - xbar||^2 in float64 (Section 6's distance times n)."""
     X = np.ascontiguousarray(X, dtype=np.float32)

@@ -26,6 +26,9 @@ EXPORTS = [
     "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
     "choco_last_cuda_error",
+    "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
+    "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
+    "choco_layers_invalidate", "choco_layers_set_step",
 ]
 
 
@@ -80,6 +83,17 @@ def load() -> ctypes.CDLL:
         lib.choco_strerror.argtypes = [ctypes.c_int]
         lib.choco_strerror.restype = ctypes.c_char_p
         lib.choco_last_cuda_error.argtypes = [vp]
+        lib.choco_layers_init.argtypes = [ctypes.POINTER(vp), i32, i32, vp, i64, vp, vp, vp,
+                                          ctypes.POINTER(choco_params), i64, i64, u64]
+        lib.choco_layers_destroy.argtypes = [vp]
+        lib.choco_layers_gossip_step.argtypes = [vp, vp, vp, vp, f32, vp]
+        lib.choco_layers_sgd_step.argtypes = [vp, vp, vp, vp, vp, f32, f32, vp]
+        lib.choco_layers_sgd_momentum_step.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, f32, vp]
+        lib.choco_layers_message_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        lib.choco_layers_get_layer.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(i64),
+                                               ctypes.POINTER(i64)]
+        lib.choco_layers_invalidate.argtypes = [vp]
+        lib.choco_layers_set_step.argtypes = [vp, u64]
         for name in EXPORTS:
             if name not in ("choco_strerror",):
                 getattr(lib, name).restype = ctypes.c_int
@@ -229,6 +243,64 @@ def choco_profile_read(ctx, stream=None) -> tuple[int, float]:
     n, ms = ctypes.c_int32(), ctypes.c_double()
     _check(load().choco_profile_read(ctx, ctypes.byref(n), ctypes.byref(ms), _stream(stream)), ctx)
     return n.value, ms.value
+
+
+def choco_layers_init(n: int, layer_off, ld: int, w_row_ptr, w_col, w_val, kind, a_num: int = 1,
+                      a_den: int = 1, s: int = 16, bucket: int = 0, qsgd_biased: bool = True,
+                      seed: int = 0):
+    """Per-layer compression: layer_off is a host array of n_layers + 1 offsets; top-k and
+    random-k keep max(1, floor(a_num / a_den * d_l)) entries of layer l."""
+    import numpy as np
+    off = np.ascontiguousarray(layer_off, dtype=np.int64)
+    rp = np.ascontiguousarray(w_row_ptr, dtype=np.int32)
+    col = np.ascontiguousarray(w_col, dtype=np.int32)
+    val = np.ascontiguousarray(w_val, dtype=np.float32)
+    p = choco_params(Q_KINDS[kind] if isinstance(kind, str) else int(kind), int(s), int(bucket),
+                     1 if qsgd_biased else 0, 0)
+    h = ctypes.c_void_p()
+    _check(load().choco_layers_init(ctypes.byref(h), n, len(off) - 1, off.ctypes.data, ld, rp.ctypes.data,
+                                    col.ctypes.data, val.ctypes.data, ctypes.byref(p), a_num, a_den, seed))
+    return h
+
+
+def choco_layers_destroy(layers) -> None:
+    _check(load().choco_layers_destroy(layers))
+
+
+def choco_layers_gossip_step(layers, X, Xhat, S, gamma: float, stream=None) -> None:
+    _check(load().choco_layers_gossip_step(layers, _ptr(X), _ptr(Xhat), _ptr(S), gamma, _stream(stream)))
+
+
+def choco_layers_sgd_step(layers, X, Xhat, S, G, eta: float, gamma: float, stream=None) -> None:
+    _check(load().choco_layers_sgd_step(layers, _ptr(X), _ptr(Xhat), _ptr(S), _ptr(G), eta, gamma,
+                                        _stream(stream)))
+
+
+def choco_layers_sgd_momentum_step(layers, X, Xhat, S, G, M, eta: float, gamma: float, lam: float,
+                                   beta: float, stream=None) -> None:
+    _check(load().choco_layers_sgd_momentum_step(layers, _ptr(X), _ptr(Xhat), _ptr(S), _ptr(G), _ptr(M),
+                                                 eta, gamma, lam, beta, _stream(stream)))
+
+
+def choco_layers_message_bytes(layers) -> tuple[int, int]:
+    a, b = ctypes.c_int64(), ctypes.c_int64()
+    _check(load().choco_layers_message_bytes(layers, ctypes.byref(a), ctypes.byref(b)))
+    return a.value, b.value
+
+
+def choco_layers_get_layer(layers, layer: int):
+    """(context handle of the layer, its first coordinate, its length)."""
+    c, o, n = ctypes.c_void_p(), ctypes.c_int64(), ctypes.c_int64()
+    _check(load().choco_layers_get_layer(layers, layer, ctypes.byref(c), ctypes.byref(o), ctypes.byref(n)))
+    return c, o.value, n.value
+
+
+def choco_layers_invalidate(layers) -> None:
+    _check(load().choco_layers_invalidate(layers))
+
+
+def choco_layers_set_step(layers, t: int) -> None:
+    _check(load().choco_layers_set_step(layers, t))
 
 
 # --------------------------------------------------------------------------- convenience

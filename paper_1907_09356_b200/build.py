@@ -13,6 +13,7 @@ LIB = os.path.join(HERE, "libchoco.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false",                      # no fused multiply-add: results must be reproducible
+    "-diag-suppress=186",               # "pointless comparison" in template branches that are compiled out
     "-Xcompiler", "-fPIC", "-shared",
 ]
 

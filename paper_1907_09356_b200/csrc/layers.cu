@@ -1,0 +1,192 @@
+// Per-layer compression (Section 5, "Setup": every compression scheme is applied to every
+// layer separately): the flat parameter vector is cut into consecutive layers and each layer is
+// its own vector for Q.  This file holds host code only.  A layered context owns one ordinary
+// context per layer, with d = the layer's length and the shared row pitch; a step runs the
+// layers' steps on column slices of the caller's arrays.  The layers are independent of each
+// other, so their kernels are spread over a few internal streams that fork from and join the
+// caller's stream.
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "internal.h"
+
+namespace {
+
+constexpr int kLayerStreams = 4;
+
+} // namespace
+
+struct choco_layers {
+    int32_t n;
+    int32_t n_layers;
+    int64_t ld;
+    std::vector<int64_t> off;      // n_layers + 1
+    std::vector<choco_ctx*> ctx;   // one per layer
+    cudaStream_t side[kLayerStreams];
+    cudaEvent_t fork;
+    cudaEvent_t join[kLayerStreams];
+    int nside;
+};
+
+namespace {
+
+void destroy_layers(choco_layers* L)
+{
+    if (!L) return;
+    for (choco_ctx* c : L->ctx)
+        if (c) choco_destroy(c);
+    for (int s = 0; s < L->nside; ++s) {
+        if (L->side[s]) cudaStreamDestroy(L->side[s]);
+        if (L->join[s]) cudaEventDestroy(L->join[s]);
+    }
+    if (L->fork) cudaEventDestroy(L->fork);
+    delete L;
+}
+
+int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+                float gamma, float lambda, float beta, void* stream)
+{
+    if (!L || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool fan = L->nside > 1 && L->n_layers > 1;
+    if (fan) {
+        if (cudaEventRecord(L->fork, st) != cudaSuccess) return CHOCO_ERR_CUDA;
+        for (int s = 0; s < L->nside; ++s)
+            if (cudaStreamWaitEvent(L->side[s], L->fork, 0) != cudaSuccess) return CHOCO_ERR_CUDA;
+    }
+    int rc = CHOCO_OK;
+    for (int32_t l = 0; l < L->n_layers && rc == CHOCO_OK; ++l) {
+        const int64_t o = L->off[l];
+        void* lst = fan ? (void*)L->side[l % L->nside] : stream;
+        if (M)
+            rc = choco_sgd_momentum_step(L->ctx[l], X + o, Xhat + o, S + o, G + o, M + o, eta, gamma, lambda,
+                                         beta, lst);
+        else if (G)
+            rc = choco_sgd_step(L->ctx[l], X + o, Xhat + o, S + o, G + o, eta, gamma, lst);
+        else
+            rc = choco_gossip_step(L->ctx[l], X + o, Xhat + o, S + o, gamma, lst);
+    }
+    if (fan) { // join even after an error so that the caller's stream stays ordered behind the layers
+        for (int s = 0; s < L->nside; ++s) {
+            if (cudaEventRecord(L->join[s], L->side[s]) != cudaSuccess) return CHOCO_ERR_CUDA;
+            if (cudaStreamWaitEvent(st, L->join[s], 0) != cudaSuccess) return CHOCO_ERR_CUDA;
+        }
+    }
+    return rc;
+}
+
+} // namespace
+
+extern "C" {
+
+int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int64_t* layer_off, int64_t ld,
+                      const int32_t* w_row_ptr, const int32_t* w_col, const float* w_val, const choco_params* p,
+                      int64_t a_num, int64_t a_den, uint64_t seed)
+{
+    if (!out || !layer_off || !p) return CHOCO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n_layers < 1 || layer_off[0] != 0) return CHOCO_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < n_layers; ++l)
+        if (layer_off[l + 1] <= layer_off[l]) return CHOCO_ERR_INVALID_ARG;
+    if (ld < layer_off[n_layers]) return CHOCO_ERR_INVALID_ARG;
+    const bool sparse = p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK;
+    if (sparse && (a_num < 1 || a_den < a_num)) return CHOCO_ERR_INVALID_ARG;
+
+    choco_layers* L = new (std::nothrow) choco_layers();
+    if (!L) return CHOCO_ERR_ALLOC;
+    L->n = n; L->n_layers = n_layers; L->ld = ld;
+    L->off.assign(layer_off, layer_off + n_layers + 1);
+    L->ctx.assign(n_layers, nullptr);
+    L->nside = 0; L->fork = nullptr;
+    std::memset(L->side, 0, sizeof(L->side));
+    std::memset(L->join, 0, sizeof(L->join));
+    for (int32_t l = 0; l < n_layers; ++l) {
+        const int64_t dl = layer_off[l + 1] - layer_off[l];
+        choco_params pl = *p;
+        if (sparse) {
+            // floor(a d_l) in integers, but never an empty message
+            const int64_t k = (int64_t)(((__int128)dl * a_num) / a_den);
+            pl.k = k < 1 ? 1 : k;
+        }
+        const int rc = choco_init(&L->ctx[l], n, dl, ld, w_row_ptr, w_col, w_val, &pl, seed + (uint64_t)l);
+        if (rc != CHOCO_OK) { destroy_layers(L); return rc; }
+    }
+    bool ok = cudaEventCreateWithFlags(&L->fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int s = 0; s < kLayerStreams && ok; ++s) {
+        ok = cudaStreamCreateWithFlags(&L->side[s], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&L->join[s], cudaEventDisableTiming) == cudaSuccess;
+        L->nside = s + 1;
+    }
+    if (!ok) { destroy_layers(L); return CHOCO_ERR_CUDA; }
+    *out = L;
+    return CHOCO_OK;
+}
+
+int choco_layers_destroy(choco_layers* L)
+{
+    destroy_layers(L);
+    return CHOCO_OK;
+}
+
+int choco_layers_gossip_step(choco_layers* L, float* X, float* Xhat, float* S, float gamma, void* stream)
+{
+    return layers_step(L, X, Xhat, S, nullptr, nullptr, 0.f, gamma, 0.f, 0.f, stream);
+}
+
+int choco_layers_sgd_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float eta,
+                          float gamma, void* stream)
+{
+    if (!G) return CHOCO_ERR_INVALID_ARG;
+    return layers_step(L, X, Xhat, S, G, nullptr, eta, gamma, 0.f, 0.f, stream);
+}
+
+int choco_layers_sgd_momentum_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M,
+                                   float eta, float gamma, float lambda, float beta, void* stream)
+{
+    if (!G || !M) return CHOCO_ERR_INVALID_ARG;
+    return layers_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+}
+
+int choco_layers_message_bytes(const choco_layers* L, int64_t* per_worker, int64_t* total)
+{
+    if (!L) return CHOCO_ERR_INVALID_ARG;
+    int64_t pw = 0;
+    for (choco_ctx* c : L->ctx) {
+        int64_t a = 0, b = 0;
+        const int rc = choco_message_bytes(c, &a, &b);
+        if (rc != CHOCO_OK) return rc;
+        pw += a;
+    }
+    if (per_worker) *per_worker = pw;
+    if (total) *total = pw * L->n;
+    return CHOCO_OK;
+}
+
+int choco_layers_get_layer(const choco_layers* L, int32_t layer, choco_ctx** ctx, int64_t* offset, int64_t* length)
+{
+    if (!L || layer < 0 || layer >= L->n_layers) return CHOCO_ERR_INVALID_ARG;
+    if (ctx) *ctx = L->ctx[layer];
+    if (offset) *offset = L->off[layer];
+    if (length) *length = L->off[layer + 1] - L->off[layer];
+    return CHOCO_OK;
+}
+
+int choco_layers_invalidate(choco_layers* L)
+{
+    if (!L) return CHOCO_ERR_INVALID_ARG;
+    for (choco_ctx* c : L->ctx) choco_invalidate(c);
+    return CHOCO_OK;
+}
+
+int choco_layers_set_step(choco_layers* L, uint64_t t)
+{
+    if (!L) return CHOCO_ERR_INVALID_ARG;
+    for (choco_ctx* c : L->ctx) {
+        const int rc = choco_set_step(c, t);
+        if (rc != CHOCO_OK) return rc;
+    }
+    return CHOCO_OK;
+}
+
+} // extern "C"

@@ -1,0 +1,106 @@
+"""Per-layer compression (choco_layers_*) vs the oracle's step_layers, through the C interface.
+
+Same acceptance as the plain step: indices, packed bits and level fields bit-exact, float32
+state within 1e-5 * max|x| and, because the operation order is fixed, identical.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1907_09356_b200 as choco
+import workloads
+from test_gpu_parity import DEV, _dev, _host, assert_state, check_messages
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [5, 1, 2048, 4097, 33, 12, 700]            # layers that start at every alignment
+
+KINDS = [
+    ("topk", dict(a=(1, 50))),
+    ("randk", dict(a=(1, 50))),
+    ("sign", dict()),
+    ("qsgd", dict(s=16, bucket=512)),
+    ("qsgd", dict(s=4, bucket=0)),
+    ("identity", dict()),
+]
+
+
+def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, seed=5,
+         check_layers=()):
+    off = workloads.layer_offsets(sizes)
+    n, d = w.n, int(off[-1])
+    a_num, a_den = kw.get("a", (1, 1))
+    X = workloads.normal_rows(n, d, 1.0, 31)
+    for l in range(len(sizes)):                                  # a different scale per layer
+        X[:, off[l]:off[l + 1]] *= np.float32(10.0 ** ((l % 5) - 2))
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    M = np.zeros_like(X) if momentum else None
+    dX, dXh, dS = _dev(X, ld), _dev(Xh, ld), _dev(S, ld)
+    dM = _dev(M, ld) if momentum else None
+    p = oracle.Params(kind, s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
+    h = choco.choco_layers_init(n, off, ld or d, w.row_ptr, w.col, w.val, kind, a_num, a_den,
+                                s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
+    try:
+        for t in range(steps):
+            G = None if gossip_only else workloads.normal_rows(n, d, 0.01, 100 + t)
+            dG = None if gossip_only else _dev(G, ld)
+            msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t,
+                                      M=M, lam=1e-4, beta=0.9)
+            if gossip_only:
+                choco.choco_layers_gossip_step(h, dX, dXh, dS, 0.2)
+            elif momentum:
+                choco.choco_layers_sgd_momentum_step(h, dX, dXh, dS, dG, dM, 0.05, 0.2, 1e-4, 0.9)
+            else:
+                choco.choco_layers_sgd_step(h, dX, dXh, dS, dG, 0.05, 0.2)
+            torch.cuda.synchronize()
+            for l in check_layers:
+                ctx, o, length = choco.choco_layers_get_layer(h, l)
+                assert (o, length) == (int(off[l]), int(off[l + 1] - off[l]))
+                check_messages(ctx, kind, msgs[l], length)
+            assert_state(_host(dX, d), X, f"X after step {t}")
+            assert_state(_host(dXh, d), Xh, f"Xhat after step {t}")
+            assert_state(_host(dS, d), S, f"S after step {t}")
+            if momentum:
+                assert_state(_host(dM, d), M, f"M after step {t}")
+        per_worker, total = choco.choco_layers_message_bytes(h)
+        assert total == per_worker * n
+        want = sum(next(iter(m.values())).paper_bytes(kind, int(off[l + 1] - off[l]), kw.get("s", 16))
+                   for l, m in enumerate(msgs))
+        assert per_worker == want
+        for l in range(len(sizes)):
+            ctx, _, _ = choco.choco_layers_get_layer(h, l)
+            assert choco.choco_get_stats(ctx)["device_timeouts"] == 0
+    finally:
+        choco.choco_layers_destroy(h)
+
+
+@pytest.mark.parametrize("kind,kw", KINDS, ids=[k + "-" + "-".join(f"{a}{b}" for a, b in kw.items()) for k, kw in KINDS])
+def test_ragged_layers(kind, kw):
+    _run(workloads.torus(2, 4), RAGGED, kind, kw, steps=4, check_layers=range(len(RAGGED)))
+
+
+@pytest.mark.parametrize("kind,kw", [KINDS[0], KINDS[2], KINDS[3]], ids=["topk", "sign", "qsgd"])
+def test_resnet20_layers_on_a_ring(kind, kw):
+    sizes = workloads.resnet20_layer_sizes()
+    _run(workloads.ring(8), sizes, kind, dict(kw, a=(1, 100)), steps=3, check_layers=(0, 1, 3, 40, 64))
+
+
+def test_padded_rows_and_momentum():
+    _run(workloads.ring(4), RAGGED, "topk", dict(a=(1, 20)), steps=3, ld=sum(RAGGED) + 11, momentum=True)
+    _run(workloads.ring(4), RAGGED, "sign", {}, steps=3, ld=sum(RAGGED) + 8, momentum=True)
+
+
+def test_gossip_only_layers():
+    _run(workloads.ring(4), RAGGED, "topk", dict(a=(1, 10)), steps=5, gossip_only=True)
+
+
+def test_rejects_bad_layer_tables():
+    w = workloads.ring(4)
+    for off in ([1, 5], [0, 5, 5], [0, 7, 3]):
+        with pytest.raises(choco.ChocoError):
+            choco.choco_layers_init(4, np.asarray(off, np.int64), 16, w.row_ptr, w.col, w.val, "sign")
+    with pytest.raises(choco.ChocoError):                        # ld shorter than the layers
+        choco.choco_layers_init(4, np.asarray([0, 8, 32], np.int64), 16, w.row_ptr, w.col, w.val, "sign")
+    with pytest.raises(choco.ChocoError):                        # a > 1
+        choco.choco_layers_init(4, np.asarray([0, 8], np.int64), 8, w.row_ptr, w.col, w.val, "topk", 3, 2)

@@ -140,6 +140,58 @@ def k_of(a_num: int, a_den: int, d: int) -> int:
     return (d * a_num) // a_den
 
 
+def resnet20_layer_sizes() -> list[int]:
+    """Lengths of the 65 parameter tensors of a CIFAR ResNet-20 in forward order (3x3
+    convolutions without bias, each followed by a batch-norm scale and shift; 1x1 projection
+    shortcuts where the width changes; a 64 -> 10 classifier).  They add up to 272 474, the
+    size the flat-vector workloads use.  Only the shape is taken from the architecture."""
+    sizes: list[int] = []
+
+    def conv_bn(cin: int, cout: int, ksz: int):
+        sizes.extend([cin * cout * ksz * ksz, cout, cout])
+
+    conv_bn(3, 16, 3)
+    width = 16
+    for stage_width in (16, 32, 64):
+        for block in range(3):
+            conv_bn(width, stage_width, 3)
+            conv_bn(stage_width, stage_width, 3)
+            if block == 0 and width != stage_width:
+                conv_bn(width, stage_width, 1)
+            width = stage_width
+    sizes.extend([64 * 10, 10])
+    return sizes
+
+
+def resnet50_layer_sizes() -> list[int]:
+    """Lengths of the 161 parameter tensors of an ImageNet ResNet-50 in forward order (7x7 stem,
+    bottleneck blocks [3, 4, 6, 3] of widths 64..512 with fourfold expansion, a batch-norm
+    scale and shift after every convolution, 1x1 projection shortcuts at the head of each
+    stage, a 2048 -> 1000 classifier).  They add up to 25 557 032."""
+    sizes: list[int] = []
+
+    def conv_bn(cin: int, cout: int, ksz: int):
+        sizes.extend([cin * cout * ksz * ksz, cout, cout])
+
+    conv_bn(3, 64, 7)
+    cin = 64
+    for width, blocks in ((64, 3), (128, 4), (256, 6), (512, 3)):
+        for block in range(blocks):
+            conv_bn(cin, width, 1)
+            conv_bn(width, width, 3)
+            conv_bn(width, 4 * width, 1)
+            if block == 0:
+                conv_bn(cin, 4 * width, 1)
+            cin = 4 * width
+    sizes.extend([2048 * 1000, 1000])
+    return sizes
+
+
+def layer_offsets(sizes) -> np.ndarray:
+    """int64 [len + 1]: first coordinate of every layer of a flat vector, then its length."""
+    return np.concatenate([[0], np.cumsum(np.asarray(sizes, dtype=np.int64))]).astype(np.int64)
+
+
 # --------------------------------------------------------------------------
 # the five workload shapes (shapes, scales and stepsizes only)
 # --------------------------------------------------------------------------
@@ -162,6 +214,12 @@ class Workload:
     g_var: float = 0.0
     g_mean_var: float = 0.0
     sgd: bool = True
+    layers: str = ""      # "" = Q on the whole row; "resnet20" / "resnet50" = Q per layer
+    a_num: int = 1        # per-layer top-k / random-k keep max(1, floor(a d_l)), a = a_num / a_den
+    a_den: int = 1
+
+    def layer_sizes(self) -> list[int]:
+        return {"resnet20": resnet20_layer_sizes, "resnet50": resnet50_layer_sizes}[self.layers]()
 
     def mixing(self) -> MixingCSR:
         if self.graph == "ring":
@@ -206,6 +264,19 @@ WORKLOADS = {
     "c6_social32_topk": Workload("c6_social32_topk", 32, 272474, "social32", "topk",
                                  k=k_of(1, 100, 272474), eta=0.1, gamma=0.04, steps=1000,
                                  x_var=0.01, g_var=1e-2),
+    # per-layer compression, as in the paper's experiments (Section 5): the same flat vectors
+    # cut into the parameter tensors of the network whose size they have
+    "l3_ring8_sign_layers": Workload("l3_ring8_sign_layers", 8, 272474, "ring", "sign", eta=0.1, gamma=0.4,
+                                     steps=1000, x_var=0.01, g_var=1e-2, layers="resnet20"),
+    "l3_ring8_topk_layers": Workload("l3_ring8_topk_layers", 8, 272474, "ring", "topk", eta=0.1, gamma=0.04,
+                                     steps=1000, x_var=0.01, g_var=1e-2, layers="resnet20",
+                                     a_num=1, a_den=100),
+    "l5_ring32_qsgd_layers": Workload("l5_ring32_qsgd_layers", 32, 25_557_032, "ring", "qsgd", s=16,
+                                      bucket=512, eta=0.1, gamma=0.1, steps=200, x_var=0.01,
+                                      g_var=1e-3, layers="resnet50"),
+    "l5_ring32_topk_layers": Workload("l5_ring32_topk_layers", 32, 25_557_032, "ring", "topk", eta=0.1,
+                                      gamma=0.1, steps=200, x_var=0.01, g_var=1e-3,
+                                      layers="resnet50", a_num=1, a_den=1000),
     # mid-sized dense cases (1 GB of state): small enough for a full counter capture,
     # larger than L2
     "p_ring8_qsgd": Workload("p_ring8_qsgd", 8, 8 * 1024 * 1024, "ring", "qsgd", s=16, bucket=512,
