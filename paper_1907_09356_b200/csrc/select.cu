@@ -19,10 +19,12 @@
 
 namespace choco {
 
-// Rank the candidate bound aims at, in units of k / 256, kept per row: it starts at 2.5 k,
+// Rank the candidate bound aims at, in units of k / 256, kept per row: it starts at 3 k,
 // creeps down to 1.75 k while the guesses keep holding (fewer candidates = less work in the
-// emit kernel) and jumps back to 3 k when a row had to be selected exactly.
-constexpr uint32_t kAimStart = 640u, kAimMin = 448u, kAimAfterMiss = 768u, kAimStep = 8u;
+// emit kernel) and jumps back to 3 k when a row had to be selected exactly.  (A start at
+// 2.5 k missed on 24 row-steps during steps 5-7 of a 32 x 25.6 M top-0.1 % run, where one
+// exact selection from the 102 MB row takes about 30 ms; from 3 k none missed.)
+constexpr uint32_t kAimStart = 768u, kAimMin = 448u, kAimAfterMiss = 768u, kAimStep = 8u;
 
 // value bits of the four coordinates of a quad (top-k: x - x^; random-k: Philox words)
 template <int KIND, bool VEC>
