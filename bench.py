@@ -279,6 +279,10 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if wl.layers:
+        # a stream that can be captured: the layered calls replay steady-state steps from CUDA
+        # graphs, which the legacy default stream does not allow
+        torch.cuda.set_stream(torch.cuda.Stream(device=dev))
 
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234 + rank)
@@ -412,6 +416,8 @@ def main():
             "finite": finite,
             "clocks": clocks,
         }
+        if wl.layers:
+            out["graph_replays"] = int(choco.choco_layers_set_graphs(lay))
         if e2e:
             out["e2e"] = {"value": whole_job_rate(world, N, e2e["steps"], e2e["seconds"]), "unit": "coords/s",
                           "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,

@@ -215,7 +215,11 @@ int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t 
  * layered step gives the same bits as running choco_*_step with d = d_l, seed + l and
  * pointers advanced by layer_off[l] for every layer.  That is also how it is carried out: one
  * library context per layer, their kernels spread over a few internal streams that fork from
- * and join `stream`, so a model of many small layers costs a few kernel launches per layer.
+ * and join `stream`, a few kernel launches per layer.  For TOPK, SIGN and IDENTITY (whose
+ * kernels do not take the step number) a steady-state step is captured into a CUDA graph the
+ * first time it is seen with a given set of arguments (the array pointers, eta, gamma, lambda,
+ * beta) and replayed by one graph launch afterwards; up to 32 such graphs are kept.  A step
+ * call made while `stream` is itself being captured is enqueued kernel by kernel instead.
  *   layer_off[n_layers + 1]   HOST, strictly increasing from 0; ld >= layer_off[n_layers].
  *   a_num, a_den              used by TOPK / RANDK only.
  * Errors are those of choco_init; on error nothing is left allocated.
@@ -238,6 +242,9 @@ int choco_layers_message_bytes(const choco_layers* layers, int64_t* per_worker, 
  * and the like), the layer's first coordinate and its length.  Any output may be NULL. */
 int choco_layers_get_layer(const choco_layers* layers, int32_t layer, choco_ctx** ctx, int64_t* offset,
                            int64_t* length);
+/* enable = 0 / 1 turns the graph replay described above off / on (default on), a negative
+ * value leaves it as it is; *replays (may be NULL) receives the number of steps replayed so far. */
+int choco_layers_set_graphs(choco_layers* layers, int32_t enable, uint64_t* replays);
 /* choco_invalidate / choco_set_step for every layer. */
 int choco_layers_invalidate(choco_layers* layers);
 int choco_layers_set_step(choco_layers* layers, uint64_t t);

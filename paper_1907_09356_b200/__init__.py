@@ -28,7 +28,7 @@ EXPORTS = [
     "choco_last_cuda_error",
     "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
     "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
-    "choco_layers_invalidate", "choco_layers_set_step",
+    "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_graphs",
 ]
 
 
@@ -94,6 +94,7 @@ def load() -> ctypes.CDLL:
                                                ctypes.POINTER(i64)]
         lib.choco_layers_invalidate.argtypes = [vp]
         lib.choco_layers_set_step.argtypes = [vp, u64]
+        lib.choco_layers_set_graphs.argtypes = [vp, i32, ctypes.POINTER(u64)]
         for name in EXPORTS:
             if name not in ("choco_strerror",):
                 getattr(lib, name).restype = ctypes.c_int
@@ -293,6 +294,14 @@ def choco_layers_get_layer(layers, layer: int):
     c, o, n = ctypes.c_void_p(), ctypes.c_int64(), ctypes.c_int64()
     _check(load().choco_layers_get_layer(layers, layer, ctypes.byref(c), ctypes.byref(o), ctypes.byref(n)))
     return c, o.value, n.value
+
+
+def choco_layers_set_graphs(layers, enable: int = -1) -> int:
+    """Turn the CUDA-graph replay of steady-state steps off (0) / on (1), or leave it (-1);
+    returns the number of steps replayed so far."""
+    n = ctypes.c_uint64()
+    _check(load().choco_layers_set_graphs(layers, enable, ctypes.byref(n)))
+    return n.value
 
 
 def choco_layers_invalidate(layers) -> None:

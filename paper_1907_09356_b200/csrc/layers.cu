@@ -5,6 +5,13 @@
 // layers' steps on column slices of the caller's arrays.  The layers are independent of each
 // other, so their kernels are spread over a few internal streams that fork from and join the
 // caller's stream.
+//
+// Many small layers make a step launch-bound (two or three launches per layer).  For the
+// operators whose kernels do not take the step number (top_a, sign, identity) the steady-state
+// step is therefore captured once into a CUDA graph per set of arguments (array pointers, step
+// sizes, message-buffer parity) and replayed with one launch; the host-side bookkeeping of the
+// layers' contexts is advanced by hand after a replay.  gsgd_b and random_a bake the step
+// number into their kernel arguments and always run eagerly.
 #include <cstring>
 #include <new>
 #include <vector>
@@ -13,7 +20,39 @@
 
 namespace {
 
-constexpr int kLayerStreams = 4;
+constexpr int kLayerStreams = 16;
+constexpr size_t kMaxGraphs = 32; // cached step graphs per layered context (least recently used goes)
+
+struct StepGraph {
+    float *X, *Xhat, *S;
+    const float* G;
+    float* M;
+    float eta, gamma, lambda, beta;
+    int parity; // which of the two dense message buffers the step reads
+    cudaGraphExec_t exec;
+    uint64_t last_use;
+};
+
+// the host-side fields of a context that a step changes
+struct HostState {
+    uint64_t step, steps_enqueued;
+    bool prepared;
+    int msg_cur, msg_last;
+    const float *last_x, *last_xhat;
+    unsigned long long launches;
+};
+
+HostState save_state(const choco_ctx* c)
+{
+    return {c->step, c->steps_enqueued, c->prepared, c->msg_cur, c->msg_last, c->last_x, c->last_xhat, c->launches};
+}
+
+void restore_state(choco_ctx* c, const HostState& h)
+{
+    c->step = h.step; c->steps_enqueued = h.steps_enqueued; c->prepared = h.prepared;
+    c->msg_cur = h.msg_cur; c->msg_last = h.msg_last; c->last_x = h.last_x; c->last_xhat = h.last_xhat;
+    c->launches = h.launches;
+}
 
 } // namespace
 
@@ -27,6 +66,11 @@ struct choco_layers {
     cudaEvent_t fork;
     cudaEvent_t join[kLayerStreams];
     int nside;
+    bool graphs_ok;                              // the operator's kernels do not take the step number
+    std::vector<StepGraph> graphs;
+    std::vector<unsigned long long> launches_per_step; // per layer, in the captured steady state
+    uint64_t use_clock;
+    uint64_t replays;
 };
 
 namespace {
@@ -36,6 +80,8 @@ void destroy_layers(choco_layers* L)
     if (!L) return;
     for (choco_ctx* c : L->ctx)
         if (c) choco_destroy(c);
+    for (StepGraph& g : L->graphs)
+        if (g.exec) cudaGraphExecDestroy(g.exec);
     for (int s = 0; s < L->nside; ++s) {
         if (L->side[s]) cudaStreamDestroy(L->side[s]);
         if (L->join[s]) cudaEventDestroy(L->join[s]);
@@ -44,10 +90,9 @@ void destroy_layers(choco_layers* L)
     delete L;
 }
 
-int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
-                float gamma, float lambda, float beta, void* stream)
+int eager_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+               float gamma, float lambda, float beta, void* stream)
 {
-    if (!L || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const bool fan = L->nside > 1 && L->n_layers > 1;
     if (fan) {
@@ -76,6 +121,89 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
     return rc;
 }
 
+// Every layer is in the steady state that a captured step assumes: its next step's compression
+// was prepared by its last step on these very arrays, and nothing asks for per-step events.
+bool steady(const choco_layers* L, const float* X, const float* Xhat)
+{
+    for (int32_t l = 0; l < L->n_layers; ++l) {
+        const choco_ctx* c = L->ctx[l];
+        const int64_t o = L->off[l];
+        if (!c->carry_enabled || !c->prepared || c->last_x != X + o || c->last_xhat != Xhat + o) return false;
+        if (c->prof_ev && c->prof_n < c->prof_cap) return false;
+    }
+    return true;
+}
+
+// What a step call leaves behind on the host side of a context (the end of a step call).
+void advance_after_replay(choco_ctx* c, unsigned long long launches)
+{
+    const bool sparse = c->dv.kind == CHOCO_Q_TOPK || c->dv.kind == CHOCO_Q_RANDK;
+    c->msg_last = c->msg_cur;
+    if (!sparse) c->msg_cur ^= 1;
+    c->step += 1;
+    c->steps_enqueued += 1;
+    c->launches += launches;
+}
+
+int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+                float gamma, float lambda, float beta, void* stream)
+{
+    if (!L || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (!L->graphs_ok || L->n_layers < 2 || cudaStreamIsCapturing(st, &cap) != cudaSuccess ||
+        cap != cudaStreamCaptureStatusNone || !steady(L, X, Xhat))
+        return eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+
+    const int parity = L->ctx[0]->msg_cur; // the layers step together, so they all agree
+    StepGraph* hit = nullptr;
+    for (StepGraph& g : L->graphs)
+        if (g.X == X && g.Xhat == Xhat && g.S == S && g.G == G && g.M == M && g.eta == eta && g.gamma == gamma &&
+            g.lambda == lambda && g.beta == beta && g.parity == parity) { hit = &g; break; }
+    if (hit) {
+        if (cudaGraphLaunch(hit->exec, st) != cudaSuccess) return CHOCO_ERR_CUDA;
+        hit->last_use = ++L->use_clock;
+        for (int32_t l = 0; l < L->n_layers; ++l) advance_after_replay(L->ctx[l], L->launches_per_step[l]);
+        L->replays += 1;
+        return CHOCO_OK;
+    }
+
+    // capture this step; on any failure put the host state back and run it eagerly
+    std::vector<HostState> before(L->n_layers);
+    for (int32_t l = 0; l < L->n_layers; ++l) before[l] = save_state(L->ctx[l]);
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    bool ok = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    if (ok) {
+        const int rc = eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+        const cudaError_t e = cudaStreamEndCapture(st, &graph);
+        ok = rc == CHOCO_OK && e == cudaSuccess && graph != nullptr;
+    }
+    if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
+    if (graph) cudaGraphDestroy(graph);
+    if (ok) ok = cudaGraphLaunch(exec, st) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        if (exec) cudaGraphExecDestroy(exec);
+        for (int32_t l = 0; l < L->n_layers; ++l) restore_state(L->ctx[l], before[l]);
+        L->graphs_ok = false; // do not try again on this context
+        return eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+    }
+    L->launches_per_step.resize(L->n_layers);
+    for (int32_t l = 0; l < L->n_layers; ++l) L->launches_per_step[l] = L->ctx[l]->launches - before[l].launches;
+    StepGraph g = {X, Xhat, S, G, M, eta, gamma, lambda, beta, parity, exec, ++L->use_clock};
+    if (L->graphs.size() < kMaxGraphs) {
+        L->graphs.push_back(g);
+    } else {
+        size_t oldest = 0;
+        for (size_t i = 1; i < L->graphs.size(); ++i)
+            if (L->graphs[i].last_use < L->graphs[oldest].last_use) oldest = i;
+        cudaGraphExecDestroy(L->graphs[oldest].exec);
+        L->graphs[oldest] = g;
+    }
+    return CHOCO_OK;
+}
+
 } // namespace
 
 extern "C" {
@@ -99,6 +227,8 @@ int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int
     L->off.assign(layer_off, layer_off + n_layers + 1);
     L->ctx.assign(n_layers, nullptr);
     L->nside = 0; L->fork = nullptr;
+    L->graphs_ok = p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_SIGN || p->kind == CHOCO_Q_IDENTITY;
+    L->use_clock = 0; L->replays = 0;
     std::memset(L->side, 0, sizeof(L->side));
     std::memset(L->join, 0, sizeof(L->join));
     for (int32_t l = 0; l < n_layers; ++l) {
@@ -169,6 +299,17 @@ int choco_layers_get_layer(const choco_layers* L, int32_t layer, choco_ctx** ctx
     if (ctx) *ctx = L->ctx[layer];
     if (offset) *offset = L->off[layer];
     if (length) *length = L->off[layer + 1] - L->off[layer];
+    return CHOCO_OK;
+}
+
+int choco_layers_set_graphs(choco_layers* L, int32_t enable, uint64_t* replays)
+{
+    if (!L) return CHOCO_ERR_INVALID_ARG;
+    if (replays) *replays = L->replays;
+    if (enable >= 0) {
+        const int kind = L->ctx[0]->dv.kind;
+        L->graphs_ok = enable != 0 && (kind == CHOCO_Q_TOPK || kind == CHOCO_Q_SIGN || kind == CHOCO_Q_IDENTITY);
+    }
     return CHOCO_OK;
 }
 

@@ -3,6 +3,8 @@
 Same acceptance as the plain step: indices, packed bits and level fields bit-exact, float32
 state within 1e-5 * max|x| and, because the operation order is fixed, identical.
 """
+import contextlib
+
 import numpy as np
 import pytest
 import torch
@@ -27,7 +29,10 @@ KINDS = [
 
 
 def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, seed=5,
-         check_layers=()):
+         check_layers=(), stream=None, g_pool=0, invalidate_at=-1):
+    """`stream`: run the steps on that (non-default) stream, where steady-state steps may be
+    replayed from a captured graph; returns the number of steps replayed.  `g_pool` > 0: the
+    gradients live in that many fixed device tensors that are refilled, so pointers repeat."""
     off = workloads.layer_offsets(sizes)
     n, d = w.n, int(off[-1])
     a_num, a_den = kw.get("a", (1, 1))
@@ -41,36 +46,49 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
     p = oracle.Params(kind, s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
     h = choco.choco_layers_init(n, off, ld or d, w.row_ptr, w.col, w.val, kind, a_num, a_den,
                                 s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
+    pool = [_dev(np.zeros_like(X), ld) for _ in range(g_pool)]
+    torch.cuda.synchronize()
+    ctx_mgr = torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
     try:
-        for t in range(steps):
-            G = None if gossip_only else workloads.normal_rows(n, d, 0.01, 100 + t)
-            dG = None if gossip_only else _dev(G, ld)
-            msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t,
-                                      M=M, lam=1e-4, beta=0.9)
-            if gossip_only:
-                choco.choco_layers_gossip_step(h, dX, dXh, dS, 0.2)
-            elif momentum:
-                choco.choco_layers_sgd_momentum_step(h, dX, dXh, dS, dG, dM, 0.05, 0.2, 1e-4, 0.9)
-            else:
-                choco.choco_layers_sgd_step(h, dX, dXh, dS, dG, 0.05, 0.2)
-            torch.cuda.synchronize()
-            for l in check_layers:
-                ctx, o, length = choco.choco_layers_get_layer(h, l)
-                assert (o, length) == (int(off[l]), int(off[l + 1] - off[l]))
-                check_messages(ctx, kind, msgs[l], length)
-            assert_state(_host(dX, d), X, f"X after step {t}")
-            assert_state(_host(dXh, d), Xh, f"Xhat after step {t}")
-            assert_state(_host(dS, d), S, f"S after step {t}")
-            if momentum:
-                assert_state(_host(dM, d), M, f"M after step {t}")
-        per_worker, total = choco.choco_layers_message_bytes(h)
-        assert total == per_worker * n
-        want = sum(next(iter(m.values())).paper_bytes(kind, int(off[l + 1] - off[l]), kw.get("s", 16))
-                   for l, m in enumerate(msgs))
-        assert per_worker == want
-        for l in range(len(sizes)):
-            ctx, _, _ = choco.choco_layers_get_layer(h, l)
-            assert choco.choco_get_stats(ctx)["device_timeouts"] == 0
+        with ctx_mgr:
+            for t in range(steps):
+                G = None if gossip_only else workloads.normal_rows(n, d, 0.01, 100 + t)
+                if gossip_only:
+                    dG = None
+                elif pool:
+                    dG = pool[t % g_pool]
+                    dG[:, :d].copy_(torch.from_numpy(G).to(DEV))
+                else:
+                    dG = _dev(G, ld)
+                if t == invalidate_at:
+                    choco.choco_layers_invalidate(h)
+                msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t,
+                                          M=M, lam=1e-4, beta=0.9)
+                if gossip_only:
+                    choco.choco_layers_gossip_step(h, dX, dXh, dS, 0.2)
+                elif momentum:
+                    choco.choco_layers_sgd_momentum_step(h, dX, dXh, dS, dG, dM, 0.05, 0.2, 1e-4, 0.9)
+                else:
+                    choco.choco_layers_sgd_step(h, dX, dXh, dS, dG, 0.05, 0.2)
+                torch.cuda.synchronize()
+                for l in check_layers:
+                    ctx, o, length = choco.choco_layers_get_layer(h, l)
+                    assert (o, length) == (int(off[l]), int(off[l + 1] - off[l]))
+                    check_messages(ctx, kind, msgs[l], length)
+                assert_state(_host(dX, d), X, f"X after step {t}")
+                assert_state(_host(dXh, d), Xh, f"Xhat after step {t}")
+                assert_state(_host(dS, d), S, f"S after step {t}")
+                if momentum:
+                    assert_state(_host(dM, d), M, f"M after step {t}")
+            per_worker, total = choco.choco_layers_message_bytes(h)
+            assert total == per_worker * n
+            want = sum(next(iter(m.values())).paper_bytes(kind, int(off[l + 1] - off[l]), kw.get("s", 16))
+                       for l, m in enumerate(msgs))
+            assert per_worker == want
+            for l in range(len(sizes)):
+                ctx, _, _ = choco.choco_layers_get_layer(h, l)
+                assert choco.choco_get_stats(ctx)["device_timeouts"] == 0
+            return choco.choco_layers_set_graphs(h)
     finally:
         choco.choco_layers_destroy(h)
 
@@ -89,6 +107,25 @@ def test_resnet20_layers_on_a_ring(kind, kw):
 def test_padded_rows_and_momentum():
     _run(workloads.ring(4), RAGGED, "topk", dict(a=(1, 20)), steps=3, ld=sum(RAGGED) + 11, momentum=True)
     _run(workloads.ring(4), RAGGED, "sign", {}, steps=3, ld=sum(RAGGED) + 8, momentum=True)
+
+
+@pytest.mark.parametrize("kind,kw", [KINDS[0], KINDS[2], KINDS[5]], ids=["topk", "sign", "identity"])
+def test_steady_steps_replayed_from_a_graph_give_the_same_bits(kind, kw):
+    # on a stream that can be captured, with gradient buffers that repeat: the first steps run
+    # kernel by kernel, each new (buffers, parity) combination is captured once, the rest replay
+    replays = _run(workloads.torus(2, 4), RAGGED, kind, kw, steps=12, stream=torch.cuda.Stream(), g_pool=2,
+                   check_layers=(0, 2, 3), invalidate_at=7)
+    assert replays >= 4
+    replays = _run(workloads.ring(4), RAGGED, kind, kw, steps=8, stream=torch.cuda.Stream(), g_pool=1,
+                   momentum=True, ld=sum(RAGGED) + 4)
+    assert replays >= 3
+
+
+def test_operators_keyed_by_the_step_number_are_never_replayed():
+    assert _run(workloads.ring(4), RAGGED, "qsgd", dict(s=16, bucket=512), steps=6,
+                stream=torch.cuda.Stream(), g_pool=1) == 0
+    assert _run(workloads.ring(4), RAGGED, "randk", dict(a=(1, 20)), steps=6,
+                stream=torch.cuda.Stream(), g_pool=1) == 0
 
 
 def test_gossip_only_layers():
