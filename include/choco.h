@@ -215,11 +215,13 @@ int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t 
  * layered step gives the same bits as running choco_*_step with d = d_l, seed + l and
  * pointers advanced by layer_off[l] for every layer.  That is also how it is carried out: one
  * library context per layer, their kernels spread over a few internal streams that fork from
- * and join `stream`, a few kernel launches per layer.  For TOPK, SIGN and IDENTITY (whose
- * kernels do not take the step number) a steady-state step is captured into a CUDA graph the
- * first time it is seen with a given set of arguments (the array pointers, eta, gamma, lambda,
- * beta) and replayed by one graph launch afterwards; up to 32 such graphs are kept.  A step
- * call made while `stream` is itself being captured is enqueued kernel by kernel instead.
+ * and join `stream`, a few kernel launches per layer.  A steady-state step is captured into a
+ * CUDA graph the first time it is seen with a given set of arguments (the array pointers, eta,
+ * gamma, lambda, beta) and replayed by one graph launch afterwards; up to 32 such graphs are
+ * kept.  (QSGD and RANDK contexts of a layered context keep the step number in device memory
+ * for this and bump it with one more tiny kernel per step.)  A step call made while `stream`
+ * is itself being captured, or on the legacy default stream, which cannot be captured, is
+ * enqueued kernel by kernel instead.
  *   layer_off[n_layers + 1]   HOST, strictly increasing from 0; ld >= layer_off[n_layers].
  *   a_num, a_den              used by TOPK / RANDK only.
  * Errors are those of choco_init; on error nothing is left allocated.

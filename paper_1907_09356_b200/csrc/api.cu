@@ -106,6 +106,8 @@ void keep_hot_in_l2(choco_ctx* ctx, cudaStream_t st)
     cudaGetLastError(); // best effort
 }
 
+__global__ void bump_step_kernel(unsigned long long* step) { *step += 1ull; }
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
 
@@ -128,6 +130,7 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     a.X = X; a.Xhat = Xhat; a.S = S; a.G = G; a.M = M;
     a.eta = eta; a.gamma = gamma; a.lambda = lambda; a.beta = beta;
     a.step = ctx->step;
+    a.step_dev = ctx->dev_step ? ctx->step_dev : nullptr;
     a.launches = &ctx->launches;
     a.vec = (dv.ld % 4 == 0) && aligned16(X) && aligned16(Xhat) && aligned16(S) &&
             (!G || aligned16(G)) && (!M || aligned16(M));
@@ -155,6 +158,11 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     }
     if (e == cudaSuccess && emit && dv.kind == CHOCO_Q_SIGN) {
         e = launch_next_sign_scale(dv, st);
+        ctx->launches += 1;
+    }
+    if (e == cudaSuccess && ctx->dev_step) {
+        bump_step_kernel<<<1, 1, 0, st>>>(ctx->step_dev);
+        e = cudaGetLastError();
         ctx->launches += 1;
     }
     if (e != cudaSuccess) return fail_cuda(ctx, e);
@@ -245,6 +253,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         dv.rd_pos = dpos; dv.rd_w = drw;
     }
     if (e == cudaSuccess) e = dev_alloc(ctx, &dv.stats, 1);
+    if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->step_dev, 1); // zeroed, as the step counter is
 
     const int64_t nwords = (d + 31) / 32;
     if (p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK) {
@@ -452,6 +461,12 @@ int choco_set_step(choco_ctx* ctx, uint64_t t)
 {
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
     if (t >> 56) return CHOCO_ERR_TOO_LARGE;
+    if (ctx->dev_step) {
+        const unsigned long long v = t;
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e == cudaSuccess) e = cudaMemcpy(ctx->step_dev, &v, sizeof(v), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
     ctx->step = t;
     ctx->prepared = false;
     return CHOCO_OK;

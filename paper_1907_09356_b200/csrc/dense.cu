@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) qsgd_pack_kernel(Dev dv, StepArgs a)
         } else {
             nu = dv.msg_norms[(int64_t)row * dv.npitch];
         }
-        const uint4 rw = coord_words(dv.seed, a.step, (uint32_t)row, kStreamDither, c);
+        const uint4 rw = coord_words(dv.seed, step_of(a), (uint32_t)row, kStreamDither, c);
         const float u[4] = {word_to_unit(rw.x), word_to_unit(rw.y), word_to_unit(rw.z),
                             word_to_unit(rw.w)};
         const float vv[4] = {v[it].x, v[it].y, v[it].z, v[it].w};

@@ -111,9 +111,19 @@ struct StepArgs {
     float* M;                    // momentum memory, may be null
     float eta, gamma, lambda, beta;
     uint64_t step;
+    const unsigned long long* step_dev; // if set, the step number is read from here instead
     bool vec;                    // rows 16-byte aligned: 128-bit accesses
     unsigned long long* launches; // host counter of kernels enqueued (not used on the device)
 };
+
+#ifdef __CUDACC__
+// The step number that keys the generator.  A context may keep it in device memory (and bump it
+// there after every step) so that a captured launch sequence stays valid from step to step.
+__device__ __forceinline__ uint64_t step_of(const StepArgs& a)
+{
+    return a.step_dev ? (uint64_t)*a.step_dev : a.step;
+}
+#endif
 
 // selection (top-k / random-k)
 cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t st);
@@ -141,6 +151,8 @@ struct choco_ctx {
     choco::Dev dv;
     choco_params params;
     uint64_t step;
+    unsigned long long* step_dev; // device copy of `step`, kept equal to it while dev_step is set
+    bool dev_step;               // kernels read the step number from step_dev (layered contexts)
     uint64_t steps_enqueued;
     int device;
     int last_cuda_error;

@@ -6,12 +6,12 @@
 // other, so their kernels are spread over a few internal streams that fork from and join the
 // caller's stream.
 //
-// Many small layers make a step launch-bound (two or three launches per layer).  For the
-// operators whose kernels do not take the step number (top_a, sign, identity) the steady-state
-// step is therefore captured once into a CUDA graph per set of arguments (array pointers, step
-// sizes, message-buffer parity) and replayed with one launch; the host-side bookkeeping of the
-// layers' contexts is advanced by hand after a replay.  gsgd_b and random_a bake the step
-// number into their kernel arguments and always run eagerly.
+// Many small layers make a step launch-bound (two or three launches per layer).  The
+// steady-state step is therefore captured once into a CUDA graph per set of arguments (array
+// pointers, step sizes, message-buffer parity) and replayed with one launch; the host-side
+// bookkeeping of the layers' contexts is advanced by hand after a replay.  gsgd_b and random_a
+// key their generator with the step number, which a captured kernel argument would freeze:
+// their contexts keep the step number in device memory and bump it there after every step.
 #include <cstring>
 #include <new>
 #include <vector>
@@ -28,7 +28,7 @@ struct StepGraph {
     const float* G;
     float* M;
     float eta, gamma, lambda, beta;
-    int parity; // which of the two dense message buffers the step reads
+    uint64_t mode; // hash over the layers of (compression carried, message buffer in use)
     cudaGraphExec_t exec;
     uint64_t last_use;
 };
@@ -66,7 +66,7 @@ struct choco_layers {
     cudaEvent_t fork;
     cudaEvent_t join[kLayerStreams];
     int nside;
-    bool graphs_ok;                              // the operator's kernels do not take the step number
+    bool graphs_ok;                              // steady-state steps may be captured and replayed
     std::vector<StepGraph> graphs;
     std::vector<unsigned long long> launches_per_step; // per layer, in the captured steady state
     uint64_t use_clock;
@@ -121,16 +121,26 @@ int eager_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G,
     return rc;
 }
 
-// Every layer is in the steady state that a captured step assumes: its next step's compression
-// was prepared by its last step on these very arrays, and nothing asks for per-step events.
-bool steady(const choco_layers* L, const float* X, const float* Xhat)
+// A captured step can stand for the next one if every layer is in a state that repeats: its
+// next step's compression was prepared by its last step on these very arrays (operators that
+// carry it across steps), or it compresses afresh every step (random_a, whole-row gsgd_b, or
+// carrying turned off); and nothing asks for per-step events.  `mode` receives a hash of what
+// selects the kernels and message buffers of the layers, part of a graph's key.
+bool steady(const choco_layers* L, const float* X, const float* Xhat, uint64_t* mode)
 {
+    uint64_t h = 1469598103934665603ull;
+    const choco::StepArgs none = {};
     for (int32_t l = 0; l < L->n_layers; ++l) {
         const choco_ctx* c = L->ctx[l];
         const int64_t o = L->off[l];
-        if (!c->carry_enabled || !c->prepared || c->last_x != X + o || c->last_xhat != Xhat + o) return false;
+        if (c->steps_enqueued == 0) return false; // the first step also sets the kernels up
+        const bool carries = c->carry_enabled && choco::apply_can_emit(c->dv, none);
+        if (c->prepared != carries) return false;
+        if (c->prepared && (c->last_x != X + o || c->last_xhat != Xhat + o)) return false;
         if (c->prof_ev && c->prof_n < c->prof_cap) return false;
+        h = (h ^ (uint64_t)((c->prepared ? 1 : 0) | (c->msg_cur << 1))) * 1099511628211ull;
     }
+    *mode = h;
     return true;
 }
 
@@ -139,7 +149,7 @@ void advance_after_replay(choco_ctx* c, unsigned long long launches)
 {
     const bool sparse = c->dv.kind == CHOCO_Q_TOPK || c->dv.kind == CHOCO_Q_RANDK;
     c->msg_last = c->msg_cur;
-    if (!sparse) c->msg_cur ^= 1;
+    if (c->prepared && !sparse) c->msg_cur ^= 1; // the step wrote the next messages into the other buffer
     c->step += 1;
     c->steps_enqueued += 1;
     c->launches += launches;
@@ -151,15 +161,15 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
     if (!L || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    uint64_t mode = 0;
     if (!L->graphs_ok || L->n_layers < 2 || cudaStreamIsCapturing(st, &cap) != cudaSuccess ||
-        cap != cudaStreamCaptureStatusNone || !steady(L, X, Xhat))
+        cap != cudaStreamCaptureStatusNone || !steady(L, X, Xhat, &mode))
         return eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
 
-    const int parity = L->ctx[0]->msg_cur; // the layers step together, so they all agree
     StepGraph* hit = nullptr;
     for (StepGraph& g : L->graphs)
         if (g.X == X && g.Xhat == Xhat && g.S == S && g.G == G && g.M == M && g.eta == eta && g.gamma == gamma &&
-            g.lambda == lambda && g.beta == beta && g.parity == parity) { hit = &g; break; }
+            g.lambda == lambda && g.beta == beta && g.mode == mode) { hit = &g; break; }
     if (hit) {
         if (cudaGraphLaunch(hit->exec, st) != cudaSuccess) return CHOCO_ERR_CUDA;
         hit->last_use = ++L->use_clock;
@@ -191,7 +201,7 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
     }
     L->launches_per_step.resize(L->n_layers);
     for (int32_t l = 0; l < L->n_layers; ++l) L->launches_per_step[l] = L->ctx[l]->launches - before[l].launches;
-    StepGraph g = {X, Xhat, S, G, M, eta, gamma, lambda, beta, parity, exec, ++L->use_clock};
+    StepGraph g = {X, Xhat, S, G, M, eta, gamma, lambda, beta, mode, exec, ++L->use_clock};
     if (L->graphs.size() < kMaxGraphs) {
         L->graphs.push_back(g);
     } else {
@@ -227,7 +237,7 @@ int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int
     L->off.assign(layer_off, layer_off + n_layers + 1);
     L->ctx.assign(n_layers, nullptr);
     L->nside = 0; L->fork = nullptr;
-    L->graphs_ok = p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_SIGN || p->kind == CHOCO_Q_IDENTITY;
+    L->graphs_ok = true;
     L->use_clock = 0; L->replays = 0;
     std::memset(L->side, 0, sizeof(L->side));
     std::memset(L->join, 0, sizeof(L->join));
@@ -241,6 +251,9 @@ int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int
         }
         const int rc = choco_init(&L->ctx[l], n, dl, ld, w_row_ptr, w_col, w_val, &pl, seed + (uint64_t)l);
         if (rc != CHOCO_OK) { destroy_layers(L); return rc; }
+        // gsgd_b and random_a key their generator with the step number: these contexts keep it
+        // in device memory, where a replayed graph finds the current value
+        L->ctx[l]->dev_step = p->kind == CHOCO_Q_QSGD || p->kind == CHOCO_Q_RANDK;
     }
     bool ok = cudaEventCreateWithFlags(&L->fork, cudaEventDisableTiming) == cudaSuccess;
     for (int s = 0; s < kLayerStreams && ok; ++s) {
@@ -306,10 +319,7 @@ int choco_layers_set_graphs(choco_layers* L, int32_t enable, uint64_t* replays)
 {
     if (!L) return CHOCO_ERR_INVALID_ARG;
     if (replays) *replays = L->replays;
-    if (enable >= 0) {
-        const int kind = L->ctx[0]->dv.kind;
-        L->graphs_ok = enable != 0 && (kind == CHOCO_Q_TOPK || kind == CHOCO_Q_SIGN || kind == CHOCO_Q_IDENTITY);
-    }
+    if (enable >= 0) L->graphs_ok = enable != 0;
     return CHOCO_OK;
 }
 

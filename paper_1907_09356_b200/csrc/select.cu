@@ -39,7 +39,7 @@ __device__ __forceinline__ void quad_bits(const Dev& dv, const StepArgs& a, int 
         out[2] = __float_as_uint(__fsub_rn(x.z, h.z));
         out[3] = __float_as_uint(__fsub_rn(x.w, h.w));
     } else {
-        const uint4 w = coord_words(dv.seed, a.step, (uint32_t)row, kStreamRandK, c);
+        const uint4 w = coord_words(dv.seed, step_of(a), (uint32_t)row, kStreamRandK, c);
         out[0] = w.x; out[1] = w.y; out[2] = w.z; out[3] = w.w;
     }
 }

@@ -284,7 +284,7 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         if (lane == 0 && warp == w0 && bucket < dv.nbuckets)
             dv.nxt_norms[(int64_t)row * dv.npitch + bucket] = nu;
         // the dither of the message that the NEXT step applies
-        const uint4 rw = coord_words(dv.seed, a.step + 1, (uint32_t)row, kStreamDither, c);
+        const uint4 rw = coord_words(dv.seed, step_of(a) + 1, (uint32_t)row, kStreamDither, c);
         const float uu[4] = {word_to_unit(rw.x), word_to_unit(rw.y), word_to_unit(rw.z), word_to_unit(rw.w)};
         const float vv[4] = {vn[it].x, vn[it].y, vn[it].z, vn[it].w};
         uint32_t lev[4] = {0u, 0u, 0u, 0u};

@@ -29,10 +29,11 @@ KINDS = [
 
 
 def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, seed=5,
-         check_layers=(), stream=None, g_pool=0, invalidate_at=-1):
+         check_layers=(), stream=None, g_pool=0, invalidate_at=-1, jump=None):
     """`stream`: run the steps on that (non-default) stream, where steady-state steps may be
     replayed from a captured graph; returns the number of steps replayed.  `g_pool` > 0: the
-    gradients live in that many fixed device tensors that are refilled, so pointers repeat."""
+    gradients live in that many fixed device tensors that are refilled, so pointers repeat.
+    `jump` = (i, t): before the i-th call the step number is set to t on both sides."""
     off = workloads.layer_offsets(sizes)
     n, d = w.n, int(off[-1])
     a_num, a_den = kw.get("a", (1, 1))
@@ -47,6 +48,7 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
     h = choco.choco_layers_init(n, off, ld or d, w.row_ptr, w.col, w.val, kind, a_num, a_den,
                                 s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
     pool = [_dev(np.zeros_like(X), ld) for _ in range(g_pool)]
+    t_shift = 0
     torch.cuda.synchronize()
     ctx_mgr = torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
     try:
@@ -62,7 +64,10 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
                     dG = _dev(G, ld)
                 if t == invalidate_at:
                     choco.choco_layers_invalidate(h)
-                msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t,
+                if jump and t == jump[0]:
+                    t_shift = jump[1] - t
+                    choco.choco_layers_set_step(h, jump[1])
+                msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t + t_shift,
                                           M=M, lam=1e-4, beta=0.9)
                 if gossip_only:
                     choco.choco_layers_gossip_step(h, dX, dXh, dS, 0.2)
@@ -121,11 +126,12 @@ def test_steady_steps_replayed_from_a_graph_give_the_same_bits(kind, kw):
     assert replays >= 3
 
 
-def test_operators_keyed_by_the_step_number_are_never_replayed():
-    assert _run(workloads.ring(4), RAGGED, "qsgd", dict(s=16, bucket=512), steps=6,
-                stream=torch.cuda.Stream(), g_pool=1) == 0
-    assert _run(workloads.ring(4), RAGGED, "randk", dict(a=(1, 20)), steps=6,
-                stream=torch.cuda.Stream(), g_pool=1) == 0
+@pytest.mark.parametrize("kind,kw", [KINDS[1], KINDS[3], KINDS[4]], ids=["randk", "qsgd512", "qsgd-row"])
+def test_replayed_steps_of_operators_keyed_by_the_step_number(kind, kw):
+    # their generator takes the step number; a replayed launch must see the current one
+    replays = _run(workloads.torus(2, 4), RAGGED, kind, kw, steps=10, stream=torch.cuda.Stream(), g_pool=2,
+                   check_layers=(0, 2, 3), invalidate_at=6, jump=(4, 1000))
+    assert replays >= 3
 
 
 def test_gossip_only_layers():
