@@ -279,9 +279,10 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    if wl.layers:
-        # a stream that can be captured: the layered calls replay steady-state steps from CUDA
-        # graphs, which the legacy default stream does not allow
+    small = N <= (1 << 22)      # the library replays such problems' steps from CUDA graphs
+    if wl.layers or small:
+        # a stream that can be captured: steady-state steps are replayed from CUDA graphs,
+        # which the legacy default stream does not allow
         torch.cuda.set_stream(torch.cuda.Stream(device=dev))
 
     gen = torch.Generator(device=dev)
@@ -325,7 +326,7 @@ def main():
         do_step(pool[t % pool_n])
     barrier()
     st0 = stats_sum()
-    if not wl.layers:
+    if not wl.layers and not small:
         choco.choco_profile_enable(ch.ctx, args.steps)
         choco.choco_profile_set_stride(ch.ctx, args.profile_stride)   # events between kernels cost time
     sampler = ClockSampler(local_rank)
@@ -344,7 +345,7 @@ def main():
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     st1 = stats_sum()
-    nrec, upd_ms = (0, 0.0) if wl.layers else choco.choco_profile_read(ch.ctx)
+    nrec, upd_ms = (0, 0.0) if (wl.layers or small) else choco.choco_profile_read(ch.ctx)
     finite = bool(torch.isfinite(X).all())
 
     # end to end: host buffers in, host buffers out, through choco_sgd_step_host
@@ -389,10 +390,12 @@ def main():
         step_bytes = step_min_bytes(wl, w)
         step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
         roof_kernel = "update (apply) kernel"
-        if wl.layers:
-            # one small set of kernels per layer: no single dominant launch to time, so the
-            # roofline entry is the whole step (all layers' kernels) against its minimum bytes
-            roof_kernel = "whole step: the kernels of all layers"
+        if wl.layers or small:
+            # one small set of kernels per layer, or a few short kernels replayed from a graph
+            # (events between them would prevent that): no single dominant launch to time, so
+            # the roofline entry is the whole step against its minimum bytes
+            roof_kernel = ("whole step: the kernels of all layers" if wl.layers
+                           else "whole step (state fits L2; replayed from a CUDA graph)")
             achieved, upd_bytes, upd_avg_s, nrec = step_gbs, step_bytes, ms_step * 1e-3, args.steps
         out = {
             "metric": "coords_per_sec", "value": value, "unit": "coords/s", "n_gpus": args.gpus,
@@ -418,6 +421,8 @@ def main():
         }
         if wl.layers:
             out["graph_replays"] = int(choco.choco_layers_set_graphs(lay))
+        else:
+            out["graph_replays"] = int(st1["graph_replays"] - st0["graph_replays"])
         if e2e:
             out["e2e"] = {"value": whole_job_rate(world, N, e2e["steps"], e2e["seconds"]), "unit": "coords/s",
                           "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,

@@ -144,6 +144,21 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
 int choco_invalidate(choco_ctx* ctx);
 int choco_set_carry(choco_ctx* ctx, int32_t enable);
 
+/*
+ * Small problems (n d <= 4 194 304), where a step is a few short kernels whose launches take
+ * longer than their work, replay their steady-state step from a CUDA graph: the second time a
+ * step call is seen with a given set of arguments (array pointers, eta, gamma, lambda, beta) in
+ * the state that repeats (see choco_invalidate above) its kernels are captured, later calls
+ * launch the graph; up to 16 graphs per context.  (A caller that passes a newly allocated
+ * gradient array every step therefore never triggers a capture, and gains nothing.)  Results
+ * are the same bits either way.  Not used on the legacy default stream (NULL), which cannot be
+ * captured, nor while `stream` is itself being captured, nor while choco_profile_enable is
+ * recording.  QSGD and RANDK contexts that replay keep the step number in device memory and
+ * bump it with one tiny kernel per step.
+ * choco_set_graphs -- enable = 0 / 1 turns this off / on for a context of any size.
+ */
+int choco_set_graphs(choco_ctx* ctx, int32_t enable);
+
 /* Step counter t (keys the generator).  Setting it, together with restoring X, Xhat and S,
  * resumes a run bit-exactly; choco_set_step implies choco_invalidate. */
 int choco_get_step(const choco_ctx* ctx, uint64_t* t);
@@ -216,7 +231,7 @@ int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t 
  * pointers advanced by layer_off[l] for every layer.  That is also how it is carried out: one
  * library context per layer, their kernels spread over a few internal streams that fork from
  * and join `stream`, a few kernel launches per layer.  A steady-state step is captured into a
- * CUDA graph the first time it is seen with a given set of arguments (the array pointers, eta,
+ * CUDA graph the second time it is seen with a given set of arguments (the array pointers, eta,
  * gamma, lambda, beta) and replayed by one graph launch afterwards; up to 32 such graphs are
  * kept.  (QSGD and RANDK contexts of a layered context keep the step number in device memory
  * for this and bump it with one more tiny kernel per step.)  A step call made while `stream`
@@ -259,6 +274,7 @@ typedef struct {
     uint64_t exact_rows;       /* rows that needed the slow exact selection                    */
     uint64_t kernel_launches;  /* kernels the step calls have enqueued                         */
     uint64_t device_timeouts;  /* bounded waits inside kernels that ran out (must stay 0)      */
+    uint64_t graph_replays;    /* step calls served by replaying a captured CUDA graph          */
 } choco_stats;
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
 

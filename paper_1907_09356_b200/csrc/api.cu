@@ -111,8 +111,8 @@ __global__ void bump_step_kernel(unsigned long long* step) { *step += 1ull; }
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
 
-int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
-             float gamma, float lambda, float beta, void* stream)
+int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+              float gamma, float lambda, float beta, void* stream)
 {
     if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
     if (!aligned4(X) || !aligned4(Xhat) || !aligned4(S) || !aligned4(G) || !aligned4(M))
@@ -176,7 +176,114 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     return CHOCO_OK;
 }
 
+// The host-side fields a step changes, to undo a capture that failed.
+struct HostState {
+    uint64_t step, steps_enqueued;
+    bool prepared;
+    int msg_cur, msg_last;
+    const float *last_x, *last_xhat;
+    unsigned long long launches;
+};
+
+// A step call: small problems replay their steady-state step from a CUDA graph captured the
+// second time a set of arguments is seen (a step there is a few short kernels, and launching
+// them one by one takes longer than running them); everything else is enqueued kernel by kernel.
+int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
+             float gamma, float lambda, float beta, void* stream)
+{
+    if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint64_t mode = 0;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    // the legacy default stream (NULL or cudaStreamLegacy) cannot be captured
+    if (!ctx->graphs_ok || st == nullptr || st == cudaStreamLegacy || !step_repeats(ctx, X, Xhat, &mode) ||
+        cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone)
+        return step_body(ctx, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+    // A set of arguments is captured the second time it is seen: a caller that passes new
+    // arrays every step (a fresh gradient tensor, say) never pays for a capture.
+    int slot = -1;
+    for (int i = 0; i < ctx->ngraphs; ++i) {
+        const choco_step_graph& g = ctx->graphs[i];
+        if (g.X == X && g.Xhat == Xhat && g.S == S && g.G == G && g.M == M && g.eta == eta && g.gamma == gamma &&
+            g.lambda == lambda && g.beta == beta && g.mode == mode) { slot = i; break; }
+    }
+    if (slot >= 0 && ctx->graphs[slot].exec) {
+        choco_step_graph& g = ctx->graphs[slot];
+        const cudaError_t e = cudaGraphLaunch(g.exec, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        g.last_use = ++ctx->graph_clock;
+        advance_after_replay(ctx, ctx->launches_per_step);
+        ctx->graph_replays += 1;
+        return CHOCO_OK;
+    }
+    if (slot < 0) { // first sighting: remember it, enqueue kernel by kernel
+        slot = ctx->ngraphs;
+        if (slot < kCtxGraphs) {
+            ctx->ngraphs += 1;
+        } else {
+            slot = 0;
+            for (int i = 1; i < kCtxGraphs; ++i)
+                if (ctx->graphs[i].last_use < ctx->graphs[slot].last_use) slot = i;
+            if (ctx->graphs[slot].exec) cudaGraphExecDestroy(ctx->graphs[slot].exec);
+        }
+        ctx->graphs[slot] = {X, Xhat, S, G, M, eta, gamma, lambda, beta, mode, nullptr, ++ctx->graph_clock};
+        return step_body(ctx, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+    }
+    const HostState before = {ctx->step, ctx->steps_enqueued, ctx->prepared, ctx->msg_cur, ctx->msg_last,
+                              ctx->last_x, ctx->last_xhat, ctx->launches};
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    bool ok = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    if (ok) {
+        const int rc = step_body(ctx, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+        const cudaError_t e = cudaStreamEndCapture(st, &graph);
+        ok = rc == CHOCO_OK && e == cudaSuccess && graph != nullptr;
+    }
+    if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
+    if (graph) cudaGraphDestroy(graph);
+    if (ok) ok = cudaGraphLaunch(exec, st) == cudaSuccess;
+    if (!ok) { // put the host state back, give graphs up for this context, enqueue the step as usual
+        cudaGetLastError();
+        if (exec) cudaGraphExecDestroy(exec);
+        ctx->step = before.step; ctx->steps_enqueued = before.steps_enqueued; ctx->prepared = before.prepared;
+        ctx->msg_cur = before.msg_cur; ctx->msg_last = before.msg_last; ctx->last_x = before.last_x;
+        ctx->last_xhat = before.last_xhat; ctx->launches = before.launches;
+        ctx->graphs_ok = false;
+        return step_body(ctx, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
+    }
+    ctx->launches_per_step = ctx->launches - before.launches;
+    ctx->graphs[slot].exec = exec;
+    ctx->graphs[slot].last_use = ++ctx->graph_clock;
+    return CHOCO_OK;
+}
+
 } // namespace
+
+namespace choco {
+
+bool step_repeats(const choco_ctx* c, const float* X, const float* Xhat, uint64_t* mode)
+{
+    if (c->steps_enqueued == 0) return false; // the first step also sets the kernels up
+    const StepArgs none = {};
+    const bool carries = c->carry_enabled && apply_can_emit(c->dv, none);
+    if (c->prepared != carries) return false;
+    if (c->prepared && (c->last_x != X || c->last_xhat != Xhat)) return false;
+    if (c->prof_ev && c->prof_n < c->prof_cap) return false;
+    *mode = (uint64_t)((c->prepared ? 1 : 0) | (c->msg_cur << 1));
+    return true;
+}
+
+void advance_after_replay(choco_ctx* c, unsigned long long launches)
+{
+    const bool sparse = c->dv.kind == CHOCO_Q_TOPK || c->dv.kind == CHOCO_Q_RANDK;
+    c->msg_last = c->msg_cur;
+    if (c->prepared && !sparse) c->msg_cur ^= 1; // the step wrote the next messages into the other buffer
+    c->step += 1;
+    c->steps_enqueued += 1;
+    c->launches += launches;
+}
+
+} // namespace choco
 
 extern "C" {
 
@@ -214,6 +321,10 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     std::memset(ctx, 0, sizeof(*ctx));
     ctx->params = *p;
     ctx->carry_enabled = true;
+    ctx->graphs_ok = (int64_t)n * d <= kGraphCoords;
+    // gsgd_b and random_a key their generator with the step number, which a captured kernel
+    // argument would freeze: such contexts keep it in device memory and bump it there
+    ctx->dev_step = ctx->graphs_ok && (p->kind == CHOCO_Q_QSGD || p->kind == CHOCO_Q_RANDK);
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
     dv.ntiles = (d + kTile - 1) / kTile;
@@ -369,6 +480,8 @@ int choco_destroy(choco_ctx* ctx)
 {
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
     for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
     for (int i = 0; i < 4; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
@@ -420,7 +533,7 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
     ctx->prepared = false; // the staging contents changed
     const bool carry = ctx->carry_enabled;
     ctx->carry_enabled = false; // the next call overwrites the staging buffers anyway
-    const int rc = run_step(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], G ? ctx->stage[3] : nullptr,
+    const int rc = step_body(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], G ? ctx->stage[3] : nullptr,
                             nullptr, eta, gamma, 0.f, 0.f, stream);
     ctx->carry_enabled = carry;
     if (rc) return rc;
@@ -447,6 +560,22 @@ int choco_set_carry(choco_ctx* ctx, int32_t enable)
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
     ctx->carry_enabled = enable != 0;
     ctx->prepared = false;
+    return CHOCO_OK;
+}
+
+int choco_set_graphs(choco_ctx* ctx, int32_t enable)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    if (enable && !ctx->graphs_ok && (ctx->dv.kind == CHOCO_Q_QSGD || ctx->dv.kind == CHOCO_Q_RANDK) &&
+        !ctx->dev_step) {
+        // from now on the kernels read the step number from device memory: bring it up to date
+        const unsigned long long v = ctx->step;
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e == cudaSuccess) e = cudaMemcpy(ctx->step_dev, &v, sizeof(v), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->dev_step = true;
+    }
+    ctx->graphs_ok = enable != 0;
     return CHOCO_OK;
 }
 
@@ -555,6 +684,7 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
     out->exact_rows = h.exact_rows;
     out->device_timeouts = h.timeouts;
     out->kernel_launches = ctx->launches;
+    out->graph_replays = ctx->graph_replays;
     return CHOCO_OK;
 }
 

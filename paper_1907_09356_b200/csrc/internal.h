@@ -147,6 +147,32 @@ cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, d
 
 } // namespace choco
 
+struct choco_ctx;
+namespace choco {
+// True if the context's next step will enqueue the same kernels, on the same buffers, as its
+// last one did: its compression was prepared by the last step on these very arrays (operators
+// that carry it across steps), or it compresses afresh every step; and no per-step events are
+// asked for.  *mode receives what else selects kernels and message buffers.
+bool step_repeats(const choco_ctx* ctx, const float* X, const float* Xhat, uint64_t* mode);
+// The host-side effects of one step call, for a step that was replayed from a graph.
+void advance_after_replay(choco_ctx* ctx, unsigned long long launches);
+} // namespace choco
+
+// A captured steady-state step of one context, kept for replay (small problems, where a step
+// is a few short kernels and their launches dominate).  exec == nullptr: the arguments were
+// seen once and will be captured when they come again.
+struct choco_step_graph {
+    float *X, *Xhat, *S;
+    const float* G;
+    float* M;
+    float eta, gamma, lambda, beta;
+    uint64_t mode;               // (compression carried, message buffer in use)
+    cudaGraphExec_t exec;
+    uint64_t last_use;
+};
+constexpr int kCtxGraphs = 16;   // per context; the least recently used one is replaced
+constexpr int64_t kGraphCoords = (int64_t)1 << 22; // contexts with n d up to this replay graphs
+
 struct choco_ctx {
     choco::Dev dv;
     choco_params params;
@@ -180,6 +206,12 @@ struct choco_ctx {
     // optional event pairs around the update kernel
     cudaEvent_t* prof_ev;
     int prof_cap, prof_n, prof_stride;
+    // replay of captured steady-state steps (see choco_step_graph)
+    bool graphs_ok;
+    choco_step_graph graphs[kCtxGraphs];
+    int ngraphs;
+    uint64_t graph_clock, graph_replays;
+    unsigned long long launches_per_step; // kernels in a captured step
     // all device allocations, for choco_destroy
     void* allocs[64];
     int nallocs;

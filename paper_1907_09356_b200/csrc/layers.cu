@@ -121,38 +121,18 @@ int eager_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G,
     return rc;
 }
 
-// A captured step can stand for the next one if every layer is in a state that repeats: its
-// next step's compression was prepared by its last step on these very arrays (operators that
-// carry it across steps), or it compresses afresh every step (random_a, whole-row gsgd_b, or
-// carrying turned off); and nothing asks for per-step events.  `mode` receives a hash of what
-// selects the kernels and message buffers of the layers, part of a graph's key.
+// A captured step can stand for the next one if every layer's step repeats; `mode` receives a
+// hash of what selects the kernels and message buffers of the layers, part of a graph's key.
 bool steady(const choco_layers* L, const float* X, const float* Xhat, uint64_t* mode)
 {
     uint64_t h = 1469598103934665603ull;
-    const choco::StepArgs none = {};
     for (int32_t l = 0; l < L->n_layers; ++l) {
-        const choco_ctx* c = L->ctx[l];
-        const int64_t o = L->off[l];
-        if (c->steps_enqueued == 0) return false; // the first step also sets the kernels up
-        const bool carries = c->carry_enabled && choco::apply_can_emit(c->dv, none);
-        if (c->prepared != carries) return false;
-        if (c->prepared && (c->last_x != X + o || c->last_xhat != Xhat + o)) return false;
-        if (c->prof_ev && c->prof_n < c->prof_cap) return false;
-        h = (h ^ (uint64_t)((c->prepared ? 1 : 0) | (c->msg_cur << 1))) * 1099511628211ull;
+        uint64_t m = 0;
+        if (!choco::step_repeats(L->ctx[l], X + L->off[l], Xhat + L->off[l], &m)) return false;
+        h = (h ^ m) * 1099511628211ull;
     }
     *mode = h;
     return true;
-}
-
-// What a step call leaves behind on the host side of a context (the end of a step call).
-void advance_after_replay(choco_ctx* c, unsigned long long launches)
-{
-    const bool sparse = c->dv.kind == CHOCO_Q_TOPK || c->dv.kind == CHOCO_Q_RANDK;
-    c->msg_last = c->msg_cur;
-    if (c->prepared && !sparse) c->msg_cur ^= 1; // the step wrote the next messages into the other buffer
-    c->step += 1;
-    c->steps_enqueued += 1;
-    c->launches += launches;
 }
 
 int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
@@ -166,16 +146,31 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
         cap != cudaStreamCaptureStatusNone || !steady(L, X, Xhat, &mode))
         return eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
 
+    // A set of arguments is captured the second time it is seen: a caller that passes new
+    // arrays every step (a fresh gradient tensor, say) never pays for a capture.
     StepGraph* hit = nullptr;
     for (StepGraph& g : L->graphs)
         if (g.X == X && g.Xhat == Xhat && g.S == S && g.G == G && g.M == M && g.eta == eta && g.gamma == gamma &&
             g.lambda == lambda && g.beta == beta && g.mode == mode) { hit = &g; break; }
-    if (hit) {
+    if (hit && hit->exec) {
         if (cudaGraphLaunch(hit->exec, st) != cudaSuccess) return CHOCO_ERR_CUDA;
         hit->last_use = ++L->use_clock;
-        for (int32_t l = 0; l < L->n_layers; ++l) advance_after_replay(L->ctx[l], L->launches_per_step[l]);
+        for (int32_t l = 0; l < L->n_layers; ++l) choco::advance_after_replay(L->ctx[l], L->launches_per_step[l]);
         L->replays += 1;
         return CHOCO_OK;
+    }
+    if (!hit) { // first sighting: remember it, enqueue kernel by kernel
+        const StepGraph g = {X, Xhat, S, G, M, eta, gamma, lambda, beta, mode, nullptr, ++L->use_clock};
+        if (L->graphs.size() < kMaxGraphs) {
+            L->graphs.push_back(g);
+        } else {
+            size_t oldest = 0;
+            for (size_t i = 1; i < L->graphs.size(); ++i)
+                if (L->graphs[i].last_use < L->graphs[oldest].last_use) oldest = i;
+            if (L->graphs[oldest].exec) cudaGraphExecDestroy(L->graphs[oldest].exec);
+            L->graphs[oldest] = g;
+        }
+        return eager_step(L, X, Xhat, S, G, M, eta, gamma, lambda, beta, stream);
     }
 
     // capture this step; on any failure put the host state back and run it eagerly
@@ -201,16 +196,8 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
     }
     L->launches_per_step.resize(L->n_layers);
     for (int32_t l = 0; l < L->n_layers; ++l) L->launches_per_step[l] = L->ctx[l]->launches - before[l].launches;
-    StepGraph g = {X, Xhat, S, G, M, eta, gamma, lambda, beta, mode, exec, ++L->use_clock};
-    if (L->graphs.size() < kMaxGraphs) {
-        L->graphs.push_back(g);
-    } else {
-        size_t oldest = 0;
-        for (size_t i = 1; i < L->graphs.size(); ++i)
-            if (L->graphs[i].last_use < L->graphs[oldest].last_use) oldest = i;
-        cudaGraphExecDestroy(L->graphs[oldest].exec);
-        L->graphs[oldest] = g;
-    }
+    hit->exec = exec;
+    hit->last_use = ++L->use_clock;
     return CHOCO_OK;
 }
 
@@ -254,6 +241,7 @@ int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int
         // gsgd_b and random_a key their generator with the step number: these contexts keep it
         // in device memory, where a replayed graph finds the current value
         L->ctx[l]->dev_step = p->kind == CHOCO_Q_QSGD || p->kind == CHOCO_Q_RANDK;
+        L->ctx[l]->graphs_ok = false; // the layered step is captured as a whole, not layer by layer
     }
     bool ok = cudaEventCreateWithFlags(&L->fork, cudaEventDisableTiming) == cudaSuccess;
     for (int s = 0; s < kLayerStreams && ok; ++s) {
