@@ -159,6 +159,19 @@ int choco_set_carry(choco_ctx* ctx, int32_t enable);
  */
 int choco_set_graphs(choco_ctx* ctx, int32_t enable);
 
+/*
+ * TOPK keeps, per row, a list of candidate coordinates gathered while the previous step formed
+ * x_i, under a key bound guessed for the next step.  When the guess misses (fewer than k, or
+ * more than the list holds) the row is selected exactly from the dense row, by one thread block:
+ * cheap for short rows, tens of milliseconds for a row of 25 M coordinates.  For rows of at
+ * least 4 194 304 coordinates every step therefore enqueues six more kernels after the
+ * selection kernel (two rounds of histogram and bound, collection, selection again) that return
+ * at once unless a row missed, in which case they rebuild that row's candidates with all SMs.  The result is the
+ * same either way.  choco_set_rescue -- enable = 0 / 1 turns these kernels off / on for a
+ * context of any row length (TOPK only; CHOCO_ERR_UNSUPPORTED for other operators).
+ */
+int choco_set_rescue(choco_ctx* ctx, int32_t enable);
+
 /* Step counter t (keys the generator).  Setting it, together with restoring X, Xhat and S,
  * resumes a run bit-exactly; choco_set_step implies choco_invalidate. */
 int choco_get_step(const choco_ctx* ctx, uint64_t* t);
@@ -275,6 +288,7 @@ typedef struct {
     uint64_t kernel_launches;  /* kernels the step calls have enqueued                         */
     uint64_t device_timeouts;  /* bounded waits inside kernels that ran out (must stay 0)      */
     uint64_t graph_replays;    /* step calls served by replaying a captured CUDA graph          */
+    uint64_t rescued_rows;     /* rows re-collected by the grid-wide kernels (choco_set_rescue) */
 } choco_stats;
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
 

@@ -143,6 +143,7 @@ int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, f
     if (sparse) {
         if (!was_prepared) e = launch_select_prepare(dv, a, st);
         if (e == cudaSuccess) e = launch_select_emit(dv, a, was_prepared, st);
+        if (e == cudaSuccess && dv.rescue && dv.kind == CHOCO_Q_TOPK) e = launch_select_rescue(dv, a, st);
     } else if (!was_prepared) {
         e = launch_compress_dense(dv, a, st);
     }
@@ -369,6 +370,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     const int64_t nwords = (d + 31) / 32;
     if (p->kind == CHOCO_Q_TOPK || p->kind == CHOCO_Q_RANDK) {
         dv.k = p->k;
+        dv.rescue = (p->kind == CHOCO_Q_TOPK && d >= kRescueMinD) ? 1 : 0;
         dv.kpitch = round_up(p->k, 4);
         // candidates per row: aimed at 2.5 k, with room for a bound that was guessed low
         int64_t cap = 6 * p->k > p->k + 8192 ? 6 * p->k : p->k + 8192;
@@ -384,7 +386,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             const int64_t b_cand = round_up(n * dv.cap * 4, 256);
             const int64_t b_seg = round_up(n * dv.ntiles * 4, 256);
             const int64_t b_row = round_up((int64_t)n * 4, 256);
-            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 4 * b_row;
+            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 5 * b_row;
             unsigned char* arena = nullptr;
             if (e == cudaSuccess) e = dev_alloc(ctx, &arena, total);
             unsigned char* q = arena;
@@ -398,6 +400,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             dv.row_count = (uint32_t*)q; q += b_row;
             dv.row_flags = (uint32_t*)q; q += b_row;
             dv.row_aim = (uint32_t*)q; q += b_row;
+            dv.row_above = (uint32_t*)q; q += b_row;
             const int64_t hot = q - arena; // the candidates behind it are written once, read once
             dv.cand_idx = (uint32_t*)q; q += b_cand;
             dv.cand_val = (uint32_t*)q; q += b_cand;
@@ -563,6 +566,18 @@ int choco_set_carry(choco_ctx* ctx, int32_t enable)
     return CHOCO_OK;
 }
 
+int choco_set_rescue(choco_ctx* ctx, int32_t enable)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->dv.kind != CHOCO_Q_TOPK) return enable ? CHOCO_ERR_UNSUPPORTED : CHOCO_OK;
+    ctx->dv.rescue = enable ? 1 : 0;
+    // the kernels a step enqueues change: no captured step stands for it any more
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) { cudaGraphExecDestroy(ctx->graphs[i].exec); }
+    ctx->ngraphs = 0;
+    return CHOCO_OK;
+}
+
 int choco_set_graphs(choco_ctx* ctx, int32_t enable)
 {
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
@@ -685,6 +700,7 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
     out->device_timeouts = h.timeouts;
     out->kernel_launches = ctx->launches;
     out->graph_replays = ctx->graph_replays;
+    out->rescued_rows = h.rescued_rows;
     return CHOCO_OK;
 }
 

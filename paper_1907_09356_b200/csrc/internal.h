@@ -10,6 +10,9 @@ namespace choco {
 
 // Row flags of the selection pipeline (top-k, random-k).
 constexpr uint32_t kRowExact = 1u;    // candidates unusable: run the exact one-block selection
+constexpr uint32_t kRowRescue = 2u;   // candidates unusable: collect afresh with grid-wide kernels
+constexpr uint32_t kRowRefine = 4u;   // the first digit's bin is too full: resolve the next 11 bits
+constexpr int64_t kRescueMinD = (int64_t)1 << 22; // rows this long are rescued rather than selected by one block
 
 constexpr int64_t kEmitSmemBudget = 200 * 1024; // dynamic shared memory the emit kernel may use
 constexpr int kHistBins = 2048;       // first radix digit: top 11 bits of the ordering key
@@ -19,6 +22,7 @@ struct Stats {
     unsigned long long recompressed_rows;
     unsigned long long exact_rows;
     unsigned long long timeouts;   // bounded device waits that ran out
+    unsigned long long rescued_rows; // rows whose candidates were collected afresh after a miss
 };
 
 // Everything the kernels need; passed by value.
@@ -50,12 +54,14 @@ struct Dev {
     float* msg_val;
     uint32_t* tile_ptr;
     // selection workspace
+    int32_t rescue;              // top-k: a row that misses is re-collected by grid-wide kernels
     int64_t cap;                 // candidate capacity per row
     uint32_t* hist;              // [n, kHistBins]
     uint32_t* row_lo;            // [n] lower bound of the ordering key for candidates
     uint32_t* row_count;         // [n] candidates collected
     uint32_t* row_aim;           // [n] rank the next bound aims at, in units of k / 256
     uint32_t* row_flags;         // [n]
+    uint32_t* row_above;         // [n] keys above the first digit's bin (while a row is refined)
     uint32_t* cand_idx;          // [n, cap]
     uint32_t* cand_val;          // [n, cap] value bits (top-k) or random word (random-k)
     uint32_t* seg_off;           // [n, ntiles] first candidate of a tile
@@ -129,6 +135,9 @@ __device__ __forceinline__ uint64_t step_of(const StepArgs& a)
 cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t st);
 // fused: the candidates came from the previous step's update kernel (statistics only)
 cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st);
+// dv.rescue: rows that the emit kernel flagged get fresh histograms, a bound and a candidate
+// list from the dense row (all SMs), then their emit; six launches that do nothing otherwise
+cudaError_t launch_select_rescue(const Dev& dv, const StepArgs& a, cudaStream_t st);
 // dense compressors
 cudaError_t launch_compress_dense(const Dev& dv, const StepArgs& a, cudaStream_t st);
 // update kernel; emit: also collect the next step's top-k candidates (if apply_can_emit)

@@ -47,37 +47,57 @@ __device__ __forceinline__ void quad_bits(const Dev& dv, const StepArgs& a, int 
 // ---------------------------------------------------------------------------------------
 // prepare 1: histogram of the top 11 bits of the key of x - x^ (top-k only)
 // ---------------------------------------------------------------------------------------
+// With `rescue` the grid is one-dimensional and its blocks stride over the spans of the rows
+// flagged kRowRescue only (normally none: every block then returns at once).  level 0 counts
+// the first digit (top 11 bits) of every key; level 1 serves rows flagged kRowRefine only and
+// counts the next 11 bits of the keys whose first digit is the one row_lo holds.
 template <bool VEC>
-__global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a)
+__global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a, int rescue, int level)
 {
     __shared__ uint32_t h[kHistBins];
-    const int row = blockIdx.y;
-    for (int b = threadIdx.x; b < kHistBins; b += kThreads) h[b] = 0u;
-    __syncthreads();
-    const int64_t c0 = (int64_t)blockIdx.x * kSpan;
+    const int row_begin = rescue ? 0 : (int)blockIdx.y, row_end = rescue ? dv.n : (int)blockIdx.y + 1;
+    for (int row = row_begin; row < row_end; ++row) {
+        const uint32_t flags = (rescue || level) ? dv.row_flags[row] : 0u;
+        if (rescue && !(flags & kRowRescue)) continue;
+        if (level && !(flags & kRowRefine)) continue;
+        const uint32_t first = level ? dv.row_lo[row] >> 21 : 0u;
+        for (int64_t sp = blockIdx.x; sp < dv.nspans; sp += rescue ? (int64_t)gridDim.x : dv.nspans) {
+            for (int b = threadIdx.x; b < kHistBins; b += kThreads) h[b] = 0u;
+            __syncthreads();
+            const int64_t c0 = sp * kSpan;
 #pragma unroll
-    for (int it = 0; it < kDenseIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
-        if (c < dv.d) {
-            uint32_t bits[4];
-            quad_bits<SEL_TOPK, VEC>(dv, a, row, c, bits);
+            for (int it = 0; it < kDenseIters; ++it) {
+                const int64_t c = c0 + (int64_t)(it * kThreads + threadIdx.x) * kQuad;
+                if (c < dv.d) {
+                    uint32_t bits[4];
+                    quad_bits<SEL_TOPK, VEC>(dv, a, row, c, bits);
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (c + e < dv.d) atomicAdd(&h[order_key<SEL_TOPK>(bits[e]) >> 21], 1u);
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t key = order_key<SEL_TOPK>(bits[e]);
+                        if (c + e >= dv.d) continue;
+                        if (!level) atomicAdd(&h[key >> 21], 1u);
+                        else if ((key >> 21) == first) atomicAdd(&h[(key >> 10) & (kHistBins - 1)], 1u);
+                    }
+                }
+            }
+            __syncthreads();
+            uint32_t* g = dv.hist + (int64_t)row * kHistBins;
+            for (int b = threadIdx.x; b < kHistBins; b += kThreads)
+                if (h[b]) atomicAdd(&g[b], h[b]);
+            __syncthreads();
         }
     }
-    __syncthreads();
-    uint32_t* g = dv.hist + (int64_t)row * kHistBins;
-    for (int b = threadIdx.x; b < kHistBins; b += kThreads)
-        if (h[b]) atomicAdd(&g[b], h[b]);
 }
 
 // prepare 2: per row, the lowest first digit that must be kept
-__global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv)
+__global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv, int rescue, int level)
 {
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t sm[36];
     const int row = blockIdx.x;
+    const uint32_t flags = dv.row_flags[row];
+    if (rescue && !(flags & kRowRescue)) return;
+    if (level && !(flags & kRowRefine)) return;
     uint32_t* g = dv.hist + (int64_t)row * kHistBins;
     for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) {
         h[b] = g[b];
@@ -86,15 +106,35 @@ __global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv)
     __syncthreads();
     // keep down to rank 2.5 k (not just k) so that emit can place the next step's bound
     const uint64_t want = 2 * (uint64_t)dv.k + (uint64_t)dv.k / 2;
-    const uint32_t need = (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d);
+    const uint32_t rank = (uint32_t)(want < (uint64_t)dv.d ? want : (uint64_t)dv.d);
+    // level 1: the keys above the first digit's bin are already counted
+    const uint32_t before = level ? dv.row_above[row] : 0u;
     uint32_t digit, above;
-    block_find_digit<kSelThreads>(h, kHistBins, need, sm, &digit, &above);
+    block_find_digit<kSelThreads>(h, kHistBins, rank - before, sm, &digit, &above);
     if (threadIdx.x == 0) {
-        dv.row_lo[row] = digit << 21;
-        dv.row_aim[row] = kAimStart;
-        dv.row_count[row] = 0u;
-        // every coordinate with this digit or a higher one becomes a candidate
-        dv.row_flags[row] = ((int64_t)above + (int64_t)h[digit] > dv.cap) ? kRowExact : 0u;
+        // Every coordinate with this digit or a higher one becomes a candidate.  If the digit's
+        // own bin makes that more than the capacity, the bins above it alone will do as long as
+        // they hold k coordinates.  Otherwise the bin is both needed and too full: after a
+        // first digit the next 11 bits are resolved (the keys of a row whose largest entries
+        // were just sent crowd under the last threshold); after those the row is left to the
+        // exact selection.
+        const int64_t upto = (int64_t)before + above; // keys above the bin
+        bool full = false;
+        if (upto + (int64_t)h[digit] > dv.cap) {
+            if (upto >= dv.k && digit + 1u < (uint32_t)kHistBins) digit += 1u;
+            else full = true;
+        }
+        const uint32_t keep = rescue ? kRowRescue : 0u;
+        if (!level) {
+            dv.row_lo[row] = digit << 21;
+            dv.row_above[row] = above;
+            dv.row_aim[row] = kAimStart;
+            dv.row_count[row] = 0u;
+            dv.row_flags[row] = keep | (full ? kRowRefine : 0u);
+        } else {
+            dv.row_lo[row] = (dv.row_lo[row] & 0xFFE00000u) | (digit << 10);
+            dv.row_flags[row] = keep | (full ? kRowExact : 0u);
+        }
     }
 }
 
@@ -113,57 +153,65 @@ __global__ void randk_bound_kernel(Dev dv, uint32_t lo)
 // ---------------------------------------------------------------------------------------
 // prepare 3: collect candidates, ascending inside each tile
 // ---------------------------------------------------------------------------------------
+// With `rescue`: one-dimensional grid striding over the tiles of the rows flagged kRowRescue.
 template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs a)
+__global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs a, int rescue)
 {
     __shared__ uint32_t sm[2][kTileThreads / 32 + 1];
     __shared__ uint32_t s_base;
-    const int row = blockIdx.y;
-    if (dv.row_flags[row] & kRowExact) return;
-    const uint32_t lo = dv.row_lo[row];
-    const int64_t c0 = (int64_t)blockIdx.x * kTile;
-
-    uint32_t bits[kTileIters][4];
-    uint32_t take = 0; // bit (4 it + e)
-    uint32_t cnt[kTileIters];
+    const int row_begin = rescue ? 0 : (int)blockIdx.y, row_end = rescue ? dv.n : (int)blockIdx.y + 1;
+    for (int row = row_begin; row < row_end; ++row) {
+        const uint32_t flags = dv.row_flags[row];
+        if (rescue && !(flags & kRowRescue)) continue;
+        if (flags & kRowExact) continue;
+        const uint32_t lo = dv.row_lo[row];
+        for (int64_t tile = blockIdx.x; tile < dv.ntiles; tile += rescue ? (int64_t)gridDim.x : dv.ntiles) {
+            const int64_t c0 = tile * kTile;
+            uint32_t bits[kTileIters][4];
+            uint32_t take = 0; // bit (4 it + e)
+            uint32_t cnt[kTileIters];
 #pragma unroll
-    for (int it = 0; it < kTileIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
-        cnt[it] = 0;
-        if (c < dv.d) {
-            quad_bits<KIND, VEC>(dv, a, row, c, bits[it]);
+            for (int it = 0; it < kTileIters; ++it) {
+                const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
+                cnt[it] = 0;
+                if (c < dv.d) {
+                    quad_bits<KIND, VEC>(dv, a, row, c, bits[it]);
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (c + e < dv.d && order_key<KIND>(bits[it][e]) >= lo) {
-                    take |= 1u << (4 * it + e);
-                    ++cnt[it];
+                    for (int e = 0; e < 4; ++e)
+                        if (c + e < dv.d && order_key<KIND>(bits[it][e]) >= lo) {
+                            take |= 1u << (4 * it + e);
+                            ++cnt[it];
+                        }
                 }
-        }
-    }
-    uint32_t start[kTileIters], total;
-    ordered_starts<kTileThreads, kTileIters>(cnt, sm, start, &total);
-    if (threadIdx.x == 0) {
-        const uint32_t base = total ? atomicAdd(&dv.row_count[row], total) : 0u;
-        dv.seg_off[(int64_t)row * dv.ntiles + blockIdx.x] = base;
-        dv.seg_cnt[(int64_t)row * dv.ntiles + blockIdx.x] = total;
-        // past the capacity nothing is written; emit sees row_count > cap and gives up
-        s_base = ((int64_t)base + total > dv.cap) ? 0xFFFFFFFFu : base;
-    }
-    __syncthreads();
-    if (s_base == 0xFFFFFFFFu) return;
-    uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + s_base;
-    uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + s_base;
-#pragma unroll
-    for (int it = 0; it < kTileIters; ++it) {
-        const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
-        uint32_t p = start[it];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (take & (1u << (4 * it + e))) {
-                ci[p] = (uint32_t)(c + e);
-                cv[p] = bits[it][e];
-                ++p;
             }
+            uint32_t start[kTileIters], total;
+            ordered_starts<kTileThreads, kTileIters>(cnt, sm, start, &total);
+            if (threadIdx.x == 0) {
+                const uint32_t base = total ? atomicAdd(&dv.row_count[row], total) : 0u;
+                dv.seg_off[(int64_t)row * dv.ntiles + tile] = base;
+                dv.seg_cnt[(int64_t)row * dv.ntiles + tile] = total;
+                // past the capacity nothing is written; emit sees row_count > cap and gives up
+                s_base = ((int64_t)base + total > dv.cap) ? 0xFFFFFFFFu : base;
+            }
+            __syncthreads();
+            const uint32_t base = s_base;
+            __syncthreads(); // s_base and sm are written again by the next tile
+            if (base == 0xFFFFFFFFu) continue;
+            uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + base;
+            uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + base;
+#pragma unroll
+            for (int it = 0; it < kTileIters; ++it) {
+                const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
+                uint32_t p = start[it];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (take & (1u << (4 * it + e))) {
+                        ci[p] = (uint32_t)(c + e);
+                        cv[p] = bits[it][e];
+                        ++p;
+                    }
+            }
+        }
     }
 }
 
@@ -447,8 +495,11 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
 //   3. prefix over tiles -> tile_ptr and the number of equal keys before each tile; prefix
 //      over slabs; per tile the two prefixes at its first candidate;
 //   4. every chosen candidate computes its own output position and writes itself.
+// `rescue`: 0 = a row whose candidates cannot be used is selected exactly by this block;
+// 1 = such a row is flagged kRowRescue instead and left to the rescue kernels that follow;
+// 2 = this launch is their last stage and serves the flagged rows only.
 template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused)
+__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
 {
     extern __shared__ uint32_t dyn[];
     __shared__ uint32_t h[kHistBins];
@@ -462,8 +513,18 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const uint32_t flags = dv.row_flags[row];
     const uint32_t k = (uint32_t)dv.k;
     __syncthreads();
-    if ((flags & kRowExact) || ncand > (uint32_t)dv.cap || ncand < k) {
-        exact_row<KIND, VEC>(dv, a, row, h, sm); // the candidates cannot be used
+    if (rescue == 2 && !(flags & kRowRescue)) return;
+    if ((flags & kRowExact) || ncand > (uint32_t)dv.cap || ncand < k) { // the candidates cannot be used
+        if (rescue == 1 && !(flags & kRowExact)) {
+            // a fresh histogram would say the same for a row flagged kRowExact; any other row
+            // gets new candidates from the kernels that follow
+            if (threadIdx.x == 0) {
+                dv.row_flags[row] = kRowRescue;
+                atomicAdd(&dv.stats->rescued_rows, 1ull);
+            }
+            return;
+        }
+        exact_row<KIND, VEC>(dv, a, row, h, sm);
         return;
     }
     const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
@@ -627,6 +688,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
+        dv.row_flags[row] = 0u;
         atomicAdd(fused ? &dv.stats->prepared_rows : &dv.stats->recompressed_rows, 1ull);
     }
 }
@@ -641,10 +703,12 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
     if (KIND == SEL_TOPK) {
         const dim3 hgrid((unsigned)dv.nspans, (unsigned)dv.n);
-        if (a.vec) hist_kernel<true><<<hgrid, kThreads, 0, st>>>(dv, a);
-        else hist_kernel<false><<<hgrid, kThreads, 0, st>>>(dv, a);
-        bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv);
-        *a.launches += 2;
+        for (int level = 0; level < 2; ++level) { // the second round returns at once unless a bin was too full
+            if (a.vec) hist_kernel<true><<<hgrid, kThreads, 0, st>>>(dv, a, 0, level);
+            else hist_kernel<false><<<hgrid, kThreads, 0, st>>>(dv, a, 0, level);
+            bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv, 0, level);
+        }
+        *a.launches += 4;
     } else {
         // keep words <= hi: about k + 6 sqrt(k) + 16 of d coordinates
         const double kk = (double)dv.k;
@@ -653,8 +717,8 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
         randk_bound_kernel<<<(dv.n + 127) / 128, 128, 0, st>>>(dv, ~hi);
         *a.launches += 1;
     }
-    if (a.vec) collect_kernel<KIND, true><<<grid, kTileThreads, 0, st>>>(dv, a);
-    else collect_kernel<KIND, false><<<grid, kTileThreads, 0, st>>>(dv, a);
+    if (a.vec) collect_kernel<KIND, true><<<grid, kTileThreads, 0, st>>>(dv, a, 0);
+    else collect_kernel<KIND, false><<<grid, kTileThreads, 0, st>>>(dv, a, 0);
     *a.launches += 1;
     return cudaGetLastError();
 }
@@ -666,7 +730,7 @@ cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t
 }
 
 template <int KIND>
-static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
+static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int rescue, cudaStream_t st)
 {
     auto kern = a.vec ? emit_kernel<KIND, true> : emit_kernel<KIND, false>;
     static bool configured[64][2] = {};
@@ -679,7 +743,7 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaS
         if (dev >= 0 && dev < 64) configured[dev][a.vec ? 1 : 0] = true;
     }
     e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st, dv, a,
-                          fused ? 1 : 0);
+                          fused ? 1 : 0, rescue);
     if (e != cudaSuccess) return e;
     *a.launches += 1;
     return cudaGetLastError();
@@ -687,8 +751,36 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, cudaS
 
 cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)
 {
-    return dv.kind == CHOCO_Q_TOPK ? emit_impl<SEL_TOPK>(dv, a, fused, st)
-                                   : emit_impl<SEL_RANDK>(dv, a, fused, st);
+    return dv.kind == CHOCO_Q_TOPK ? emit_impl<SEL_TOPK>(dv, a, fused, dv.rescue ? 1 : 0, st)
+                                   : emit_impl<SEL_RANDK>(dv, a, fused, 0, st);
+}
+
+cudaError_t launch_select_rescue(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    // enough blocks to fill the device when a row does need them; they return at once otherwise
+    static int sms[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    int nsm = (dev >= 0 && dev < 64) ? sms[dev] : 0;
+    if (nsm == 0) {
+        e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) sms[dev] = nsm;
+    }
+    const unsigned hblocks = (unsigned)(dv.nspans < 8 * (int64_t)nsm ? dv.nspans : 8 * (int64_t)nsm);
+    const unsigned cblocks = (unsigned)(dv.ntiles < 8 * (int64_t)nsm ? dv.ntiles : 8 * (int64_t)nsm);
+    for (int level = 0; level < 2; ++level) {
+        if (a.vec) hist_kernel<true><<<hblocks, kThreads, 0, st>>>(dv, a, 1, level);
+        else hist_kernel<false><<<hblocks, kThreads, 0, st>>>(dv, a, 1, level);
+        bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv, 1, level);
+    }
+    if (a.vec) collect_kernel<SEL_TOPK, true><<<cblocks, kTileThreads, 0, st>>>(dv, a, 1);
+    else collect_kernel<SEL_TOPK, false><<<cblocks, kTileThreads, 0, st>>>(dv, a, 1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    *a.launches += 5;
+    return emit_impl<SEL_TOPK>(dv, a, false, 2, st);
 }
 
 } // namespace choco
