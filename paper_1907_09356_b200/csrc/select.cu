@@ -47,6 +47,16 @@ __device__ __forceinline__ void quad_bits(const Dev& dv, const StepArgs& a, int 
 // ---------------------------------------------------------------------------------------
 // prepare 1: histogram of the top 11 bits of the key of x - x^ (top-k only)
 // ---------------------------------------------------------------------------------------
+// True (for every thread of the block) if any row carries one of the flags in `mask`.  The
+// rescue kernels ask this first: the rows' flags are read side by side rather than one after
+// the other, so a launch with nothing to do is over in about a microsecond.
+__device__ __forceinline__ bool any_row_flagged(const Dev& dv, uint32_t mask)
+{
+    int mine = 0;
+    for (int r = threadIdx.x; r < dv.n; r += blockDim.x) mine |= (dv.row_flags[r] & mask) != 0u;
+    return __syncthreads_or(mine) != 0;
+}
+
 // With `rescue` the grid is one-dimensional and its blocks stride over the spans of the rows
 // flagged kRowRescue only (normally none: every block then returns at once).  level 0 counts
 // the first digit (top 11 bits) of every key; level 1 serves rows flagged kRowRefine only and
@@ -55,6 +65,7 @@ template <bool VEC>
 __global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a, int rescue, int level)
 {
     __shared__ uint32_t h[kHistBins];
+    if (rescue && !any_row_flagged(dv, kRowRescue)) return;
     const int row_begin = rescue ? 0 : (int)blockIdx.y, row_end = rescue ? dv.n : (int)blockIdx.y + 1;
     for (int row = row_begin; row < row_end; ++row) {
         const uint32_t flags = (rescue || level) ? dv.row_flags[row] : 0u;
@@ -159,6 +170,7 @@ __global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs 
 {
     __shared__ uint32_t sm[2][kTileThreads / 32 + 1];
     __shared__ uint32_t s_base;
+    if (rescue && !any_row_flagged(dv, kRowRescue)) return;
     const int row_begin = rescue ? 0 : (int)blockIdx.y, row_end = rescue ? dv.n : (int)blockIdx.y + 1;
     for (int row = row_begin; row < row_end; ++row) {
         const uint32_t flags = dv.row_flags[row];
