@@ -292,6 +292,12 @@ def main():
     S = torch.zeros_like(X)
     free_b = torch.cuda.mem_get_info(dev)[0]
     pool_n = int(max(2, min(args.pool, (free_b * 0.5) // (4 * N))))
+    if small:
+        pool_n = 2                  # the state fits L2 anyway; fewer argument sets to capture
+    if wl.layers or small:
+        # graph replay: an argument set (gradient tensor x message-buffer parity) runs kernel by
+        # kernel when first seen and is captured when seen again; the warm-up covers both
+        args.warmup = max(args.warmup, 4 * pool_n + 2)
     pool = [torch.randn(wl.n, wl.d, device=dev, generator=gen) * float(np.sqrt(wl.g_var or 1e-2))
             for _ in range(pool_n)]
     if wl.layers:

@@ -271,6 +271,9 @@ WORKLOADS = {
     "l3_ring8_topk_layers": Workload("l3_ring8_topk_layers", 8, 272474, "ring", "topk", eta=0.1, gamma=0.04,
                                      steps=1000, x_var=0.01, g_var=1e-2, layers="resnet20",
                                      a_num=1, a_den=100),
+    "l3_ring8_qsgd_layers": Workload("l3_ring8_qsgd_layers", 8, 272474, "ring", "qsgd", s=16, bucket=512,
+                                     eta=0.1, gamma=0.1, steps=1000, x_var=0.01, g_var=1e-2,
+                                     layers="resnet20"),
     "l5_ring32_qsgd_layers": Workload("l5_ring32_qsgd_layers", 32, 25_557_032, "ring", "qsgd", s=16,
                                       bucket=512, eta=0.1, gamma=0.1, steps=200, x_var=0.01,
                                       g_var=1e-3, layers="resnet50"),
