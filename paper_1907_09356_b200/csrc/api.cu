@@ -416,14 +416,16 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             // as the budget allows: slab prefixes, per-tile arrays, a cache of the keys
             dv.slab_pitch = dv.cap / 32 + 2;
             int64_t left = kEmitSmemBudget;
-            dv.emit_slabs_smem = 2 * dv.slab_pitch * 4 <= left ? 1 : 0;
-            if (dv.emit_slabs_smem) left -= 2 * dv.slab_pitch * 4;
+            dv.emit_slabs_smem = 4 * dv.slab_pitch * 4 <= left ? 1 : 0; // two prefix arrays, two masks
+            if (dv.emit_slabs_smem) left -= 4 * dv.slab_pitch * 4;
             dv.emit_tiles_smem = 3 * dv.ntiles * 4 <= left ? 1 : 0;
             if (dv.emit_tiles_smem) left -= 3 * dv.ntiles * 4;
             dv.emit_keys_cap = std::min<int64_t>(dv.cap, left / 8); // value bits and index per candidate
             dv.emit_smem_bytes = kEmitSmemBudget - left + dv.emit_keys_cap * 8;
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_c, n * dv.slab_pitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_d, n * dv.slab_pitch);
         }
         ctx->msg_bytes_per_worker = (p->kind == CHOCO_Q_TOPK ? 8 : 4) * p->k;
     } else if (p->kind == CHOCO_Q_SIGN) {

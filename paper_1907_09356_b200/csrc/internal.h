@@ -73,6 +73,8 @@ struct Dev {
     int64_t slab_pitch;          // cap / 32 + 2: slabs of 32 candidates per row
     uint32_t* slab_a;            // [n, slab_pitch] scratch (used when not in shared memory)
     uint32_t* slab_b;            // [n, slab_pitch]
+    uint32_t* slab_c;            // [n, slab_pitch] ballot of the keys above the k-th, per slab
+    uint32_t* slab_d;            // [n, slab_pitch] ballot of the keys equal to it
     int32_t emit_slabs_smem;     // slab arrays in shared memory
     int32_t emit_tiles_smem;     // per-tile arrays in shared memory
     int64_t emit_keys_cap;       // candidate keys cached in shared memory up to this many

@@ -545,9 +545,15 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
 
     // carve the dynamic shared memory
     uint32_t* cursor = dyn;
-    uint32_t *slab_g, *slab_e, *t_gt, *t_eq, *t_sbe;
-    if (dv.emit_slabs_smem) { slab_g = cursor; slab_e = cursor + dv.slab_pitch; cursor += 2 * dv.slab_pitch; }
-    else { slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch; }
+    uint32_t *slab_g, *slab_e, *slab_gm, *slab_em, *t_gt, *t_eq, *t_sbe;
+    if (dv.emit_slabs_smem) {
+        slab_g = cursor; slab_e = cursor + dv.slab_pitch;
+        slab_gm = cursor + 2 * dv.slab_pitch; slab_em = cursor + 3 * dv.slab_pitch;
+        cursor += 4 * dv.slab_pitch;
+    } else {
+        slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch;
+        slab_gm = dv.slab_c + (int64_t)row * dv.slab_pitch; slab_em = dv.slab_d + (int64_t)row * dv.slab_pitch;
+    }
     if (dv.emit_tiles_smem) { t_gt = cursor; t_eq = cursor + dv.ntiles; t_sbe = cursor + 2 * dv.ntiles; cursor += 3 * dv.ntiles; }
     else { t_gt = dv.tile_a + (int64_t)row * dv.ntiles; t_eq = dv.tile_b + (int64_t)row * dv.ntiles; t_sbe = dv.tile_c + (int64_t)row * dv.ntiles; }
     uint32_t* sbits = cursor;                      // the candidates' value bits and
@@ -628,7 +634,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
                 if (gt | eq) atomicAdd(gt ? &t_gt[idx[u] / kTile] : &t_eq[idx[u] / kTile], 1u);
             }
             const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-            if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); }
+            if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); slab_gm[sl] = bg; slab_em[sl] = be; }
         }
     }
     __syncthreads();
@@ -645,13 +651,11 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         uint32_t pg = 0, pe = 0;
         if (own_tile ? my_sc : sc[t]) {
             const uint32_t first = own_tile ? my_so : so[t], s0 = first >> 5;
-            pg = slab_g[s0];
-            pe = slab_e[s0];
-            for (uint32_t p = s0 << 5; p < first; ++p) {
-                const uint32_t kk = key_at(p);
-                pg += kk > T;
-                pe += kk == T;
-            }
+            // keys above / equal to T before `first`: whole slabs from the prefixes, the rest of
+            // its own slab from the slab's ballots
+            const uint32_t below = (1u << (first & 31u)) - 1u;
+            pg = slab_g[s0] + __popc(slab_gm[s0] & below);
+            pe = slab_e[s0] + __popc(slab_em[s0] & below);
         }
         t_gt[t] = pg;
         t_sbe[t] = pe;
@@ -664,35 +668,22 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const float* xr = a.X + (int64_t)row * dv.ld;
     const float* hr = a.Xhat + (int64_t)row * dv.ld;
     const uint32_t lt = (1u << lane) - 1u;
-    for (int64_t s0 = warp; s0 < nslab; s0 += (kSelThreads / 32) * kBatch) {
-        uint32_t idx[kBatch];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
+    // (which candidates those are is in the slabs' ballots: only they are fetched again)
+    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+        const uint32_t bg = slab_gm[sl], be = slab_em[sl];
+        const bool gt = (bg >> lane) & 1u, eq = (be >> lane) & 1u;
+        if (gt | eq) {
             const uint32_t p = (uint32_t)(sl << 5) + lane;
-            idx[u] = (sl < nslab && p < ncand) ? idx_at(p) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
-            if (sl >= nslab) break;
-            const uint32_t p = (uint32_t)(sl << 5) + lane;
-            const bool act = p < ncand;
-            const uint32_t bits = act ? bits_at(p) : 0u;
-            const uint32_t kk = order_key<KIND>(bits);
-            const bool gt = act && kk > T, eq = act && kk == T;
-            const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-            if (gt | eq) {
-                const uint32_t tile = idx[u] / kTile;
-                const uint32_t g_in = slab_g[sl] + __popc(bg & lt) - t_gt[tile];  // above T, earlier in the tile
-                const uint32_t e_in = slab_e[sl] + __popc(be & lt) - t_sbe[tile]; // equal to T, earlier in the tile
-                const uint32_t eqb = t_eq[tile];                                  // equal to T, in earlier tiles
-                const uint32_t room = r > eqb ? r - eqb : 0u;                     // equal keys this tile may keep
-                if (gt || e_in < room) {
-                    const uint32_t pos = tp[tile] + g_in + (e_in < room ? e_in : room);
-                    mi[pos] = idx[u];
-                    mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits) : __fsub_rn(xr[idx[u]], hr[idx[u]]);
-                }
+            const uint32_t id = idx_at(p);
+            const uint32_t tile = id / kTile;
+            const uint32_t g_in = slab_g[sl] + __popc(bg & lt) - t_gt[tile];  // above T, earlier in the tile
+            const uint32_t e_in = slab_e[sl] + __popc(be & lt) - t_sbe[tile]; // equal to T, earlier in the tile
+            const uint32_t eqb = t_eq[tile];                                  // equal to T, in earlier tiles
+            const uint32_t room = r > eqb ? r - eqb : 0u;                     // equal keys this tile may keep
+            if (gt || e_in < room) {
+                const uint32_t pos = tp[tile] + g_in + (e_in < room ? e_in : room);
+                mi[pos] = id;
+                mv[pos] = KIND == SEL_TOPK ? __uint_as_float(bits_at(p)) : __fsub_rn(xr[id], hr[id]);
             }
         }
     }
