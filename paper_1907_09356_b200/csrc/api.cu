@@ -374,7 +374,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         dv.kpitch = round_up(p->k, 4);
         // candidates per row: aimed at 2.5 k, with room for a bound that was guessed low
         int64_t cap = 6 * p->k > p->k + 8192 ? 6 * p->k : p->k + 8192;
-        dv.cap = cap < d ? cap : d;
+        dv.cap = round_up(cap < d ? cap : d, 4); // rows of the candidate arrays stay 16-byte aligned
         {
             // One arena for what one kernel writes and the next reads back within a step.  Its
             // head (range records, messages, per-tile tables) is read with dependent loads by
@@ -414,13 +414,18 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         {
             // the emit kernel keeps in shared memory, in this order of preference and as far
             // as the budget allows: slab prefixes, per-tile arrays, a cache of the keys
-            dv.slab_pitch = dv.cap / 32 + 2;
-            int64_t left = kEmitSmemBudget;
-            dv.emit_slabs_smem = 4 * dv.slab_pitch * 4 <= left ? 1 : 0; // two prefix arrays, two masks
-            if (dv.emit_slabs_smem) left -= 4 * dv.slab_pitch * 4;
-            dv.emit_tiles_smem = 3 * dv.ntiles * 4 <= left ? 1 : 0;
-            if (dv.emit_tiles_smem) left -= 3 * dv.ntiles * 4;
-            dv.emit_keys_cap = std::min<int64_t>(dv.cap, left / 8); // value bits and index per candidate
+            // every piece a multiple of 16 bytes, so that the key cache behind them can be the
+            // destination of bulk copies; 16 bytes in front for their barrier
+            dv.slab_pitch = round_up(dv.cap / 32 + 2, 4);
+            const int64_t tpitch = round_up(dv.ntiles, 4);
+            int64_t left = kEmitSmemBudget - 16;
+            dv.emit_slabs_smem = 2 * dv.slab_pitch * 4 <= left ? 1 : 0;
+            if (dv.emit_slabs_smem) left -= 2 * dv.slab_pitch * 4;
+            dv.emit_tiles_smem = 3 * tpitch * 4 <= left ? 1 : 0;
+            if (dv.emit_tiles_smem) left -= 3 * tpitch * 4;
+            dv.emit_masks_smem = 2 * dv.slab_pitch * 4 <= left ? 1 : 0;
+            if (dv.emit_masks_smem) left -= 2 * dv.slab_pitch * 4;
+            dv.emit_keys_cap = std::min<int64_t>(dv.cap, (left / 8) & ~(int64_t)3); // value bits and index per candidate
             dv.emit_smem_bytes = kEmitSmemBudget - left + dv.emit_keys_cap * 8;
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);

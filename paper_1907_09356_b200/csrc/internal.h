@@ -77,6 +77,7 @@ struct Dev {
     uint32_t* slab_d;            // [n, slab_pitch] ballot of the keys equal to it
     int32_t emit_slabs_smem;     // slab arrays in shared memory
     int32_t emit_tiles_smem;     // per-tile arrays in shared memory
+    int32_t emit_masks_smem;     // slab ballots in shared memory
     int64_t emit_keys_cap;       // candidate keys cached in shared memory up to this many
     int64_t emit_smem_bytes;     // dynamic shared memory of the emit kernel
     Stats* stats;

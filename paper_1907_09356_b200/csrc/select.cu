@@ -15,6 +15,7 @@
 //             next step.
 //   exact   : rows whose candidates are unusable (too many, too few, overflow) are selected
 //             exactly, by the same block, straight from the dense row.
+#include "bulk.cuh"
 #include "select.cuh"
 
 namespace choco {
@@ -318,14 +319,15 @@ __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t ran
 // Tell every reader of worker `row` where row's message enters each tile (tp[t] .. tp[t+1]),
 // in the reader's own CSR position, with the reader's own weight.  Called by all threads of
 // the block after tp[] is complete and visible.
-__device__ __forceinline__ void publish_ranges(const Dev& dv, int row, const uint32_t* tp)
+// `tid` of `nthreads` threads share the work (all threads of the block by default).
+__device__ __forceinline__ void publish_ranges(const Dev& dv, int row, const uint32_t* tp, int tid, int nthreads)
 {
     for (int e = dv.row_ptr[row]; e < dv.row_ptr[row + 1]; ++e) {
         const int64_t reader = dv.col[e];
         const int pos = dv.rd_pos[e];
         const uint32_t wbits = __float_as_uint(dv.rd_w[e]);
         uint4* rec = dv.rec + (reader * dv.ntiles) * dv.maxdeg + pos;
-        for (int64_t t = threadIdx.x; t < dv.ntiles; t += blockDim.x) {
+        for (int64_t t = tid; t < dv.ntiles; t += nthreads) {
             const uint32_t lo = tp[t];
             rec[t * dv.maxdeg] = make_uint4((uint32_t)row, lo, tp[t + 1] - lo, wbits);
         }
@@ -483,7 +485,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     }
     if (threadIdx.x == 0) tp[dv.ntiles] = k;
     __syncthreads();
-    publish_ranges(dv, row, tp);
+    publish_ranges(dv, row, tp, threadIdx.x, kSelThreads);
     if (threadIdx.x == 0) {
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
@@ -513,7 +515,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
 template <int KIND, bool VEC>
 __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
 {
-    extern __shared__ uint32_t dyn[];
+    extern __shared__ __align__(16) uint32_t dyn[];
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t sm[64];
     __shared__ uint32_t s_carry[2];
@@ -543,51 +545,68 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
     const int64_t nslab = ((int64_t)ncand + 31) >> 5;
 
-    // carve the dynamic shared memory
-    uint32_t* cursor = dyn;
+    // carve the dynamic shared memory (every piece a multiple of 16 bytes)
+    uint64_t* bar = reinterpret_cast<uint64_t*>(dyn); // for the bulk copies of the candidates
+    uint32_t* cursor = dyn + 4;
+    const int64_t tpitch = (dv.ntiles + 3) & ~(int64_t)3;
     uint32_t *slab_g, *slab_e, *slab_gm, *slab_em, *t_gt, *t_eq, *t_sbe;
-    if (dv.emit_slabs_smem) {
-        slab_g = cursor; slab_e = cursor + dv.slab_pitch;
-        slab_gm = cursor + 2 * dv.slab_pitch; slab_em = cursor + 3 * dv.slab_pitch;
-        cursor += 4 * dv.slab_pitch;
-    } else {
-        slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch;
-        slab_gm = dv.slab_c + (int64_t)row * dv.slab_pitch; slab_em = dv.slab_d + (int64_t)row * dv.slab_pitch;
-    }
-    if (dv.emit_tiles_smem) { t_gt = cursor; t_eq = cursor + dv.ntiles; t_sbe = cursor + 2 * dv.ntiles; cursor += 3 * dv.ntiles; }
+    if (dv.emit_slabs_smem) { slab_g = cursor; slab_e = cursor + dv.slab_pitch; cursor += 2 * dv.slab_pitch; }
+    else { slab_g = dv.slab_a + (int64_t)row * dv.slab_pitch; slab_e = dv.slab_b + (int64_t)row * dv.slab_pitch; }
+    if (dv.emit_tiles_smem) { t_gt = cursor; t_eq = cursor + tpitch; t_sbe = cursor + 2 * tpitch; cursor += 3 * tpitch; }
     else { t_gt = dv.tile_a + (int64_t)row * dv.ntiles; t_eq = dv.tile_b + (int64_t)row * dv.ntiles; t_sbe = dv.tile_c + (int64_t)row * dv.ntiles; }
+    if (dv.emit_masks_smem) { slab_gm = cursor; slab_em = cursor + dv.slab_pitch; cursor += 2 * dv.slab_pitch; }
+    else { slab_gm = dv.slab_c + (int64_t)row * dv.slab_pitch; slab_em = dv.slab_d + (int64_t)row * dv.slab_pitch; }
     uint32_t* sbits = cursor;                      // the candidates' value bits and
     uint32_t* sidx = cursor + dv.emit_keys_cap;    // coordinates, when they fit
     const bool cached = ncand <= (uint32_t)dv.emit_keys_cap;
-    // a thread's own tile segment, fetched now so that the wait overlaps the copy below
+    if (cached && threadIdx.x == 0) {
+        // both arrays in two bulk copies: nothing is staged in registers, and all of it is in
+        // flight at once (rows of the candidate arrays are 16-byte aligned, cap % 4 == 0)
+        const uint32_t bytes = ((ncand + 3u) & ~3u) * (uint32_t)sizeof(uint32_t);
+        mbar_init(bar, 1);
+        mbar_expect_tx(bar, 2u * bytes);
+        bulk_load(sbits, cv, bytes, bar);
+        bulk_load(sidx, ci, bytes, bar);
+    }
+    // a thread's own tile segment, fetched now so that the wait overlaps the copies
     const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
     const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
     const bool own_tile = dv.ntiles <= kSelThreads;
     uint32_t my_so = 0u, my_sc = 0u;
     if (own_tile && threadIdx.x < dv.ntiles) { my_so = __ldg(so + threadIdx.x); my_sc = __ldg(sc + threadIdx.x); }
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
     uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
-    for (uint32_t p0 = threadIdx.x; p0 < ncand; p0 += 4 * kSelThreads) {
-        uint32_t bits[4], idx[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t p = p0 + j * kSelThreads;
-            if (p < ncand) {
-                bits[j] = __ldg(cv + p);
-                if (cached) idx[j] = __ldg(ci + p);
-            }
+    if (cached) {
+        // thread 0 polls (bounded); the others wait at the barrier, then each thread observes
+        // the completed phase itself so that the copied data is visible to it
+        int ok = 1;
+        if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
+        if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
+        (void)mbar_wait_bounded(bar, 0, dv.stats);
+        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+            const uint32_t kk = order_key<KIND>(sbits[p]);
+            klo = kk < klo ? kk : klo;
+            khi = kk > khi ? kk : khi;
         }
+    } else {
+        for (uint32_t p0 = threadIdx.x; p0 < ncand; p0 += 4 * kSelThreads) {
+            uint32_t bits[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t p = p0 + j * kSelThreads;
-            if (p < ncand) {
-                if (cached) { sbits[p] = bits[j]; sidx[p] = idx[j]; }
-                const uint32_t kk = order_key<KIND>(bits[j]);
-                klo = kk < klo ? kk : klo;
-                khi = kk > khi ? kk : khi;
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t p = p0 + j * kSelThreads;
+                if (p < ncand) bits[j] = __ldg(cv + p);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t p = p0 + j * kSelThreads;
+                if (p < ncand) {
+                    const uint32_t kk = order_key<KIND>(bits[j]);
+                    klo = kk < klo ? kk : klo;
+                    khi = kk > khi ? kk : khi;
+                }
             }
         }
     }
-    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
     block_min_max(klo, khi, sm);
     auto bits_at = [&](uint32_t p) -> uint32_t { return cached ? sbits[p] : __ldg(cv + p); };
     auto idx_at = [&](uint32_t p) -> uint32_t { return cached ? sidx[p] : __ldg(ci + p); };
@@ -669,7 +688,10 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const float* hr = a.Xhat + (int64_t)row * dv.ld;
     const uint32_t lt = (1u << lane) - 1u;
     // (which candidates those are is in the slabs' ballots: only they are fetched again)
-    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+    // Three quarters of the warps do that; the last quarter publishes the range records
+    // meanwhile (both are bound by the latency of their scattered stores).
+    constexpr int kWriteWarps = (kSelThreads / 32) * 3 / 4;
+    for (int64_t sl = warp; warp < kWriteWarps && sl < nslab; sl += kWriteWarps) {
         const uint32_t bg = slab_gm[sl], be = slab_em[sl];
         const bool gt = (bg >> lane) & 1u, eq = (be >> lane) & 1u;
         if (gt | eq) {
@@ -687,7 +709,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
             }
         }
     }
-    publish_ranges(dv, row, tp);
+    if (warp >= kWriteWarps) publish_ranges(dv, row, tp, threadIdx.x - kWriteWarps * 32, kSelThreads - kWriteWarps * 32);
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
