@@ -574,7 +574,6 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const bool own_tile = dv.ntiles <= kSelThreads;
     uint32_t my_so = 0u, my_sc = 0u;
     if (own_tile && threadIdx.x < dv.ntiles) { my_so = __ldg(so + threadIdx.x); my_sc = __ldg(sc + threadIdx.x); }
-    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) { t_gt[t] = 0u; t_eq[t] = 0u; }
     uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
     if (cached) {
         // thread 0 polls (bounded); the others wait at the barrier, then each thread observes
@@ -629,53 +628,58 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         }
     }
 
-    // 2. counts per tile and per slab.  kBatch slabs at a time so that the index loads of a
-    // batch are in flight together.
-    constexpr int kBatch = 8;
-    for (int64_t s0 = warp; s0 < nslab; s0 += (kSelThreads / 32) * kBatch) {
-        uint32_t idx[kBatch];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
-            const uint32_t p = (uint32_t)(sl << 5) + lane;
-            idx[u] = (sl < nslab && p < ncand) ? idx_at(p) : 0u;
+    // 2. per slab of 32 candidates: which keys lie above T, which equal it (ballots), how many
+    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+        const uint32_t p = (uint32_t)(sl << 5) + lane;
+        bool gt = false, eq = false;
+        if (p < ncand) {
+            const uint32_t kk = key_at(p);
+            gt = kk > T;
+            eq = kk == T;
         }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int64_t sl = s0 + (int64_t)u * (kSelThreads / 32);
-            if (sl >= nslab) break;
-            const uint32_t p = (uint32_t)(sl << 5) + lane;
-            bool gt = false, eq = false;
-            if (p < ncand) {
-                const uint32_t kk = key_at(p);
-                gt = kk > T;
-                eq = kk == T;
-                if (gt | eq) atomicAdd(gt ? &t_gt[idx[u] / kTile] : &t_eq[idx[u] / kTile], 1u);
-            }
-            const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-            if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); slab_gm[sl] = bg; slab_em[sl] = be; }
-        }
+        const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); slab_gm[sl] = bg; slab_em[sl] = be; }
     }
     __syncthreads();
 
-    // 3. prefixes.  Tiles: t_gt <- keys above T before the tile, t_eq <- equal keys before it.
+    // 3. prefixes.  Slabs first: with them the number of keys above / equal to T before any
+    // candidate position follows from one prefix and one ballot ...
+    uint32_t tot_g, tot_e;
+    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
+    auto before = [&](uint32_t pos, uint32_t& g, uint32_t& e) {
+        const uint32_t s0 = pos >> 5;
+        if ((int64_t)s0 < nslab) {
+            const uint32_t below = (1u << (pos & 31u)) - 1u;
+            g = slab_g[s0] + __popc(slab_gm[s0] & below);
+            e = slab_e[s0] + __popc(slab_em[s0] & below);
+        } else {
+            g = tot_g;
+            e = tot_e;
+        }
+    };
+    // ... so a tile, whose candidates are consecutive, gets its two counts as differences
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
+        const uint32_t cnt = own_tile ? my_sc : sc[t];
+        uint32_t g0 = 0, e0 = 0, g1 = 0, e1 = 0;
+        if (cnt) {
+            const uint32_t first = own_tile ? my_so : so[t];
+            before(first, g0, e0);
+            before(first + cnt, g1, e1);
+        }
+        t_gt[t] = g1 - g0;
+        t_eq[t] = e1 - e0;
+    }
+    __syncthreads();
+    // tiles: t_gt <- keys above T before the tile, t_eq <- equal keys before it
     uint32_t tot_a, tot_b;
     block_scan_pair(t_gt, t_eq, dv.ntiles, sm, s_carry, &tot_a, &tot_b);
-    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_a, &tot_b);
     uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
     for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
         const uint32_t gb = t_gt[t], eb = t_eq[t];
         tp[t] = gb + (eb < r ? eb : r);
         // the two flat prefixes at the tile's first candidate: t_gt <- above, t_sbe <- equal
         uint32_t pg = 0, pe = 0;
-        if (own_tile ? my_sc : sc[t]) {
-            const uint32_t first = own_tile ? my_so : so[t], s0 = first >> 5;
-            // keys above / equal to T before `first`: whole slabs from the prefixes, the rest of
-            // its own slab from the slab's ballots
-            const uint32_t below = (1u << (first & 31u)) - 1u;
-            pg = slab_g[s0] + __popc(slab_gm[s0] & below);
-            pe = slab_e[s0] + __popc(slab_em[s0] & below);
-        }
+        if (own_tile ? my_sc : sc[t]) before(own_tile ? my_so : so[t], pg, pe);
         t_gt[t] = pg;
         t_sbe[t] = pe;
     }
