@@ -692,9 +692,13 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     const float* hr = a.Xhat + (int64_t)row * dv.ld;
     const uint32_t lt = (1u << lane) - 1u;
     // (which candidates those are is in the slabs' ballots: only they are fetched again)
-    // Three quarters of the warps do that; the last quarter publishes the range records
-    // meanwhile (both are bound by the latency of their scattered stores).
-    constexpr int kWriteWarps = (kSelThreads / 32) * 3 / 4;
+    // Some of the warps do that while the others publish the range records (both are bound by
+    // the latency of their scattered stores); the split follows the two amounts of work, one
+    // slab per warp iteration here, 32 records per warp iteration there.
+    const int nwarps = kSelThreads / 32;
+    const int64_t pub_iters = (dv.ntiles * (dv.row_ptr[row + 1] - dv.row_ptr[row]) + 31) / 32;
+    int kWriteWarps = (int)((nslab * nwarps + (nslab + pub_iters) / 2) / (nslab + pub_iters));
+    kWriteWarps = kWriteWarps < 1 ? 1 : (kWriteWarps > nwarps - 1 ? nwarps - 1 : kWriteWarps);
     for (int64_t sl = warp; warp < kWriteWarps && sl < nslab; sl += kWriteWarps) {
         const uint32_t bg = slab_gm[sl], be = slab_em[sl];
         const bool gt = (bg >> lane) & 1u, eq = (be >> lane) & 1u;
