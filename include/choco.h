@@ -8,16 +8,16 @@
  *     Xhat [n, ld]   public copies x^_i                          (Algorithm 1)
  *     S    [n, ld]   neighbour sums s_i = sum_j w_ij x^_j        (the "3 vectors per
  *                    node" storage of Section 3, last paragraph)
- *     G    [n, ld]   stochastic gradients g_i, read-only          (Algorithm 1, line 8)
+ *     G    [n, ld]   stochastic gradients g_i, read-only          (Algorithm 1)
  * A fresh run starts from Xhat = S = 0 (Algorithm 1, input); any state with
  * S = W Xhat resumes one.  Only the first d elements of each row are used.
  *
  * One step call performs, for every worker i at once,
- *     q_i    = Q(x_i - x^_i)                     Algorithm 1, line 3
- *     x^_i  += q_i                               line 6 with j = i
- *     s_i   += sum_j w_ij q_j                    line 6 for all neighbours j, folded into s_i
+ *     q_i    = Q(x_i - x^_i)                     Algorithm 1: compression
+ *     x^_i  += q_i                               update of the public copy (j = i)
+ *     s_i   += sum_j w_ij q_j                    the same for all neighbours j, folded into s_i
  *     x_i    = (x_i - eta g_i) + gamma (s_i - x^_i)
- *                                                line 9, then line 2 of the next iteration
+ *                                                gradient step, then the gossip step of the next iteration
  *                                                (sum_j w_ij (x^_j - x^_i) = s_i - x^_i as
  *                                                rows of W sum to one)
  * i.e. the gossip scheme h of Appendix A.1 ("Example: CHOCO-SGD"), with the communication
@@ -105,15 +105,16 @@ int choco_destroy(choco_ctx* ctx);
 int choco_gossip_step(choco_ctx* ctx, float* X, float* Xhat, float* S, float gamma, void* stream);
 
 /*
- * choco_sgd_step -- Algorithm 1, lines 3-9 of iteration t followed by line 2 of iteration
- * t+1, with g_i = G[i] the gradient the caller evaluated at the current x_i (line 8).
+ * choco_sgd_step -- Algorithm 1: iteration t from its compression step to its gradient step,
+ * followed by the gossip step of iteration t+1, with g_i = G[i] the gradient the caller
+ * evaluated at the current x_i.
  * G: DEVICE pointer, read-only.  Advances the step counter by one.
  */
 int choco_sgd_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float eta,
                    float gamma, void* stream);
 
 /*
- * choco_sgd_momentum_step -- Algorithm 2 (CHOCO-SGD with momentum): line 9 becomes
+ * choco_sgd_momentum_step -- Algorithm 2 (CHOCO-SGD with momentum): the gradient step becomes
  *     m_i = (g_i + lambda x_i) + beta m_i ;   x_i = (x_i - eta m_i) + gamma (s_i - x^_i)
  * with M [n, ld] the local momentum memory (DEVICE, updated in place, starts at 0).
  */

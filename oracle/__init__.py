@@ -226,7 +226,7 @@ def difference(x: np.ndarray, xhat: np.ndarray) -> np.ndarray:
 
 
 def compress(p: Params, v: np.ndarray, step: int, worker: int) -> Message:
-    """q = Q(v) for worker `worker` at step `step` (Algorithm 1, line 3)."""
+    """q = Q(v) for worker `worker` at step `step` (Algorithm 1, the compression step)."""
     d = v.shape[0]
     if p.kind == "identity":
         return Message(q=v.copy())
@@ -357,7 +357,7 @@ def alg1_literal(w, p: Params, x0: np.ndarray, grads, eta: float, gamma: float,
                  steps: int, final_gossip: bool = False) -> np.ndarray:
     """Algorithm 1 with per-neighbour copies.  `x0` is x^(-1/2) [n, d]; `grads(t, X)`
     returns the [n, d] float32 gradients at x^(t) (or None for pure gossip).  Returns
-    x^(T-1/2), the iterate after the last SGD step, or x^(T) (one more line 2) with
+    x^(T-1/2), the iterate after the last SGD step, or x^(T) (one more gossip step) with
     `final_gossip`.  float32 throughout."""
     n, d = x0.shape
     x = x0.astype(np.float32).copy()
@@ -366,14 +366,14 @@ def alg1_literal(w, p: Params, x0: np.ndarray, grads, eta: float, gamma: float,
     # hat[i][j]: worker i's copy of x^_j
     hat = [{j: np.zeros(d, dtype=np.float32) for j in nbrs[i]} for i in range(n)]
     for t in range(steps):
-        _line2(x, hat, nbrs, wts, gamma)                       # line 2
-        q = [compress(p, difference(x[i], hat[i][i]), t, i).q for i in range(n)]   # line 3
-        for i in range(n):                                     # lines 4-7
+        _line2(x, hat, nbrs, wts, gamma)                       # gossip step
+        q = [compress(p, difference(x[i], hat[i][i]), t, i).q for i in range(n)]   # compression
+        for i in range(n):                                     # exchange q, update the copies
             for j in nbrs[i]:
                 hat[i][j] = hat[i][j] + q[j]
-        g = grads(t, x) if grads is not None else None         # line 8
+        g = grads(t, x) if grads is not None else None         # gradient evaluation
         if g is not None:
-            x = x - np.float32(eta) * g                        # line 9
+            x = x - np.float32(eta) * g                        # gradient step
     if final_gossip:
         _line2(x, hat, nbrs, wts, gamma)
     return x
@@ -382,7 +382,7 @@ def alg1_literal(w, p: Params, x0: np.ndarray, grads, eta: float, gamma: float,
 def alg4_error_feedback(w, p: Params, x0: np.ndarray, grads, eta: float, gamma: float,
                         steps: int, final_gossip: bool = False) -> np.ndarray:
     """Algorithm 4: the same iterates with v = x^(t) - x^(t-1) + m, q = Q(v),
-    m <- v - q in place of line 3, x^(-1) = 0."""
+    m <- v - q in place of the compression step, x^(-1) = 0."""
     n, d = x0.shape
     x = x0.astype(np.float32).copy()
     nbrs = [[int(c) for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]]] for i in range(n)]

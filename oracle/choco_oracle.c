@@ -9,7 +9,8 @@
  * What follows the paper:
  *   - the compression operators of Appendix C ("Compression Schemes"): top_a,
  *     random_a (biased form), gsgd_b (biased and unbiased forms), scaled sign;
- *   - the per-worker updates of Algorithm 1 (lines 2, 3, 6, 9) in the form that
+ *   - the per-worker updates of Algorithm 1 (gossip, compression, public copies,
+ *     gradient step) in the form that
  *     keeps three vectors per worker (x_i, x^_i and s_i = sum_j w_ij x^_j), the
  *     storage the end of Section 3 describes;
  *   - the consensus distance of Section 6, (1/n) sum_i ||x_i - xbar||^2.
@@ -138,7 +139,7 @@ static uint32_t f32_bits(float f)
     return u;
 }
 
-/* v = x - x^ (Algorithm 1, line 3, the argument of Q) */
+/* v = x - x^ (Algorithm 1, the argument of Q in the compression step) */
 void oracle_difference(const float* x, const float* xhat, int64_t d, float* v)
 {
     for (int64_t c = 0; c < d; ++c) v[c] = x[c] - xhat[c];
@@ -295,18 +296,18 @@ int oracle_compress_qsgd(const float* v, const float* u, int64_t d, int32_t s, i
 
 /*
  * One worker's update in three-vector form.  With q_j = Q(x_j - x^_j) already formed
- * for this worker and its neighbours (Algorithm 1 line 3):
- *     x^_i  <- x^_i + q_i                              (line 6 with j = i)
- *     s_i   <- s_i + sum_j w_ij q_j                    (line 6 for all j, folded into
+ * for this worker and its neighbours (Algorithm 1, compression step):
+ *     x^_i  <- x^_i + q_i                              (public copy, j = i)
+ *     s_i   <- s_i + sum_j w_ij q_j                    (the same for all j, folded into
  *                                                       s_i = sum_j w_ij x^_j)
- *     x_i   <- x_i + gamma (s_i - x^_i) - eta g_i      (line 2 of the next iteration,
+ *     x_i   <- x_i + gamma (s_i - x^_i) - eta g_i      (gossip step of the next iteration,
  *                                                       = gamma sum_j w_ij (x^_j - x^_i)
  *                                                       because rows of W sum to one,
- *                                                       and line 9)
+ *                                                       and the gradient step)
  * Operation order, fixed here because the paper does not give one: neighbours are
  * added in the order given (CSR column order), acc = +0; acc = acc + w_ij * q_j; then
- * s' = s + acc; c = s' - x^'; x' = (x - eta * g) + gamma * c, i.e. line 9 and then
- * line 2 (x' = x + gamma * c when g is NULL).  For sparse q (mask given) coordinates that no neighbour touches
+ * s' = s + acc; c = s' - x^'; x' = (x - eta * g) + gamma * c, i.e. the gradient step and then
+ * the gossip step (x' = x + gamma * c when g is NULL).  For sparse q (mask given) coordinates that no neighbour touches
  * leave s and x^ as they are.
  */
 void oracle_apply_row(int64_t d, float* x, float* xhat, float* s, const float* g,
@@ -336,7 +337,7 @@ void oracle_apply_row(int64_t d, float* x, float* xhat, float* s, const float* g
 }
 
 /*
- * Momentum variant (Algorithm 2): line 9 becomes
+ * Momentum variant (Algorithm 2): the gradient step becomes
  *     v <- (g + lambda x) + beta v ;  x <- x - eta v
  * with x the iterate the gradient was taken at, followed by the gossip correction of
  * the next iteration as in oracle_apply_row:

@@ -1,4 +1,4 @@
-// The update half of a CHOCO step (Algorithm 1, lines 6, 2 and 9; Algorithm 2 for the
+// The update half of a CHOCO step (Algorithm 1: public copies, gossip, gradient step; Algorithm 2 for the
 // momentum variant): every worker reads its neighbours' messages back and forms
 //     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
 //     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i).

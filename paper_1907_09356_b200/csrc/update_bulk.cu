@@ -1,5 +1,6 @@
-// Update kernel for sparse Q (top_a / random_a), bulk-copy variant: Algorithm 1, lines 6, 2
-// and 9 (Algorithm 2 with momentum) for one tile of one worker per block,
+// Update kernel for sparse Q (top_a / random_a), bulk-copy variant: Algorithm 1, the update of
+// the public copies, the gossip step and the gradient step (Algorithm 2 with momentum) for one
+// tile of one worker per block,
 //     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
 //     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i).
 //

@@ -1,5 +1,5 @@
-// Update kernel for dense Q (scaled sign, gsgd_b, identity): Algorithm 1, lines 6, 2 and 9
-// (Algorithm 2 with momentum).  Every thread decodes its neighbours' packed messages for the
+// Update kernel for dense Q (scaled sign, gsgd_b, identity): Algorithm 1, the update of the
+// public copies, the gossip step and the gradient step (Algorithm 2 with momentum).  Every thread decodes its neighbours' packed messages for the
 // four coordinates it owns and forms
 //     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
 //     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i).

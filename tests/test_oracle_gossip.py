@@ -210,7 +210,7 @@ def test_momentum_variant_matches_algorithm2():
     eta, gamma, lam, beta = 0.1, 0.2, 1e-2, 0.9
     oracle.step(w, oracle.Params("identity"), X, Xh, S, G, eta, gamma, 0, M=M, lam=lam, beta=beta)
     f = np.float32
-    v1 = (G + f(lam) * X0) + f(beta) * M0                     # Algorithm 2, line 9
+    v1 = (G + f(lam) * X0) + f(beta) * M0                     # Algorithm 2, momentum update
     assert np.array_equal(M, v1)
     W = w.dense()
     want = (X0.astype(np.float64) - eta * v1) + gamma * ((W - np.eye(n)) @ X0.astype(np.float64))

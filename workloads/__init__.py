@@ -290,7 +290,7 @@ WORKLOADS = {
 
 
 # --------------------------------------------------------------------------
-# the convex problem of the d = 2000 workload (caller-side gradient, Alg. 1 line 8)
+# the convex problem of the d = 2000 workload (caller-side gradient of Algorithm 1)
 # --------------------------------------------------------------------------
 
 
@@ -299,7 +299,7 @@ class LogisticProblem:
 
     Features ~ N(0, 1/d), labels sign(a . w*) for a seeded planted w*; all samples
     are sorted by label and dealt contiguously to the workers.  The gradient is the
-    caller's job in Algorithm 1 (line 8); it is evaluated here in float64 and handed,
+    caller's job in Algorithm 1; it is evaluated here in float64 and handed,
     as float32, to whichever implementation is being driven.
     """
 
