@@ -1,6 +1,6 @@
 // Update kernel for scaled sign and bucketed gsgd_b, bulk-copy variant (rows 16-byte
-// aligned, d a multiple of 4): the same arithmetic as update_dense_kernel, Algorithm 1 lines
-// 6, 2 and 9 followed by the compression of x' - x^' for the next step, with the x, x^, s, g
+// aligned, d a multiple of 4): the same arithmetic as update_dense_kernel (Algorithm 1:
+// public copies, gossip step, gradient step) followed by the compression of x' - x^' for the next step, with the x, x^, s, g
 // (and momentum) tiles of 2048 coordinates staged in shared memory by asynchronous bulk
 // copies.  The neighbours' packed message pieces that a thread needs are small; they are
 // fetched into registers while the copies are in flight.
