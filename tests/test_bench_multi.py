@@ -67,3 +67,33 @@ def test_reference_arm_runs_on_rank0_only(rank):
     assert line["impl"] == "reference" and line["n_gpus"] == 2
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_byte_model_of_the_step():
+    """Minimum bytes a step must move: each dense array once, messages once per reader."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import workloads
+    wl = workloads.WORKLOADS["c4_torus64_topk"]
+    w = wl.mixing()
+    N, k, nnz = 64 * 1_000_000, 10_000, 64 * 5
+    assert bench.message_bytes(wl) == 8 * k
+    want = 20 * N + 8 * k * 64 + 8 * k * (nnz - 64) + 4 * (64 * k + nnz * k)
+    assert bench.step_min_bytes(wl, w) == want == 1_320_960_000
+    assert bench.update_kernel_bytes(wl, w) == 20 * N + 8 * k * nnz + 4 * (64 * k + nnz * k)
+
+    wl = workloads.WORKLOADS["c5_ring32_qsgd"]
+    w = wl.mixing()
+    d = 25_557_032
+    per_worker = 4 * ((d + 511) // 512) + 4 * ((d + 31) // 32) + d // 2      # norms, sign plane, nibbles
+    assert bench.message_bytes(wl) == per_worker
+    assert bench.step_min_bytes(wl, w) == 28 * 32 * d + per_worker * 32 * 3  # written once, read by two neighbours
+    assert abs(bench.step_min_bytes(wl, w) - 24.45e9) < 0.01e9
+
+    # per layer: the entries kept and the message are sums over the layers
+    wl = workloads.WORKLOADS["l3_ring8_topk_layers"]
+    sizes = wl.layer_sizes()
+    assert bench.entries_per_row(wl) == sum(max(1, s // 100) for s in sizes)
+    assert bench.message_bytes(wl) == 8 * bench.entries_per_row(wl)
+    wl = workloads.WORKLOADS["l3_ring8_sign_layers"]
+    assert bench.message_bytes(wl) == sum(4 * ((s + 31) // 32) + 4 for s in sizes)
