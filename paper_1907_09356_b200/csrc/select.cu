@@ -58,22 +58,25 @@ __device__ __forceinline__ bool any_row_flagged(const Dev& dv, uint32_t mask)
     return __syncthreads_or(mine) != 0;
 }
 
-// With `rescue` the grid is one-dimensional and its blocks stride over the spans of the rows
-// flagged kRowRescue only (normally none: every block then returns at once).  level 0 counts
-// the first digit (top 11 bits) of every key; level 1 serves rows flagged kRowRefine only and
-// counts the next 11 bits of the keys whose first digit is the one row_lo holds.
+// level 0 counts the first digit (top 11 bits) of every key; level 1 serves rows flagged
+// kRowRefine only and counts the next 11 bits of the keys whose first digit is the one row_lo
+// holds.  With `rescue` only rows flagged kRowRescue are served.  Whenever rows are picked by
+// flag the grid is one-dimensional and its blocks stride over the spans of those rows
+// (normally there are none, and every block returns at once).
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads) hist_kernel(Dev dv, StepArgs a, int rescue, int level)
 {
     __shared__ uint32_t h[kHistBins];
-    if (rescue && !any_row_flagged(dv, kRowRescue)) return;
-    const int row_begin = rescue ? 0 : (int)blockIdx.y, row_end = rescue ? dv.n : (int)blockIdx.y + 1;
+    // rows served: those flagged for the rescue (if this is one) and, at level 1, for refinement;
+    // with either condition the grid is one-dimensional and strides over the rows that qualify
+    const uint32_t need = (rescue ? kRowRescue : 0u) | (level ? kRowRefine : 0u);
+    const bool strided = need != 0u;
+    if (strided && !any_row_flagged(dv, kRowRefine | kRowRescue)) return;
+    const int row_begin = strided ? 0 : (int)blockIdx.y, row_end = strided ? dv.n : (int)blockIdx.y + 1;
     for (int row = row_begin; row < row_end; ++row) {
-        const uint32_t flags = (rescue || level) ? dv.row_flags[row] : 0u;
-        if (rescue && !(flags & kRowRescue)) continue;
-        if (level && !(flags & kRowRefine)) continue;
+        if (need && (dv.row_flags[row] & need) != need) continue;
         const uint32_t first = level ? dv.row_lo[row] >> 21 : 0u;
-        for (int64_t sp = blockIdx.x; sp < dv.nspans; sp += rescue ? (int64_t)gridDim.x : dv.nspans) {
+        for (int64_t sp = blockIdx.x; sp < dv.nspans; sp += strided ? (int64_t)gridDim.x : dv.nspans) {
             for (int b = threadIdx.x; b < kHistBins; b += kThreads) h[b] = 0u;
             __syncthreads();
             const int64_t c0 = sp * kSpan;
@@ -737,8 +740,9 @@ static cudaError_t prepare_impl(const Dev& dv, const StepArgs& a, cudaStream_t s
     if (KIND == SEL_TOPK) {
         const dim3 hgrid((unsigned)dv.nspans, (unsigned)dv.n);
         for (int level = 0; level < 2; ++level) { // the second round returns at once unless a bin was too full
-            if (a.vec) hist_kernel<true><<<hgrid, kThreads, 0, st>>>(dv, a, 0, level);
-            else hist_kernel<false><<<hgrid, kThreads, 0, st>>>(dv, a, 0, level);
+            const dim3 g = level ? dim3((unsigned)(dv.nspans < 1024 ? dv.nspans : 1024)) : hgrid;
+            if (a.vec) hist_kernel<true><<<g, kThreads, 0, st>>>(dv, a, 0, level);
+            else hist_kernel<false><<<g, kThreads, 0, st>>>(dv, a, 0, level);
             bound_kernel<<<dv.n, kSelThreads, 0, st>>>(dv, 0, level);
         }
         *a.launches += 4;
