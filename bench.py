@@ -36,6 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 # launch (29.70 B per coordinate), as the capture of the full-size workload would be too large.
 NCU_TRAFFIC = {("c4_torus64_topk", "update"): 1.367e9,
                ("p_ring8_qsgd", "update"): 1.993e9,
+               ("p_ring8_sign", "update"): 1.856e9,
                ("c5_ring32_qsgd", "update"): 29.70 * 32 * 25_557_032}
 
 
