@@ -33,6 +33,30 @@
  * enqueued.  Calls on one context must be issued in stream order, from one host thread at
  * a time.  `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  * Step calls are asynchronous: they enqueue kernels on `stream` and return.
+ *
+ * Device-side waits.  The kernels stage their tiles with asynchronous copies and wait for them
+ * with a bounded number of polls (about 4 million, seconds of wall time; a copy normally lands
+ * within microseconds).  A block whose wait runs out counts it in choco_stats.device_timeouts,
+ * waits once more (again bounded) for its copies in flight and returns without writing its part
+ * of X, Xhat and S: nothing hangs and nothing faults, but the arrays are then no valid state.
+ * Step calls do not synchronise and therefore cannot report this themselves; every call that
+ * does synchronise `stream` (choco_get_stats, choco_read_message, choco_consensus_error,
+ * choco_sgd_step_host) reads the counter and returns CHOCO_ERR_TIMEOUT once it is non-zero, and
+ * from then on every step call on the context returns CHOCO_ERR_TIMEOUT without enqueuing
+ * anything.  Recover by restoring X, Xhat and S from a checkpoint into a fresh context
+ * (choco_set_step resumes the generator).
+ *
+ * Memory reads: rows that are not 16-byte aligned (base pointer or ld * 4 not a multiple of 16, or
+ * d not a multiple of 4) are staged in whole 16-byte units, so up to 12 bytes before the first and
+ * after the last element of a row are read (never written, and never used): the arrays must lie in
+ * memory that is readable up to the enclosing 16-byte boundaries, which holds for anything
+ * cudaMalloc or a caching allocator hands out.
+ *
+ * L2 residency (TOPK / RANDK contexts): choco_init raises the device's persisting-L2 limit
+ * (cudaLimitPersistingL2CacheSize) if it is below what the context's message arena needs, and never
+ * lowers it; the selection and update kernels are launched with an access-policy window over that
+ * arena (a per-launch attribute: no stream attribute is left on `stream`).  choco_destroy calls
+ * cudaCtxResetPersistingL2Cache, which returns all persisting lines on the device to normal.
  */
 #ifndef CHOCO_H_
 #define CHOCO_H_
@@ -53,7 +77,9 @@ typedef enum {
     CHOCO_ERR_CUDA = -4,        /* a CUDA runtime call failed (see choco_last_cuda_error)      */
     CHOCO_ERR_MISALIGNED = -5,  /* a state pointer is not 4-byte aligned                       */
     CHOCO_ERR_UNSUPPORTED = -6, /* valid in the paper, not built (e.g. an odd QSGD bucket)     */
-    CHOCO_ERR_TOO_LARGE = -7    /* a size exceeds a documented limit                           */
+    CHOCO_ERR_TOO_LARGE = -7,   /* a size exceeds a documented limit                           */
+    CHOCO_ERR_TIMEOUT = -8      /* a bounded wait inside a kernel ran out: the state arrays are */
+                                /* no longer a valid CHOCO state (see "Device-side waits")      */
 } choco_status;
 
 /* Compression operator Q (Appendix C, "Compression Schemes"). */
@@ -77,8 +103,8 @@ typedef struct {
 
 /*
  * choco_init -- Algorithm 1, "input": the communication graph with its mixing matrix W
- * (Assumption 1), the compression operator and the shared random seed (Appendix C,
- * random_a: "if it knows the random seed").
+ * (Assumption 1), the compression operator and the random seed that sender and receiver of a
+ * random_a message share (Appendix C: the receiver regenerates the positions from it).
  *   n, d, ld     workers, coordinates per worker, row pitch of all state arrays (ld >= d;
  *                d < 2^31).
  *   w_row_ptr[n+1], w_col[nnz], w_val[nnz]   HOST pointers to W in CSR; copied.  Every row
@@ -220,7 +246,11 @@ int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* str
  * it, for the life of the process; larger d returns CHOCO_ERR_TOO_LARGE and enqueues nothing.
  * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
  * First use on a device looks up the address of that array (a one-time query, done with that
- * device current); make this first call before starting any stream capture.
+ * device current).  With CUDA's lazy module loading that first use may also load the kernels'
+ * code and the array itself onto the device, which takes device memory: make one warm-up call
+ * at start-up, while memory is still to be had and before starting any stream capture.  The
+ * looked-up address is cached per device for the life of the process and is not refreshed
+ * after cudaDeviceReset.
  * All calls on a device share the array.  Each call overwrites every partial it later reads,
  * so nothing carries over from one call to the next, but two calls whose kernels overlap on
  * the GPU (different streams, no ordering between them) race on it: order them.
@@ -291,7 +321,17 @@ typedef struct {
     uint64_t graph_replays;    /* step calls served by replaying a captured CUDA graph          */
     uint64_t rescued_rows;     /* rows re-collected by the grid-wide kernels (choco_set_rescue) */
 } choco_stats;
+/* Fills *out; returns CHOCO_ERR_TIMEOUT (with *out filled) if device_timeouts is non-zero. */
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
+
+/*
+ * Test hook for the timeout path described at the top: the number of polls a kernel of this
+ * context spends on its first wait before it gives up (default 4 194 304).  With 0 every block
+ * gives up at once, then sits out its copies in the second, still bounded, wait and returns --
+ * the only way to see CHOCO_ERR_TIMEOUT without a stalled memory system.  The state arrays are
+ * invalid after such a step.  Not for production use.
+ */
+int choco_debug_set_wait_polls(choco_ctx* ctx, uint32_t polls);
 
 /*
  * Optional timing of the update kernel (the one pass that streams X, Xhat, S and G): after

@@ -4,7 +4,7 @@ Thin numpy/ctypes layer over ``choco_oracle.c`` (the arithmetic lives there) plu
 three drivers written straight from the paper:
 
 * :func:`step`            -- one call of the three-vector form (Section 3, last
-  paragraph): q = Q(x - x^); x^ += q; s += W q; x += gamma (s - x^) - eta g.
+  paragraph): q = Q(x - x^); x^ += q; s += W q; x = (x - eta g) + gamma (s - x^).
 * :func:`alg1_literal`    -- Algorithm 1 as printed, every worker holding its own
   copy of x^_j for each neighbour (tiny sizes; cross-check of :func:`step`).
 * :func:`alg4_error_feedback` -- the error-feedback rewrite (Algorithm 4).
@@ -274,21 +274,26 @@ def _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M=None, lam=0.0, beta=0.0)
 def step(w, p: Params, X: np.ndarray, Xhat: np.ndarray, S: np.ndarray,
          G: Optional[np.ndarray], eta: float, gamma: float, t: int,
          rows: Optional[Sequence[int]] = None, M: Optional[np.ndarray] = None,
-         lam: float = 0.0, beta: float = 0.0) -> dict:
+         lam: float = 0.0, beta: float = 0.0, executor=None) -> dict:
     """One call on float32 [n, d] arrays, in place.  Returns {worker: Message}.
 
     With `rows`, only those workers are updated (their neighbours' messages are still
     formed): a way to check single rows of a large problem.  With `M` the momentum
-    variant of Algorithm 2 is applied instead of the plain SGD step.
+    variant of Algorithm 2 is applied instead of the plain SGD step.  `executor` (a
+    concurrent.futures executor of threads; the C routines run without the interpreter
+    lock) only spreads the per-worker calls over host cores: all messages are formed
+    before any row is updated, and rows are independent of each other, so the result
+    is the same.
     """
     n = X.shape[0]
     todo = list(range(n)) if rows is None else list(rows)
     need = set()
     for i in todo:
         need.update(int(c) for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]])
-    msgs = {j: compress(p, difference(X[j], Xhat[j]), t, j) for j in sorted(need)}
-    for i in todo:
-        _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M, lam, beta)
+    need = sorted(need)
+    run = map if executor is None else executor.map
+    msgs = dict(zip(need, run(lambda j: compress(p, difference(X[j], Xhat[j]), t, j), need)))
+    list(run(lambda i: _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M, lam, beta), todo))
     return msgs
 
 

@@ -300,10 +300,10 @@ int oracle_compress_qsgd(const float* v, const float* u, int64_t d, int32_t s, i
  *     x^_i  <- x^_i + q_i                              (public copy, j = i)
  *     s_i   <- s_i + sum_j w_ij q_j                    (the same for all j, folded into
  *                                                       s_i = sum_j w_ij x^_j)
- *     x_i   <- x_i + gamma (s_i - x^_i) - eta g_i      (gossip step of the next iteration,
- *                                                       = gamma sum_j w_ij (x^_j - x^_i)
- *                                                       because rows of W sum to one,
- *                                                       and the gradient step)
+ *     x_i   <- (x_i - eta g_i) + gamma (s_i - x^_i)    (the gradient step, then the gossip
+ *                                                       step of the next iteration, which is
+ *                                                       gamma sum_j w_ij (x^_j - x^_i)
+ *                                                       because rows of W sum to one)
  * Operation order, fixed here because the paper does not give one: neighbours are
  * added in the order given (CSR column order), acc = +0; acc = acc + w_ij * q_j; then
  * s' = s + acc; c = s' - x^'; x' = (x - eta * g) + gamma * c, i.e. the gradient step and then

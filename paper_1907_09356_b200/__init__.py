@@ -25,15 +25,22 @@ EXPORTS = [
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
-    "choco_last_cuda_error",
+    "choco_last_cuda_error", "choco_debug_set_wait_polls",
     "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
     "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
     "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_graphs",
 ]
 
 
+ERR_TIMEOUT = -8
+
+
 class ChocoError(RuntimeError):
-    pass
+    """A libchoco call returned a negative status; `code` holds it."""
+
+    def __init__(self, message: str, code: int = 0):
+        super().__init__(message)
+        self.code = code
 
 
 class choco_params(ctypes.Structure):
@@ -86,6 +93,7 @@ def load() -> ctypes.CDLL:
         lib.choco_strerror.argtypes = [ctypes.c_int]
         lib.choco_strerror.restype = ctypes.c_char_p
         lib.choco_last_cuda_error.argtypes = [vp]
+        lib.choco_debug_set_wait_polls.argtypes = [vp, ctypes.c_uint32]
         lib.choco_layers_init.argtypes = [ctypes.POINTER(vp), i32, i32, vp, i64, vp, vp, vp,
                                           ctypes.POINTER(choco_params), i64, i64, u64]
         lib.choco_layers_destroy.argtypes = [vp]
@@ -111,7 +119,7 @@ def _check(rc: int, ctx=None) -> None:
         msg = lib.choco_strerror(rc).decode()
         if ctx is not None and rc == -4:
             msg += f" (cudaError {lib.choco_last_cuda_error(ctx)})"
-        raise ChocoError(f"libchoco: {msg} [{rc}]")
+        raise ChocoError(f"libchoco: {msg} [{rc}]", rc)
 
 
 def _ptr(t) -> Optional[int]:
@@ -240,6 +248,11 @@ def choco_get_stats(ctx, stream=None) -> dict:
     st = choco_stats()
     _check(load().choco_get_stats(ctx, ctypes.byref(st), _stream(stream)), ctx)
     return {f: getattr(st, f) for f, _ in choco_stats._fields_}
+
+
+def choco_debug_set_wait_polls(ctx, polls: int) -> None:
+    """Test hook: polls a kernel spends on its first wait for staged copies (0 = give up at once)."""
+    _check(load().choco_debug_set_wait_polls(ctx, polls), ctx)
 
 
 def choco_profile_enable(ctx, max_steps: int) -> None:

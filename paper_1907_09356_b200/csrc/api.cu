@@ -77,33 +77,31 @@ float qsgd_tau(int64_t len, int32_t s, bool biased)
     return (float)(1.0 + (a < b ? a : b));
 }
 
-// Ask the L2 cache to keep the context's hot arena resident for work on `st` (best effort:
-// failures are ignored, the results do not depend on it).  Raises the persisting-L2 carve-out
-// of the current context if it is smaller than the arena needs; it is never lowered here.
-void keep_hot_in_l2(choco_ctx* ctx, cudaStream_t st)
+// Raise the device's persisting-L2 carve-out so that the context's hot arena (messages, range
+// records, per-tile tables) can stay resident while the dense arrays stream past; kernels then
+// carry an access-policy window over it as a launch attribute.  Best effort: failures are
+// ignored, the results do not depend on it.  The limit is never lowered here.
+void reserve_hot_l2(choco_ctx* ctx, void* base, int64_t bytes)
 {
-    ctx->hot_set = true;
-    ctx->hot_stream = st;
     int dev = 0, max_persist = 0, max_window = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return;
     cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev);
     cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev);
-    if (max_persist <= 0 || max_window <= 0) { cudaGetLastError(); return; }
-    const size_t want = std::min<size_t>((size_t)ctx->hot_bytes, (size_t)max_persist / 4 * 3);
+    if (max_persist <= 0 || max_window <= 0 || bytes <= 0) { cudaGetLastError(); return; }
+    const size_t want = std::min<size_t>((size_t)bytes, (size_t)max_persist / 4 * 3);
     size_t have = 0;
     cudaDeviceGetLimit(&have, cudaLimitPersistingL2CacheSize);
     if (have < want) cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want);
+    have = 0;
     cudaDeviceGetLimit(&have, cudaLimitPersistingL2CacheSize);
-    cudaStreamAttrValue av;
-    std::memset(&av, 0, sizeof(av));
-    av.accessPolicyWindow.base_ptr = ctx->hot_base;
-    av.accessPolicyWindow.num_bytes = std::min<size_t>((size_t)ctx->hot_bytes, (size_t)max_window);
-    const double ratio = (double)have / (double)av.accessPolicyWindow.num_bytes;
-    av.accessPolicyWindow.hitRatio = ratio >= 1.0 ? 1.0f : (float)ratio;
-    av.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
-    av.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
-    cudaStreamSetAttribute(st, cudaStreamAttributeAccessPolicyWindow, &av);
     cudaGetLastError(); // best effort
+    if (have == 0) return;
+    const size_t window = std::min<size_t>((size_t)bytes, (size_t)max_window);
+    const double ratio = (double)have / (double)window;
+    ctx->dv.hot_base = base;
+    ctx->dv.hot_bytes = (int64_t)window;
+    ctx->dv.hot_ratio = ratio >= 1.0 ? 1.0f : (float)ratio;
+    ctx->hot_l2 = true;
 }
 
 __global__ void bump_step_kernel(unsigned long long* step) { *step += 1ull; }
@@ -115,6 +113,7 @@ int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, f
               float gamma, float lambda, float beta, void* stream)
 {
     if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->timed_out) return CHOCO_ERR_TIMEOUT; // the arrays are no valid state any more
     if (!aligned4(X) || !aligned4(Xhat) || !aligned4(S) || !aligned4(G) || !aligned4(M))
         return CHOCO_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
@@ -135,7 +134,6 @@ int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, f
     a.vec = (dv.ld % 4 == 0) && aligned16(X) && aligned16(Xhat) && aligned16(S) &&
             (!G || aligned16(G)) && (!M || aligned16(M));
     if (ctx->last_x != X || ctx->last_xhat != Xhat) ctx->prepared = false;
-    if (ctx->hot_base && (!ctx->hot_set || ctx->hot_stream != st)) keep_hot_in_l2(ctx, st);
 
     cudaError_t e = cudaSuccess;
     const bool sparse = dv.kind == CHOCO_Q_TOPK || dv.kind == CHOCO_Q_RANDK;
@@ -193,6 +191,7 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
              float gamma, float lambda, float beta, void* stream)
 {
     if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->timed_out) return CHOCO_ERR_TIMEOUT;
     cudaStream_t st = (cudaStream_t)stream;
     uint64_t mode = 0;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -255,6 +254,21 @@ int run_step(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, fl
     ctx->launches_per_step = ctx->launches - before.launches;
     ctx->graphs[slot].exec = exec;
     ctx->graphs[slot].last_use = ++ctx->graph_clock;
+    return CHOCO_OK;
+}
+
+// For calls that have just synchronised `st`: did a bounded wait inside a kernel run out?
+int check_device_timeouts(choco_ctx* ctx, cudaStream_t st)
+{
+    if (ctx->timed_out) return CHOCO_ERR_TIMEOUT;
+    unsigned long long t = 0;
+    cudaError_t e = cudaMemcpyAsync(&t, &ctx->dv.stats->timeouts, sizeof(t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (t != 0) {
+        ctx->timed_out = true;
+        return CHOCO_ERR_TIMEOUT;
+    }
     return CHOCO_OK;
 }
 
@@ -328,6 +342,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     ctx->dev_step = ctx->graphs_ok && (p->kind == CHOCO_Q_QSGD || p->kind == CHOCO_Q_RANDK);
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
+    dv.wait_polls = kSpinLimit;
     dv.ntiles = (d + kTile - 1) / kTile;
     dv.nspans = (d + kSpan - 1) / kSpan;
     dv.nchunks = (d + kChunk - 1) / kChunk;
@@ -404,8 +419,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             const int64_t hot = q - arena; // the candidates behind it are written once, read once
             dv.cand_idx = (uint32_t*)q; q += b_cand;
             dv.cand_val = (uint32_t*)q; q += b_cand;
-            ctx->hot_base = arena;
-            ctx->hot_bytes = hot;
+            if (e == cudaSuccess) reserve_hot_l2(ctx, arena, hot);
         }
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.hist, (int64_t)n * kHistBins);
         if (e == cudaSuccess) e = dev_alloc(ctx, &dv.tile_a, n * dv.ntiles);
@@ -492,6 +506,7 @@ int choco_destroy(choco_ctx* ctx)
     cudaDeviceSynchronize();
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+    if (ctx->hot_l2) { cudaCtxResetPersistingL2Cache(); cudaGetLastError(); }
     for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
     for (int i = 0; i < 4; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
@@ -555,7 +570,7 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
     cudaError_t e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->prepared = false;
-    return CHOCO_OK;
+    return check_device_timeouts(ctx, st);
 }
 
 int choco_invalidate(choco_ctx* ctx)
@@ -678,7 +693,7 @@ int choco_read_message(choco_ctx* ctx, int32_t worker, int32_t plane, void* host
     cudaError_t e = cudaStreamSynchronize(st);
     if (e == cudaSuccess && *nbytes > 0 && *nbytes <= capacity)
         e = cudaMemcpy(host_dst, src, (size_t)*nbytes, cudaMemcpyDeviceToHost);
-    return e == cudaSuccess ? CHOCO_OK : fail_cuda(ctx, e);
+    return e == cudaSuccess ? check_device_timeouts(ctx, st) : fail_cuda(ctx, e);
 }
 
 int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* stream)
@@ -689,7 +704,7 @@ int choco_consensus_error(choco_ctx* ctx, const float* X, double* out, void* str
                                      ctx->cons_blocks, ctx->cons_out, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(out, ctx->cons_out, sizeof(double), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    return e == cudaSuccess ? CHOCO_OK : fail_cuda(ctx, e);
+    return e == cudaSuccess ? check_device_timeouts(ctx, st) : fail_cuda(ctx, e);
 }
 
 int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
@@ -708,6 +723,18 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream)
     out->kernel_launches = ctx->launches;
     out->graph_replays = ctx->graph_replays;
     out->rescued_rows = h.rescued_rows;
+    if (h.timeouts != 0) ctx->timed_out = true;
+    return ctx->timed_out ? CHOCO_ERR_TIMEOUT : CHOCO_OK;
+}
+
+int choco_debug_set_wait_polls(choco_ctx* ctx, uint32_t polls)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    ctx->dv.wait_polls = polls > kSpinLimit ? kSpinLimit : polls;
+    // the bound is a kernel argument: no captured step stands for it any more
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+    ctx->ngraphs = 0;
     return CHOCO_OK;
 }
 
@@ -772,6 +799,7 @@ const char* choco_strerror(int code)
     case CHOCO_ERR_MISALIGNED: return "pointer not 4-byte aligned";
     case CHOCO_ERR_UNSUPPORTED: return "unsupported configuration";
     case CHOCO_ERR_TOO_LARGE: return "size exceeds a documented limit";
+    case CHOCO_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out; the state arrays are invalid";
     default: return "unknown error";
     }
 }

@@ -39,13 +39,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
                  : "memory");
     return ok != 0;
 }
-// Wait for phase `parity` with a bound: after kSpinLimit polls the wait is recorded as timed
-// out; the copies in flight are then given a second bounded grace period so that the block
-// does not retire under them.  Returns false on a timeout.
-constexpr uint32_t kSpinLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, Stats* stats)
+// Wait for phase `parity` with a bound: after `polls` polls (Dev::wait_polls, kSpinLimit unless
+// a test lowered it) the wait is recorded as timed out; the copies in flight are then given a
+// second bounded grace period so that the block does not retire under them.  Returns false on
+// a timeout.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, Stats* stats, uint32_t polls)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     if ((threadIdx.x & 31) == 0) atomicAdd(&stats->timeouts, 1ull);
     for (uint32_t i = 0; i < kSpinLimit; ++i) {

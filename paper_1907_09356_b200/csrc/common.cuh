@@ -10,11 +10,13 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "internal.h"
+
 namespace choco {
 
 constexpr int kThreads = 256;            // threads per block of the streaming kernels
 constexpr int kQuad = 4;                 // coordinates per thread per iteration (one 128-bit access)
-constexpr int kChunk = kThreads * kQuad; // 2048 coordinates: one block iteration, one tree leaf group
+constexpr int kChunk = kThreads * kQuad; // 1024 coordinates: one block iteration, one tree leaf group
 constexpr int kDenseIters = 4;           // dense kernels: iterations per block
 constexpr int kSpan = kChunk * kDenseIters; // dense kernels: coordinates per block (4096)
 // sparse path (top-k, random-k): one block owns one tile of one row
@@ -156,22 +158,35 @@ __device__ __forceinline__ void allow_next_kernel()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// `hot` (optional, base == nullptr for none): a range this launch asks the L2 cache to keep
+// resident (a fraction `ratio` of it) while everything else it touches streams through.  A
+// per-launch attribute: nothing stays behind on the stream.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                     cudaStream_t st, Args... args)
+                                     cudaStream_t st, HotRange hot, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (hot.base && hot.bytes > 0 && hot.ratio > 0.f) {
+        attr[1].id = cudaLaunchAttributeAccessPolicyWindow;
+        attr[1].val.accessPolicyWindow.base_ptr = hot.base;
+        attr[1].val.accessPolicyWindow.num_bytes = hot.bytes;
+        attr[1].val.accessPolicyWindow.hitRatio = hot.ratio;
+        attr[1].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        attr[1].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
+
 
 __device__ __forceinline__ uint32_t abs_key(float v)
 {

@@ -14,6 +14,8 @@ constexpr uint32_t kRowRescue = 2u;   // candidates unusable: collect afresh wit
 constexpr uint32_t kRowRefine = 4u;   // the first digit's bin is too full: resolve the next 11 bits
 constexpr int64_t kRescueMinD = (int64_t)1 << 22; // rows this long are rescued rather than selected by one block
 
+constexpr uint32_t kSpinLimit = 1u << 22;   // polls a kernel spends on a wait before it gives up
+
 constexpr int64_t kEmitSmemBudget = 200 * 1024; // dynamic shared memory the emit kernel may use
 constexpr int kHistBins = 2048;       // first radix digit: top 11 bits of the ordering key
 
@@ -23,6 +25,13 @@ struct Stats {
     unsigned long long exact_rows;
     unsigned long long timeouts;   // bounded device waits that ran out
     unsigned long long rescued_rows; // rows whose candidates were collected afresh after a miss
+};
+
+// A range of device memory that a launch asks the L2 cache to keep resident.
+struct HotRange {
+    void* base;
+    size_t bytes;
+    float ratio;
 };
 
 // Everything the kernels need; passed by value.
@@ -81,6 +90,11 @@ struct Dev {
     int64_t emit_keys_cap;       // candidate keys cached in shared memory up to this many
     int64_t emit_smem_bytes;     // dynamic shared memory of the emit kernel
     Stats* stats;
+    uint32_t wait_polls;         // bound of the kernels' first wait for their staged copies
+    // what steps ask the L2 cache to keep resident (sparse Q): messages, range records, tables
+    void* hot_base;
+    int64_t hot_bytes;
+    float hot_ratio;
     // dense messages
     int64_t wpitch;              // sign-plane words per row (multiple of 4)
     uint32_t* msg_bits;          // [n, wpitch]
@@ -111,6 +125,8 @@ struct Dev {
     float* partial;              // [n, nchunks] per-1024 partial sums
     float* partial2;             // [n, nchunks] ping-pong for the tree
 };
+
+inline HotRange hot_range_of(const Dev& dv) { return {dv.hot_base, (size_t)dv.hot_bytes, dv.hot_ratio}; }
 
 struct StepArgs {
     float* X;
@@ -203,11 +219,8 @@ struct choco_ctx {
     // kernel, msg_last holds the message applied most recently (choco_get_message)
     struct DenseBuf { uint32_t* bits; float* scale; float* norms; uint8_t* levels; float* dense; } dbuf[2];
     int msg_cur, msg_last;
-    // arena that steps ask the L2 cache to keep resident (messages, records, candidates)
-    void* hot_base;
-    int64_t hot_bytes;
-    bool hot_set;
-    cudaStream_t hot_stream;
+    bool timed_out;              // a synchronising call saw device_timeouts != 0: steps refuse
+    bool hot_l2;                 // the context asked for persisting L2 lines (reset on destroy)
     // host staging for choco_sgd_step_host
     float* stage[4];
     // consensus scratch

@@ -139,6 +139,8 @@ int layers_step(choco_layers* L, float* X, float* Xhat, float* S, const float* G
                 float gamma, float lambda, float beta, void* stream)
 {
     if (!L || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
+    for (const choco_ctx* c : L->ctx)
+        if (c->timed_out) return CHOCO_ERR_TIMEOUT;
     cudaStream_t st = (cudaStream_t)stream;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     uint64_t mode = 0;

@@ -582,9 +582,9 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
         // thread 0 polls (bounded); the others wait at the barrier, then each thread observes
         // the completed phase itself so that the copied data is visible to it
         int ok = 1;
-        if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
+        if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats, dv.wait_polls) ? 1 : 0;
         if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
-        (void)mbar_wait_bounded(bar, 0, dv.stats);
+        (void)mbar_wait_bounded(bar, 0, dv.stats, kSpinLimit);
         for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
             const uint32_t kk = order_key<KIND>(sbits[p]);
             klo = kk < klo ? kk : klo;
@@ -779,7 +779,8 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int r
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev][a.vec ? 1 : 0] = true;
     }
-    e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st, dv, a,
+    e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st,
+                          hot_range_of(dv), dv, a,
                           fused ? 1 : 0, rescue);
     if (e != cudaSuccess) return e;
     *a.launches += 1;

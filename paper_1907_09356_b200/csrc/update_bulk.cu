@@ -210,9 +210,9 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
     // completed phase itself so that the copied tiles are visible to it
     int ok = 1;
-    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
+    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats, dv.wait_polls) ? 1 : 0;
     if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
-    if (!mbar_wait_bounded(bar, 0, dv.stats)) return;
+    if (!mbar_wait_bounded(bar, 0, dv.stats, kSpinLimit)) return;
 
     // x^ += q_i in place on the staged tile
     if (self_in_regs) {
@@ -349,7 +349,8 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
-    return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT, AL>, grid, dim3(NT), smem, st, dv, a);
+    return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT, AL>, grid, dim3(NT), smem, st,
+                             hot_range_of(dv), dv, a);
 }
 
 template <bool AL>

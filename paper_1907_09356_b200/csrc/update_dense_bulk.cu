@@ -179,9 +179,9 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
     // completed phase itself so that the copied tiles are visible to it
     int ok = 1;
-    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats) ? 1 : 0;
+    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats, dv.wait_polls) ? 1 : 0;
     if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
-    (void)mbar_wait_bounded(bar, 0, dv.stats);
+    (void)mbar_wait_bounded(bar, 0, dv.stats, kSpinLimit);
 
     float4 vn[NIT]; // x' - x^': the next step's argument of Q
 #pragma unroll

@@ -81,7 +81,7 @@ def test_mixing_matrix_checks(lib):
 
 def test_strerror(lib):
     assert lib.choco_strerror(0) == b"ok"
-    for code in range(-7, 0):
+    for code in range(-8, 0):
         assert lib.choco_strerror(code) not in (b"ok", b"unknown error")
     assert lib.choco_strerror(-99) == b"unknown error"
 

@@ -1,10 +1,14 @@
 """Parity at the full workload sizes, in the launch configuration bench.py times.
 
-The 8x8-torus d = 1e6 top-1 % step is compared whole; the ResNet-50-sized rows (d = 25.6 M,
-32 workers) are compared on sampled workers that the oracle computes one by one, plus
-properties that hold at any size (the S = W Xhat invariant on a coordinate sample, message
-structure).
+The 8x8-torus d = 1e6 top-1 % step is compared whole (its full 500-step run is compared in
+test_gpu_full_runs.py); the ResNet-50-sized rows (d = 25.6 M, 32 workers) are compared on a
+sampled worker that the oracle follows for several steps together with the workers its result
+depends on, plus properties that hold at any size (the S = W Xhat invariant on a coordinate
+sample, carried against uncarried compression).
 """
+import concurrent.futures
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -49,70 +53,122 @@ def test_config4_full_step():
     ch.close()
 
 
+CONE_STEPS = 4      # steps the sampled worker is followed for
+CONE_ROW = 17       # the sampled worker (its cone 13..21 does not wrap around the ring)
+
+
+def _segment_csr(m):
+    """Rows 0..m-1 of a ring segment: interior rows mix with both neighbours at 1/3 each, in
+    ascending column order (as the ring rows they stand for); the two end rows are never updated."""
+    rp, col, val = [0], [], []
+    for a in range(m):
+        if 0 < a < m - 1:
+            col += [a - 1, a, a + 1]; val += [1.0 / 3.0] * 3
+        else:
+            col.append(a); val.append(1.0)
+        rp.append(len(col))
+    return workloads.MixingCSR(m, np.asarray(rp, np.int32), np.asarray(col, np.int32), np.asarray(val, np.float32))
+
+
 @pytest.mark.parametrize("name", ["c5_ring32_qsgd", "c5_ring32_topk"])
-def test_config5_sampled_rows(name):
+def test_config5_sampled_row_over_several_steps(name):
+    """Worker 17 of the 32-ring after CONE_STEPS steps depends on workers 13..21 at the start.  The
+    oracle follows that shrinking cone (it updates 7, 5, 3, 1 rows and forms 9, 7, 5, 3 messages);
+    the library runs all 32 rows.  Every message the oracle forms and every row it updates is
+    compared bit for bit at every step, so steps 2.. check what the update kernel prepared for
+    them: carried top-k candidates selected by the emit kernel with its working arrays in global
+    memory, and the gsgd_b messages the update kernel wrote."""
     wl = workloads.WORKLOADS[name]
     w = wl.mixing()
-    n, d = wl.n, wl.d
-    free_b = torch.cuda.mem_get_info()[0]
-    if free_b < 16 * n * d + (4 << 30):
+    n, d, T, i0 = wl.n, wl.d, CONE_STEPS, CONE_ROW
+    if torch.cuda.mem_get_info()[0] < 24 * n * d + (4 << 30):
         pytest.skip("not enough free device memory for the 32 x 25.6M state")
-    sample = [0, 17]
-    need = sorted({int(c) for i in sample for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]]})
-    # device state generated on the device; the needed rows are copied to the host for the oracle
+    cone = list(range(i0 - T, i0 + T + 1))
+    m = len(cone)
+    for i in cone[1:-1]:    # the segment's column order is the ring's
+        assert [int(c) for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]]] == [i - 1, i, i + 1]
     gen = torch.Generator(device=DEV)
     gen.manual_seed(5)
     dX = torch.randn(n, d, device=DEV, generator=gen) * float(np.sqrt(wl.x_var))
     dXh = torch.randn(n, d, device=DEV, generator=gen) * 0.05
-    dG = torch.randn(n, d, device=DEV, generator=gen) * float(np.sqrt(wl.g_var))
-    # S must equal W Xhat: ring weights are 1/3
-    dS = (dXh + torch.roll(dXh, 1, 0) + torch.roll(dXh, -1, 0)) * (1.0 / 3.0)
-    hX = {j: dX[j].cpu().numpy() for j in need}
-    hXh = {j: dXh[j].cpu().numpy() for j in need}
-    hS = {j: dS[j].cpu().numpy() for j in sample}
-    hG = {j: dG[j].cpu().numpy() for j in sample}
-    ch = choco.Choco(w, d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=21)
-    ch.sgd_step(dX, dXh, dS, dG, wl.eta, wl.gamma)
-    torch.cuda.synchronize()
+    dGs = [torch.randn(n, d, device=DEV, generator=gen) * float(np.sqrt(wl.g_var)) for _ in range(2)]
+    dS = (dXh + torch.roll(dXh, 1, 0) + torch.roll(dXh, -1, 0)) * (1.0 / 3.0)   # S = W Xhat on the ring
+    X = np.stack([dX[j].cpu().numpy() for j in cone])
+    Xh = np.stack([dXh[j].cpu().numpy() for j in cone])
+    S = np.stack([dS[j].cpu().numpy() for j in cone])
+    Gs = [np.stack([g[j].cpu().numpy() for j in cone]) for g in dGs]
+    seg = _segment_csr(m)
     p = oracle.Params(wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=21)
-    msgs = {j: oracle.compress(p, oracle.difference(hX[j], hXh[j]), 0, j) for j in need}
-    for j in need:
+    ch = choco.Choco(w, d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=21)
+    try:
+        with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+            for t in range(T):
+                ch.sgd_step(dX, dXh, dS, dGs[t % 2], wl.eta, wl.gamma)
+                # the oracle: messages of the rows within distance T - t (keyed by the true worker
+                # number), then the rows within distance T - 1 - t
+                send = [a for a in range(m) if abs(cone[a] - i0) <= T - t]
+                upd = [a for a in range(m) if abs(cone[a] - i0) <= T - 1 - t]
+                msgs = dict(zip(send, ex.map(
+                    lambda a: oracle.compress(p, oracle.difference(X[a], Xh[a]), t, cone[a]), send)))
+                list(ex.map(lambda a: oracle._apply_row(a, seg, X, Xh, S, Gs[t % 2], msgs, wl.eta, wl.gamma), upd))
+                torch.cuda.synchronize()
+                for a in send:
+                    j, mm = cone[a], msgs[a]
+                    if wl.q == "topk":
+                        assert np.array_equal(choco.choco_read_message(ch.ctx, j, 0).view(np.uint32), mm.idx), (t, j)
+                        assert np.array_equal(choco.choco_read_message(ch.ctx, j, 1).view(np.uint32),
+                                              mm.val.view(np.uint32)), (t, j)
+                    else:
+                        assert np.array_equal(choco.choco_read_message(ch.ctx, j, 0).view(np.uint32), mm.bits), (t, j)
+                        assert np.array_equal(choco.choco_read_message(ch.ctx, j, 1).view(np.float32), mm.norms), (t, j)
+                        assert np.array_equal(choco.choco_read_message(ch.ctx, j, 2), mm.levels), (t, j)
+                for a in upd:
+                    j = cone[a]
+                    _exact(dXh[j].cpu().numpy(), Xh[a], f"Xhat row {j} after step {t}")
+                    _exact(dS[j].cpu().numpy(), S[a], f"S row {j} after step {t}")
+                    _exact(dX[j].cpu().numpy(), X[a], f"X row {j} after step {t}")
+        # property at any size: S = W Xhat still holds on a coordinate sample (float32 rounding)
+        cols = torch.randint(0, d, (4096,), device=DEV)
+        H = dXh[:, cols].double()
+        want = (H + torch.roll(H, 1, 0) + torch.roll(H, -1, 0)) / 3.0
+        assert float((dS[:, cols].double() - want).abs().max()) < 1e-5
+        st = choco.choco_get_stats(ch.ctx)
+        assert st["device_timeouts"] == 0 and st["exact_rows"] == 0, st
         if wl.q == "topk":
-            assert np.array_equal(choco.choco_read_message(ch.ctx, j, 0).view(np.uint32), msgs[j].idx)
-            assert np.array_equal(choco.choco_read_message(ch.ctx, j, 1).view(np.uint32),
-                                  msgs[j].val.view(np.uint32))
-        else:
-            assert np.array_equal(choco.choco_read_message(ch.ctx, j, 0).view(np.uint32), msgs[j].bits)
-            assert np.array_equal(choco.choco_read_message(ch.ctx, j, 1).view(np.float32), msgs[j].norms)
-            assert np.array_equal(choco.choco_read_message(ch.ctx, j, 2), msgs[j].levels)
-    pos = {j: a for a, j in enumerate(need)}
-    for i in sample:
-        # the oracle's row update on a sub-problem that holds only the needed workers
-        sub_X = np.stack([hX[j] for j in need])
-        sub_H = np.stack([hXh[j] for j in need])
-        sub_S = np.zeros_like(sub_X)
-        sub_S[pos[i]] = hS[i]
-        sub_G = np.zeros_like(sub_X)
-        sub_G[pos[i]] = hG[i]
-        rp = np.zeros(len(need) + 1, np.int32)
-        col, val = [], []
-        for a, j in enumerate(need):
-            if j == i:
-                for e in range(w.row_ptr[i], w.row_ptr[i + 1]):
-                    col.append(pos[int(w.col[e])]); val.append(float(w.val[e]))
-            else:
-                col.append(a); val.append(1.0)
-            rp[a + 1] = len(col)
-        sub_w = workloads.MixingCSR(len(need), rp, np.asarray(col, np.int32), np.asarray(val, np.float32))
-        sub_msgs = {pos[j]: msgs[j] for j in need}
-        oracle._apply_row(pos[i], sub_w, sub_X, sub_H, sub_S, sub_G, sub_msgs, wl.eta, wl.gamma)
-        _exact(dXh[i].cpu().numpy(), sub_H[pos[i]], f"Xhat row {i}")
-        _exact(dS[i].cpu().numpy(), sub_S[pos[i]], f"S row {i}")
-        _exact(dX[i].cpu().numpy(), sub_X[pos[i]], f"X row {i}")
-    # property at any size: S = W Xhat still holds on a coordinate sample (float32 rounding)
-    cols = torch.randint(0, d, (4096,), device=DEV)
-    H = dXh[:, cols].double()
-    want = (H + torch.roll(H, 1, 0) + torch.roll(H, -1, 0)) / 3.0
-    assert float((dS[:, cols].double() - want).abs().max()) < 1e-5
-    assert choco.choco_get_stats(ch.ctx)["exact_rows"] == 0
-    ch.close()
+            # steps 2.. ran on the candidates the update kernel had collected
+            assert st["prepared_rows"] + st["rescued_rows"] == n * (T - 1), st
+            assert st["prepared_rows"] >= n * (T - 1) - 8, st
+    finally:
+        ch.close()
+
+
+@pytest.mark.parametrize("name", ["c5_ring32_qsgd", "c5_ring32_topk"])
+def test_config5_carried_compression_changes_nothing(name):
+    """Five steps at full size with the compression carried from step to step (candidates and
+    messages prepared by the update kernel) and five with every step compressing afresh from X
+    and Xhat: the whole state must be identical."""
+    wl = workloads.WORKLOADS[name]
+    w = wl.mixing()
+    n, d, steps = wl.n, wl.d, 5
+    if torch.cuda.mem_get_info()[0] < 36 * n * d + (4 << 30):
+        pytest.skip("not enough free device memory for two copies of the 32 x 25.6M state")
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(6)
+    X0 = torch.randn(n, d, device=DEV, generator=gen) * float(np.sqrt(wl.x_var))
+    Gs = [torch.randn(n, d, device=DEV, generator=gen) * float(np.sqrt(wl.g_var)) for _ in range(2)]
+    out = []
+    for carry in (True, False):
+        ch = choco.Choco(w, d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=22)
+        choco.choco_set_carry(ch.ctx, carry)
+        st = [X0.clone(), torch.zeros_like(X0), torch.zeros_like(X0)]
+        for t in range(steps):
+            ch.sgd_step(st[0], st[1], st[2], Gs[t % 2], wl.eta, wl.gamma)
+        torch.cuda.synchronize()
+        stats = choco.choco_get_stats(ch.ctx)
+        assert stats["device_timeouts"] == 0
+        if wl.q == "topk":
+            assert (stats["prepared_rows"] > 0) == carry
+        out.append(st)
+        ch.close()
+    for a, b, what in zip(out[0], out[1], ("X", "Xhat", "S")):
+        assert torch.equal(a, b), what

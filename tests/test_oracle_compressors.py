@@ -55,6 +55,16 @@ def test_unit_interval_statistics():
     assert abs(float(np.corrcoef(u[:-1], u[1:])[0, 1])) < 0.01
 
 
+def test_words_to_unit_exact_values():
+    """u = (word >> 8) * 2^-24: the TOP 24 bits, so the low byte never matters and the
+    largest word stays below one.  (The low 24 bits, or a 23-bit shift, fail these.)"""
+    words = np.array([0, 0xFF, 0x100, 0x80000000, 0xFFFFFFFF, 0x00FFFFFF, 0x12345678], dtype=np.uint32)
+    want = [0.0, 0.0, 2.0 ** -24, 0.5, 1.0 - 2.0 ** -24, 0xFFFF * 2.0 ** -24, 0x123456 * 2.0 ** -24]
+    got = oracle.words_to_unit(words)
+    assert got.dtype == np.float32
+    assert [float(x) for x in got] == want
+
+
 def test_tree_sum_matches_hand_tree():
     a = np.array([1e8, 1.0, -1e8, 1.0, 3.0], dtype=np.float32)
     # ((a0+a1)+(a2+a3)) + a4 with float32 rounding at every node
@@ -231,6 +241,32 @@ def test_qsgd_zero_dither_is_floor_quantiser():
     mb = oracle.compress_qsgd(v, np.zeros(2, np.float32), s=16, bucket=0, biased=True)
     tau = 1 + min(2 / 256, np.sqrt(2) / 16)
     assert np.allclose(mb.q, m.q / tau, rtol=1e-6)
+
+
+# v = (1, -2, 2, 0, 0, 0, 0, 0, 0, 4): the squares sum to 25, so nu = 5 exactly.
+_HAND_V = np.array([1, -2, 2, 0, 0, 0, 0, 0, 0, 4], dtype=np.float32)
+
+
+@pytest.mark.parametrize("s,u,levels,packed", [
+    # s = 2, 1-bit fields: s|v|/nu = .4 .8 .8 0 ... 1.6 -> only the last reaches 1 (saturated)
+    (2, 0.0, [0, 0, 0, 0, 0, 0, 0, 0, 0, 1], [0b00000000, 0b10]),
+    # the same with u = 1/2: .9 1.3 1.3 .5 ... 2.1 -> 0 1 1 0 ... 1 (2 saturates to s - 1 = 1)
+    (2, 0.5, [0, 1, 1, 0, 0, 0, 0, 0, 0, 1], [0b00000110, 0b10]),
+    # s = 4, 2-bit fields: .8 1.6 1.6 0 ... 3.2 -> 0 1 1 0 ... 3; coordinate c at bits 2c, 2c+1
+    (4, 0.0, [0, 1, 1, 0, 0, 0, 0, 0, 0, 3], [0b00010100, 0, 0b1100]),
+    # s = 128, 8-bit fields: 25.6 51.2 51.2 0 ... 102.4 -> one byte per coordinate
+    (128, 0.0, [25, 51, 51, 0, 0, 0, 0, 0, 0, 102], [25, 51, 51, 0, 0, 0, 0, 0, 0, 102]),
+])
+def test_qsgd_level_fields_by_hand(s, u, levels, packed):
+    """Level fields of 1, 2 and 8 bits written out by hand (Appendix C: a level is an integer
+    in {0..s-1}; stored in the smallest of 1, 2, 4, 8 bits, coordinate c at bit c * width)."""
+    m = oracle.compress_qsgd(_HAND_V, np.full(10, u, np.float32), s=s, bucket=0, biased=False)
+    assert m.norms[0] == np.float32(5.0)
+    assert list(m.levels) == packed
+    assert list(m.bits) == [0b10]                       # only coordinate 1 is negative
+    want_q = np.array([5.0 / s * l for l in levels], dtype=np.float32)
+    want_q[1] = -want_q[1]
+    assert np.array_equal(m.q, want_q)
 
 
 def test_qsgd_tau_values():

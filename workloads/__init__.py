@@ -140,6 +140,35 @@ def k_of(a_num: int, a_den: int, d: int) -> int:
     return (d * a_num) // a_den
 
 
+FINGERPRINT_MODULUS = 65521
+
+
+def fingerprint(a: np.ndarray) -> tuple[int, int]:
+    """Two 64-bit check sums of a float32 array's bit patterns, taken in row-major order:
+    the sum of the 32-bit words, and the sum of word_i * (i mod 65521 + 1), both modulo 2^64.
+    Equal arrays give equal pairs; a changed, moved or swapped word changes them.  (A way to
+    compare a large state with a stored run without storing the state.)"""
+    words = np.ascontiguousarray(a, dtype=np.float32).reshape(-1).view(np.uint32).astype(np.uint64)
+    weight = (np.arange(words.size, dtype=np.uint64) % np.uint64(FINGERPRINT_MODULUS)) + np.uint64(1)
+    with np.errstate(over="ignore"):
+        return int(words.sum(dtype=np.uint64)), int((words * weight).sum(dtype=np.uint64))
+
+
+def gradient_pool(wl: "Workload", count: int, seed: int) -> list[np.ndarray]:
+    """`count` pre-generated gradient tensors [n, d] that a run cycles through (step t uses
+    tensor t mod count): g ~ N(mu_i, g_var) per coordinate, where mu_i is a per-worker offset
+    vector ~ N(0, g_mean_var) shared by all tensors of the pool (workers with different
+    objectives), or zero if the workload has no g_mean_var."""
+    mu = normal_rows(wl.n, wl.d, wl.g_mean_var, seed + 1_000_003) if wl.g_mean_var > 0 else None
+    pool = []
+    for p in range(count):
+        g = normal_rows(wl.n, wl.d, wl.g_var, seed + p)
+        if mu is not None:
+            g += mu
+        pool.append(g)
+    return pool
+
+
 def resnet20_layer_sizes() -> list[int]:
     """Lengths of the 65 parameter tensors of a CIFAR ResNet-20 in forward order (3x3
     convolutions without bias, each followed by a batch-norm scale and shift; 1x1 projection
@@ -217,6 +246,8 @@ class Workload:
     layers: str = ""      # "" = Q on the whole row; "resnet20" / "resnet50" = Q per layer
     a_num: int = 1        # per-layer top-k / random-k keep max(1, floor(a d_l)), a = a_num / a_den
     a_den: int = 1
+    momentum: float = 0.0      # > 0: Algorithm 2 with this momentum factor ...
+    weight_decay: float = 0.0  # ... and this weight decay
 
     def layer_sizes(self) -> list[int]:
         return {"resnet20": resnet20_layer_sizes, "resnet50": resnet50_layer_sizes}[self.layers]()
@@ -239,6 +270,9 @@ WORKLOADS = {
     # logistic regression d=2000 on a 16-ring: random-k 1 % and QSGD s=16 (whole-row norm)
     "c2_ring16_randk": Workload("c2_ring16_randk", 16, 2000, "ring", "randk",
                                 k=k_of(1, 100, 2000), eta=0.1, gamma=0.1, steps=2000, x_var=0.0),
+    # random-1 % at the consensus stepsize Table 4 lists for it (at 0.1 the run diverges)
+    "c2_ring16_randk_g006": Workload("c2_ring16_randk_g006", 16, 2000, "ring", "randk",
+                                     k=k_of(1, 100, 2000), eta=0.1, gamma=0.00625, steps=2000, x_var=0.0),
     "c2_ring16_qsgd": Workload("c2_ring16_qsgd", 16, 2000, "ring", "qsgd", s=16, bucket=0,
                                eta=0.1, gamma=0.1, steps=2000, x_var=0.0),
     # ResNet-20-sized flat vector, 8-ring, scaled sign
@@ -248,6 +282,18 @@ WORKLOADS = {
     "c4_torus64_topk": Workload("c4_torus64_topk", 64, 1_000_000, "torus8x8", "topk",
                                 k=k_of(1, 100, 1_000_000), eta=0.05, gamma=0.2, steps=500,
                                 x_var=1.0, g_var=1e-2),
+    # the same at a consensus stepsize in the stable range for top-1 % (Table 4 lists 0.0375 as
+    # the tuned value; with 0.2 the differences x - x^ grow over a run, with 0.04 they decay)
+    "c4_torus64_topk_g004": Workload("c4_torus64_topk_g004", 64, 1_000_000, "torus8x8", "topk",
+                                     k=k_of(1, 100, 1_000_000), eta=0.05, gamma=0.04, steps=500,
+                                     x_var=1.0, g_var=1e-2),
+    # Algorithm 2 (momentum 0.9, weight decay 1e-4) on the headline shape and on the 32-ring
+    "c4_torus64_topk_mom": Workload("c4_torus64_topk_mom", 64, 1_000_000, "torus8x8", "topk",
+                                    k=k_of(1, 100, 1_000_000), eta=0.05, gamma=0.04, steps=500,
+                                    x_var=1.0, g_var=1e-2, momentum=0.9, weight_decay=1e-4),
+    "c5_ring32_qsgd_mom": Workload("c5_ring32_qsgd_mom", 32, 25_557_032, "ring", "qsgd", s=16,
+                                   bucket=512, eta=0.1, gamma=0.1, steps=200, x_var=0.01,
+                                   g_var=1e-3, momentum=0.9, weight_decay=1e-4),
     # ResNet-50-sized flat vector, 32-ring: QSGD s=16 in 512-buckets, or top-0.1 %
     "c5_ring32_qsgd": Workload("c5_ring32_qsgd", 32, 25_557_032, "ring", "qsgd", s=16,
                                bucket=512, eta=0.1, gamma=0.1, steps=200, x_var=0.01,
@@ -319,14 +365,19 @@ class LogisticProblem:
         return rng.integers(0, self.per_worker, size=batch)
 
     def gradient(self, x: np.ndarray, step: int, batch: int = 32) -> np.ndarray:
+        """Mini-batch gradient of every worker at its x_i.  Written without a matrix product
+        and without numpy's vectorised exp (both pick a code path by CPU model, so their last
+        bits can differ between machines): products summed by numpy's fixed pairwise scheme,
+        the exponential one sample at a time through the C library."""
         g = np.empty((self.n, self.d), dtype=np.float32)
         for i in range(self.n):
             rows = self.minibatch(step, i, batch)
             a, y = self.a[i, rows], self.y[i, rows]
             xi = x[i].astype(np.float64)
-            margin = y * (a @ xi)
-            coef = -y / (1.0 + np.exp(margin))
-            g[i] = ((coef[:, None] * a).mean(axis=0) + self.lam * xi).astype(np.float32)
+            margin = y * np.sum(a * xi, axis=1)
+            # (a margin beyond the range of exp has a vanishing coefficient)
+            coef = np.array([-yy / (1.0 + math.exp(mm)) if mm < 700.0 else 0.0 for yy, mm in zip(y, margin)])
+            g[i] = ((coef[:, None] * a).sum(axis=0) / batch + self.lam * xi).astype(np.float32)
         return g
 
     def loss(self, xbar: np.ndarray) -> float:
