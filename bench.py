@@ -13,6 +13,7 @@ independent replicas, one per process, and reports their aggregate.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -30,14 +31,15 @@ import workloads  # noqa: E402
 L2_BYTES = 126 * 2 ** 20
 NOMINAL_HBM_GBS = 8000.0           # the figure the 60 % target is quoted against
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, from the ncu
-# captures summarised under profiles/ (None for workloads that were not captured).  The
-# 32-ring QSGD figure is the 8-ring capture of the same kernel scaled by the coordinates per
-# launch (29.70 B per coordinate), as the capture of the full-size workload would be too large.
-NCU_TRAFFIC = {("c4_torus64_topk", "update"): 1.367e9,
-               ("p_ring8_qsgd", "update"): 1.993e9,
-               ("p_ring8_sign", "update"): 1.856e9,
-               ("c5_ring32_qsgd", "update"): 29.70 * 32 * 25_557_032}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, QUOTED from the
+# ncu captures summarised under profiles/ (this run does not measure it; None for workloads that
+# were not captured, or whose kernel changed since).  The 32-ring QSGD figure is the 8-ring
+# capture of the same kernel scaled by the coordinates per launch, as the capture of the
+# full-size workload would be too large.
+NCU_TRAFFIC = {
+    "c4_torus64_topk": (1.367e9, "profiles/update_and_emit_kernels_c4_torus64_topk.md"),
+    "p_ring8_sign": (1.856e9, "profiles/update_dense_bulk_kernel_p_ring8_sign.md"),
+}
 
 
 def measured_peak():
@@ -90,7 +92,10 @@ def message_bytes(wl) -> int:
 
 def step_min_bytes(wl, w, sgd=True) -> int:
     """Whole step: X, Xhat, S (and G) read once, every densely changing array written once,
-    messages written once and read once per off-diagonal neighbour, sparse updates at 4 B."""
+    messages written once and read once per off-diagonal neighbour, sparse updates at 4 B;
+    Algorithm 2 reads and writes the momentum memory as well (8 B per coordinate)."""
+    if wl.momentum > 0:
+        return step_min_bytes(dataclasses.replace(wl, momentum=0.0), w, sgd) + 8 * wl.n * wl.d
     N = wl.n * wl.d
     nnz = int(w.row_ptr[-1])
     deg_off = nnz - wl.n
@@ -105,7 +110,10 @@ def step_min_bytes(wl, w, sgd=True) -> int:
 
 def update_kernel_bytes(wl, w, sgd=True) -> int:
     """The update kernel alone: reads X, Xhat, S, G and every neighbour's message (self
-    included), writes X densely and Xhat, S where touched (all of them for dense Q)."""
+    included), writes X densely and Xhat, S where touched (all of them for dense Q); with
+    momentum (Algorithm 2) M is read and written too."""
+    if wl.momentum > 0:
+        return update_kernel_bytes(dataclasses.replace(wl, momentum=0.0), w, sgd) + 8 * wl.n * wl.d
     N = wl.n * wl.d
     nnz = int(w.row_ptr[-1])
     msg = message_bytes(wl)
@@ -165,7 +173,12 @@ class ClockSampler:
 
 
 def oracle_sample(wl, w, budget_rows=None):
-    """Run one oracle step on (a row sample of) the workload; returns (coords, seconds, text)."""
+    """Time the oracle, as it stands and on one thread, on a row sample of the workload, and
+    build the time of a WHOLE step from it: a step forms n messages and updates n rows, so
+    step seconds = n * (seconds per message + seconds per row update), both measured here
+    (the sample updates `rows` rows and has to form the messages of all their neighbours, which
+    are more; each cost is divided by its own count).  Returns (seconds per whole step, seconds
+    spent, text)."""
     import oracle
     rows = list(range(wl.n)) if budget_rows is None else list(range(min(budget_rows, wl.n)))
     need = sorted({int(c) for i in rows for c in w.col[w.row_ptr[i]:w.row_ptr[i + 1]]})
@@ -173,6 +186,7 @@ def oracle_sample(wl, w, budget_rows=None):
     X = workloads.normal_rows(len(need), wl.d, wl.x_var or 1.0, 11)
     Xh, S = np.zeros_like(X), np.zeros_like(X)
     G = workloads.normal_rows(len(need), wl.d, wl.g_var or 1e-2, 12)
+    M = np.zeros_like(X) if wl.momentum > 0 else None
     # a sub-problem holding only the needed rows, W's rows restricted accordingly
     rp, col, val = [0], [], []
     for j in need:
@@ -185,22 +199,41 @@ def oracle_sample(wl, w, budget_rows=None):
     sub = workloads.MixingCSR(len(need), np.asarray(rp, np.int32), np.asarray(col, np.int32),
                               np.asarray(val, np.float32))
     p = oracle.Params(wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=1)
-    t0 = time.perf_counter()
-    if wl.layers:
-        oracle.step_layers(sub, p, workloads.layer_offsets(wl.layer_sizes()), wl.a_num, wl.a_den, X, Xh, S, G,
-                           wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
-    else:
-        oracle.step(sub, p, X, Xh, S, G, wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows])
-    dt = time.perf_counter() - t0
-    text = (f"one oracle step for {len(rows)} of {wl.n} workers of {wl.name} "
-            f"(their {len(need)} neighbours' messages formed too), single thread")
-    return len(rows) * wl.d, dt, text
+    # a stop-watch around the oracle's compression call: everything else a step does is the row update
+    spent = {"compress": 0.0}
+    plain_compress = oracle.compress
+
+    def timed_compress(*a, **kw):
+        t = time.perf_counter()
+        out = plain_compress(*a, **kw)
+        spent["compress"] += time.perf_counter() - t
+        return out
+
+    oracle.compress = timed_compress
+    try:
+        t0 = time.perf_counter()
+        if wl.layers:
+            oracle.step_layers(sub, p, workloads.layer_offsets(wl.layer_sizes()), wl.a_num, wl.a_den, X, Xh, S, G,
+                               wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows], M=M, lam=wl.weight_decay,
+                               beta=wl.momentum)
+        else:
+            oracle.step(sub, p, X, Xh, S, G, wl.eta, wl.gamma, 0, rows=[remap[i] for i in rows], M=M,
+                        lam=wl.weight_decay, beta=wl.momentum)
+        dt = time.perf_counter() - t0
+    finally:
+        oracle.compress = plain_compress
+    per_msg = spent["compress"] / len(need)
+    per_row = (dt - spent["compress"]) / len(rows)
+    text = (f"whole step of {wl.name} built from measured costs: n * (per message + per row update), "
+            f"{per_msg:.4f} s per message over {len(need)} messages and {per_row:.4f} s per row update over "
+            f"{len(rows)} of {wl.n} rows, oracle as it stands, single thread")
+    return wl.n * (per_msg + per_row), dt, text
 
 
-def rows_for_budget(wl) -> int:
-    # about 10-30 s of single-thread work: ~0.15 s per million coordinates compressed + applied
+def rows_for_budget(wl, seconds=20.0) -> int:
+    # ~0.15 s per million coordinates compressed + applied; a sparse Q sorts the row (3x)
     per_row = 0.25 * wl.d / 1e6 * (3 if wl.q in ("topk", "randk") else 1)
-    return max(1, min(wl.n, int(20.0 / max(per_row, 1e-3))))
+    return max(1, min(wl.n, int(seconds / max(per_row, 1e-3))))
 
 
 # ------------------------------------------------------------------------------------------
@@ -229,11 +262,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-stride", type=int, default=8,
-                    help="time the update kernel with CUDA events on every Nth timed step")
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps steps each; the median is reported")
+    ap.add_argument("--kernel-launches", type=int, default=32,
+                    help="launches of the update kernel timed one by one after the timed regions")
     ap.add_argument("--pool", type=int, default=8, help="gradient tensors cycled through (>= 2)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.repeats = max(args.repeats, 1)
+    args.kernel_launches = max(args.kernel_launches, 16)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -248,26 +284,27 @@ def main():
               "parallelism": "replicas only" if args.gpus > 1 else "single GPU",
               "l2": "inputs per step exceed L2" if 20 * N > 2 * L2_BYTES else "state fits L2 (no flush)"}
 
+    host_cores = os.cpu_count()
     if args.impl == "reference":
         if rank != 0:
             return
-        times = []
-        coords = 0
-        text = ""
-        rows = rows_for_budget(wl)
-        rows = max(1, rows // max(1, args.steps + args.warmup))
+        # every timed step is a whole step of the stated workload, its time built from a bounded
+        # sample (see oracle_sample); the whole run is sized to about two minutes
+        rows = rows_for_budget(wl, 120.0 / (args.steps + args.warmup))
+        step_s, text = [], ""
         for i in range(args.warmup + args.steps):
-            coords, dt, text = oracle_sample(wl, w, rows)
+            sec, _, text = oracle_sample(wl, w, rows)
             if i >= args.warmup:
-                times.append(dt)
-        val = coords * len(times) / sum(times)
+                step_s.append(sec)
+        mean_s = sum(step_s) / len(step_s)
+        val = N / mean_s
         print(json.dumps({
             "impl": "reference", "metric": "coords_per_sec", "value": val, "unit": "coords/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": 1e3 * mean_s, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-            "cpu_baseline": {"value": val, "unit": "coords/s", "cores": 1, "kind": "oracle",
-                             "sample": text},
+            "cpu_baseline": {"value": val, "unit": "coords/s", "cores": 1, "host_cores": host_cores,
+                             "kind": "oracle", "sample": text},
             "e2e": {"value": val, "unit": "coords/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         }))
         return
@@ -301,6 +338,8 @@ def main():
         args.warmup = max(args.warmup, 4 * pool_n + 2)
     pool = [torch.randn(wl.n, wl.d, device=dev, generator=gen) * float(np.sqrt(wl.g_var or 1e-2))
             for _ in range(pool_n)]
+    mom = wl.momentum > 0
+    M = torch.zeros_like(X) if mom else None
     if wl.layers:
         off = workloads.layer_offsets(wl.layer_sizes())
         lay = choco.choco_layers_init(wl.n, off, wl.d, w.row_ptr, w.col, w.val, wl.q, wl.a_num, wl.a_den,
@@ -308,13 +347,20 @@ def main():
         ctxs = [choco.choco_layers_get_layer(lay, l)[0] for l in range(len(off) - 1)]
 
         def do_step(G):
-            choco.choco_layers_sgd_step(lay, X, Xh, S, G, wl.eta, wl.gamma)
+            if mom:
+                choco.choco_layers_sgd_momentum_step(lay, X, Xh, S, G, M, wl.eta, wl.gamma, wl.weight_decay,
+                                                     wl.momentum)
+            else:
+                choco.choco_layers_sgd_step(lay, X, Xh, S, G, wl.eta, wl.gamma)
     else:
         ch = choco.Choco(w, wl.d, wl.q, k=wl.k, s=wl.s or 16, bucket=wl.bucket, seed=7)
         ctxs = [ch.ctx]
 
         def do_step(G):
-            ch.sgd_step(X, Xh, S, G, wl.eta, wl.gamma)
+            if mom:
+                ch.sgd_momentum_step(X, Xh, S, G, M, wl.eta, wl.gamma, wl.weight_decay, wl.momentum)
+            else:
+                ch.sgd_step(X, Xh, S, G, wl.eta, wl.gamma)
 
     def stats_sum():
         tot = {}
@@ -333,26 +379,39 @@ def main():
         do_step(pool[t % pool_n])
     barrier()
     st0 = stats_sum()
-    if not wl.layers and not small:
-        choco.choco_profile_enable(ch.ctx, args.steps)
-        choco.choco_profile_set_stride(ch.ctx, args.profile_stride)   # events between kernels cost time
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    # the timed region, EXACTLY --steps steps between a barrier + synchronize on both sides, taken
+    # --repeats times back to back; the line reports the median repeat (and the fastest beside it)
     t_wall0 = time.time()
-    e0.record()
-    for t in range(args.steps):
-        do_step(pool[(args.warmup + t) % pool_n])
-    e1.record()
+    step_no = args.warmup
+    rep_ms = []
+    for _ in range(args.repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for t in range(args.steps):
+            do_step(pool[step_no % pool_n])
+            step_no += 1
+        e1.record()
+        barrier()
+        rep_ms.append(e0.elapsed_time(e1))
+    st1 = stats_sum()
+    # the dominant kernel by itself: CUDA events around the update kernel on the step's stream, on
+    # every one of a few further steps (outside the timed region: events between a step's kernels
+    # keep them from overlapping and would slow the steps down)
+    nrec, upd_ms = 0, 0.0
+    if not wl.layers and not small:
+        choco.choco_profile_enable(ch.ctx, args.kernel_launches)
+        for t in range(args.kernel_launches):
+            do_step(pool[step_no % pool_n])
+            step_no += 1
+        nrec, upd_ms = choco.choco_profile_read(ch.ctx)
     barrier()
     t_wall1 = time.time()
-    ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    st1 = stats_sum()
-    nrec, upd_ms = (0, 0.0) if (wl.layers or small) else choco.choco_profile_read(ch.ctx)
     finite = bool(torch.isfinite(X).all())
 
     # end to end: host buffers in, host buffers out, through choco_sgd_step_host
@@ -360,16 +419,18 @@ def main():
     if args.e2e_steps > 0:
         hX, hXh, hS = (t.cpu().pin_memory() for t in (X, Xh, S))
         hG = pool[0].cpu().pin_memory()
-        if wl.layers:
-            # the layered calls take device arrays: copy in from pinned memory, step, copy out
+        hM = M.cpu().pin_memory() if mom else None
+        if wl.layers or mom:
+            # these calls take device arrays: copy in from pinned memory, step, copy out
             def host_step():
-                for dst, src in ((X, hX), (Xh, hXh), (S, hS), (pool[0], hG)):
+                for dst, src in ((X, hX), (Xh, hXh), (S, hS), (pool[0], hG)) + (((M, hM),) if mom else ()):
                     dst.copy_(src, non_blocking=True)
+                for c in ctxs:
+                    choco.choco_invalidate(c)      # the arrays were overwritten behind the library's back
                 do_step(pool[0])
-                for dst, src in ((hX, X), (hXh, Xh), (hS, S)):
+                for dst, src in ((hX, X), (hXh, Xh), (hS, S)) + (((hM, M),) if mom else ()):
                     dst.copy_(src, non_blocking=True)
                 torch.cuda.synchronize()
-            choco.choco_layers_invalidate(lay)
         else:
             def host_step():
                 choco.choco_sgd_step_host(ch.ctx, hX, hXh, hS, hG, wl.eta, wl.gamma)
@@ -383,12 +444,14 @@ def main():
         e2e = {"seconds": e2e_s, "steps": args.e2e_steps}
 
     if world > 1:
-        ms, e2e_s = max_over_ranks([ms, e2e["seconds"] if e2e else 0.0], dev)
+        got = max_over_ranks(rep_ms + [e2e["seconds"] if e2e else 0.0], dev)
+        rep_ms = got[:-1]
         if e2e:
-            e2e["seconds"] = e2e_s
+            e2e["seconds"] = got[-1]
 
     if rank == 0:
         peak, peak_src = measured_peak()
+        ms = sorted(rep_ms)[len(rep_ms) // 2]           # the median repeat
         ms_step = ms / args.steps
         value = whole_job_rate(world, N, args.steps, ms * 1e-3)
         upd_bytes = update_kernel_bytes(wl, w)
@@ -398,17 +461,21 @@ def main():
         step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
         roof_kernel = "update (apply) kernel"
         if wl.layers or small:
-            # one small set of kernels per layer, or a few short kernels replayed from a graph
-            # (events between them would prevent that): no single dominant launch to time, so
-            # the roofline entry is the whole step against its minimum bytes
+            # a few short kernels replayed from a graph (events between them would prevent that):
+            # no single dominant launch to time, so the roofline entry is the whole step against
+            # its minimum bytes
             roof_kernel = ("whole step: the kernels of all layers" if wl.layers
                            else "whole step (state fits L2; replayed from a CUDA graph)")
             achieved, upd_bytes, upd_avg_s, nrec = step_gbs, step_bytes, ms_step * 1e-3, args.steps
+        traffic, traffic_src = NCU_TRAFFIC.get(wl.name, (None, None))
         out = {
             "metric": "coords_per_sec", "value": value, "unit": "coords/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config,
+            "repeats": {"count": len(rep_ms), "ms_per_step": [m / args.steps for m in rep_ms],
+                        "median_ms_per_step": ms_step, "min_ms_per_step": min(rep_ms) / args.steps,
+                        "reported": "median"},
             "steps_per_sec": 1e3 / ms_step,
             "compressed_bytes_per_step": message_bytes(wl) * wl.n,
             "step_min_bytes": step_bytes, "step_hbm_gbs": step_gbs,
@@ -417,12 +484,14 @@ def main():
             "roofline": {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None,
-                         "traffic": NCU_TRAFFIC.get((wl.name, "update")),
+                         "traffic": traffic,
+                         "traffic_source": (f"quoted from the ncu capture in {traffic_src}, not measured by this run"
+                                            if traffic_src else None),
                          "algorithmic_bytes_per_launch": upd_bytes,
-                         "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec,
-                         "timed_every": args.profile_stride},
+                         "avg_launch_ms": upd_avg_s * 1e3, "launches_timed": nrec},
             "gpu_launches": int(st1["kernel_launches"] - st0["kernel_launches"]),
-            "selection": {k: int(st1[k] - st0[k]) for k in ("prepared_rows", "recompressed_rows", "exact_rows")},
+            "selection": {k: int(st1[k] - st0[k]) for k in ("prepared_rows", "recompressed_rows", "exact_rows",
+                                                          "rescued_rows")},
             "finite": finite,
             "clocks": clocks,
         }
@@ -431,14 +500,15 @@ def main():
         else:
             out["graph_replays"] = int(st1["graph_replays"] - st0["graph_replays"])
         if e2e:
+            arrays_in, arrays_out = (5, 4) if mom else (4, 3)
             out["e2e"] = {"value": whole_job_rate(world, N, e2e["steps"], e2e["seconds"]), "unit": "coords/s",
-                          "h2d_bytes_per_step": 16 * N, "d2h_bytes_per_step": 12 * N,
+                          "h2d_bytes_per_step": 4 * arrays_in * N, "d2h_bytes_per_step": 4 * arrays_out * N,
                           "steps": e2e["steps"],
-                          "api": ("pinned host buffers copied in and out around choco_layers_sgd_step" if wl.layers
-                                  else "choco_sgd_step_host, pinned host buffers")}
+                          "api": ("pinned host buffers copied in and out around the device-pointer step call"
+                                  if (wl.layers or mom) else "choco_sgd_step_host, pinned host buffers")}
         if not args.no_cpu_baseline and world == 1:
-            coords, dt, text = oracle_sample(wl, w, rows_for_budget(wl))
-            out["cpu_baseline"] = {"value": coords / dt, "unit": "coords/s", "cores": 1,
+            step_s, dt, text = oracle_sample(wl, w, rows_for_budget(wl))
+            out["cpu_baseline"] = {"value": N / step_s, "unit": "coords/s", "cores": 1, "host_cores": host_cores,
                                    "kind": "oracle", "sample": text, "seconds": dt}
         print(json.dumps(out))
     if wl.layers:

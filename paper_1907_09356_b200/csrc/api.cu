@@ -343,6 +343,10 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
     dv.wait_polls = kSpinLimit;
+    for (uint32_t r = 0; r < 10; ++r) {
+        dv.round_key[r][0] = (uint32_t)seed + r * 0x9E3779B9u;
+        dv.round_key[r][1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
+    }
     dv.ntiles = (d + kTile - 1) / kTile;
     dv.nspans = (d + kSpan - 1) / kSpan;
     dv.nchunks = (d + kChunk - 1) / kChunk;

@@ -56,6 +56,7 @@ struct Dev {
     uint4* rec;                  // [n, ntiles, maxdeg]
     // generator
     uint64_t seed;
+    uint32_t round_key[10][2];   // Philox4x32-10 key schedule of `seed`: key + r * (0x9E3779B9, 0xBB67AE85)
     // sparse messages: idx / val [n, kpitch], tile_ptr [n, ntiles + 1]
     int64_t k;
     int64_t kpitch;

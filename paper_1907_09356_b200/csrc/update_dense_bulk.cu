@@ -1,9 +1,28 @@
-// Update kernel for scaled sign and bucketed gsgd_b, bulk-copy variant (rows 16-byte
-// aligned, d a multiple of 4): the same arithmetic as update_dense_kernel (Algorithm 1:
-// public copies, gossip step, gradient step) followed by the compression of x' - x^' for the next step, with the x, x^, s, g
-// (and momentum) tiles of 2048 coordinates staged in shared memory by asynchronous bulk
-// copies.  The neighbours' packed message pieces that a thread needs are small; they are
-// fetched into registers while the copies are in flight.
+// Update kernel for scaled sign and bucketed gsgd_b (rows 16-byte aligned, d a multiple of 4):
+// Algorithm 1's update of the public copies, gossip step and gradient step (Algorithm 2 with
+// momentum) for one tile of 2048 coordinates of one worker per block,
+//     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
+//     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i),
+// followed (EMIT) by the compression of x' - x^' (Appendix C) into the other message buffer,
+// so that the next step's messages cost no further pass over X and Xhat.
+//
+// Everything a block touches moves through shared memory by asynchronous bulk copies: the x, x^,
+// s, g (and momentum) tiles and, for every neighbour, the 2048-coordinate slice of its packed
+// message (sign plane, level fields) are fetched with one mbarrier to wait on; the results are
+// written back over the staged tiles and leave by bulk stores, as do the sign plane and the level
+// fields of the next message.  No thread holds a global address or a loaded value across a wait.
+//
+// The per-coordinate work is kept to what the definition needs:
+//   * a neighbour's contribution w_ij q_j takes only s distinct magnitudes per block of the norm,
+//     fl(w fl(mag l)) for l = 0..s-1; they are tabulated once per tile (s <= 16) and a
+//     coordinate's decode is a table read plus its sign bit -- the same products, the same bits;
+//   * the quotient fl(fl(s |v|) / nu) of the quantiser is formed as the product with 1 / nu in
+//     float64, rounded once to float32: for float32 operands that is the correctly rounded
+//     quotient (the float64 product is within 2^-52 of a / nu, no quotient of two float32 numbers
+//     lies within 2^-49 of the midpoint of two float32 numbers, and none is such a midpoint);
+//   * floor(r + u), saturated at s - 1, is taken by clamping at s - 1/2 and adding 2^23 rounded
+//     down, which leaves the integer in the low bits of the sum;
+//   * the round keys of the generator depend on the seed only and come as kernel arguments.
 #include "bulk.cuh"
 
 namespace choco {
@@ -11,9 +30,10 @@ namespace choco {
 namespace {
 
 constexpr int NT = 256;
-constexpr int NIT = 2;                  // quads per thread
+constexpr int NIT = 2;                   // quads per thread
 constexpr int kDTile = NT * kQuad * NIT; // 2048 coordinates per block
-constexpr int kPre = 4;                 // neighbours whose pieces are fetched ahead
+constexpr int kBatch = 16;               // neighbours whose message slices are staged at a time
+constexpr int kTabLevels = 16;           // level magnitudes are tabulated for s <= 16
 
 struct Upd {
     float eta, gamma, lambda, beta;
@@ -33,38 +53,29 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
     return __fadd_rn(xn, __fmul_rn(u.gamma, cons));
 }
 
-// The pieces of worker j's message that cover coordinates [c, c+4): the quad's four sign
-// bits and (gsgd_b) its packed level fields.  The magnitude that goes with them -- the row's
-// scale, or norm / (tau s) of the block -- is the same for many quads and is kept apart.
-struct Piece {
-    uint32_t nib;    // bit e: coordinate c + e is negative
-    uint32_t packed; // level fields, wbits each (gsgd_b)
-};
-
-template <int KIND>
-__device__ __forceinline__ Piece load_piece(const Dev& dv, int j, int64_t c)
+// shared memory -> global; both addresses 16-byte aligned, bytes % 16 == 0
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes)
 {
-    Piece p;
-    p.nib = __ldg(dv.msg_bits + (int64_t)j * dv.wpitch + (c >> 5));
-    p.packed = 0u;
-    if (KIND == CHOCO_Q_QSGD) {
-        const uint8_t* lrow = dv.msg_levels + (int64_t)j * dv.lpitch;
-        const uint32_t width = (uint32_t)dv.wbits;
-        if (width == 8) p.packed = __ldg(reinterpret_cast<const uint32_t*>(lrow + c));
-        else if (width == 4) p.packed = __ldg(reinterpret_cast<const uint16_t*>(lrow + (c >> 1)));
-        else if (width == 2) p.packed = __ldg(lrow + (c >> 2));
-        else p.packed = (__ldg(lrow + (c >> 3)) >> (c & 7)) & 0xFu;
-    }
-    return p;
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_commit_and_drain()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    // the staged tiles may be released once the copy engine has read them
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// order this thread's shared-memory accesses before what the copy engine does next
+__device__ __forceinline__ void fence_before_bulk_copy()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// magnitude shared by the coordinates of one block of worker j's message
-template <int KIND>
-__device__ __forceinline__ float load_mag(const Dev& dv, int j, int64_t bucket)
+// mag is >= 0, so setting the sign bit negates it; bit e of nib is coordinate e's sign
+__device__ __forceinline__ float with_sign(float mag, uint32_t nib, int e)
 {
-    if (KIND == CHOCO_Q_SIGN) return __ldg(dv.msg_scale + j);
-    const float nu = __ldg(dv.msg_norms + (int64_t)j * dv.npitch + bucket);
-    return __fdiv_rn(nu, __fmul_rn(bucket == dv.tail_bucket ? dv.tau_tail : dv.tau_full, (float)dv.s));
+    return __uint_as_float(__float_as_uint(mag) | ((nib << (31 - e)) & 0x80000000u));
 }
 
 // small non-negative integer -> float without the conversion unit: exact below 2^23
@@ -73,130 +84,218 @@ __device__ __forceinline__ float small_uint_to_float(uint32_t v)
     return __fsub_rn(__uint_as_float(0x4B000000u | v), 8388608.f);
 }
 
-// mag is >= 0, so setting the sign bit negates it
-__device__ __forceinline__ float with_sign(float mag, uint32_t nib, int e)
+// Philox4x32-10 with the round keys precomputed (Dev::round_key): the same words as philox4x32_10.
+__device__ __forceinline__ uint4 philox_with_round_keys(uint4 ctr, const Dev& dv)
 {
-    return __uint_as_float(__float_as_uint(mag) | ((nib << (31 - e)) & 0x80000000u));
-}
-
-template <int KIND>
-__device__ __forceinline__ float4 decode_piece(const Dev& dv, const Piece& pp, float mag, int64_t c)
-{
-    Piece p = pp; p.nib = (pp.nib >> (c & 31)) & 0xFu;
-    float m[4];
-    if (KIND == CHOCO_Q_SIGN) {
-        m[0] = m[1] = m[2] = m[3] = mag;
-    } else {
-        const uint32_t width = (uint32_t)dv.wbits, mask = (1u << width) - 1u;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) m[e] = __fmul_rn(mag, small_uint_to_float((p.packed >> (e * width)) & mask));
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * ctr.x;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * ctr.z;
+        ctr = make_uint4((uint32_t)(p1 >> 32) ^ ctr.y ^ dv.round_key[r][0], (uint32_t)p1,
+                         (uint32_t)(p0 >> 32) ^ ctr.w ^ dv.round_key[r][1], (uint32_t)p0);
     }
-    return make_float4(with_sign(m[0], p.nib, 0), with_sign(m[1], p.nib, 1), with_sign(m[2], p.nib, 2),
-                       with_sign(m[3], p.nib, 3));
+    return ctr;
 }
 
-__device__ __forceinline__ uint32_t sign_nibble4(const float4& v)
-{
-    return (uint32_t)(v.x < 0.f) | ((uint32_t)(v.y < 0.f) << 1) | ((uint32_t)(v.z < 0.f) << 2) |
-           ((uint32_t)(v.w < 0.f) << 3);
-}
+// Shared-memory layout, in bytes from the (128-byte aligned) base.  WBITS == 0: scaled sign.
+template <int WBITS, bool HAS_G, bool HAS_M>
+struct Layout {
+    static constexpr int kArrays = 3 + (HAS_G ? 1 : 0) + (HAS_M ? 1 : 0);
+    static constexpr int kBitsTile = kDTile / 8;               // 256 bytes of sign plane
+    static constexpr int kLevTile = kDTile * WBITS / 8;        // level fields of a tile
+    static constexpr int kMsgTile = kBitsTile + kLevTile;      // one neighbour's slice
+    static constexpr bool kTable = WBITS >= 1 && WBITS <= 4;   // s <= 16: magnitudes tabulated
+    __host__ __device__ static constexpr int msg_in() { return kArrays * kDTile * 4; }
+    __host__ __device__ static int msg_out(int nb) { return msg_in() + nb * kMsgTile; }
+    __host__ __device__ static int tables(int nb) { return msg_out(nb) + kMsgTile; }
+    // per neighbour and block of the norm: 16 weighted magnitudes (or, without a table, one
+    // magnitude and the weight); then the worker's own unweighted magnitudes
+    __host__ __device__ static int table_floats(int nb, int nbk) { return (nb + 1) * nbk * kTabLevels; }
+    __host__ __device__ static int misc(int nb, int nbk) { return tables(nb) + table_floats(nb, nbk) * 4; }
+    // misc: warp sums [NIT][8] floats, per-block reciprocal norms [16] doubles, the barrier
+    __host__ __device__ static int total(int nb, int nbk) { return misc(nb, nbk) + NIT * 8 * 4 + 16 * 8 + 16; }
+};
 
-template <bool HAS_G, bool HAS_M>
-__host__ __device__ constexpr int n_arrays() { return 3 + (HAS_G ? 1 : 0) + (HAS_M ? 1 : 0); }
-
-template <int KIND, bool HAS_G, bool HAS_M, bool EMIT>
-__global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a)
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT>
+__global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
 {
+    using L = Layout<WBITS, HAS_G, HAS_M>;
+    static_assert((KIND == CHOCO_Q_SIGN) == (WBITS == 0), "sign has no level fields");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* hs = xs + kDTile;
     float* ss = hs + kDTile;
     float* gs = ss + kDTile;                     // used when HAS_G
     float* ms = gs + (HAS_G ? kDTile : 0);       // used when HAS_M
-    float* ws = ms + (HAS_M ? kDTile : 0);       // [NIT][8] warp sums
-    uint64_t* bar = reinterpret_cast<uint64_t*>(ws + NIT * 8);
+    unsigned char* msg_in = smem_raw + L::msg_in();
+    unsigned char* msg_out = smem_raw + L::msg_out(nb_stage);
+    // blocks of the norm per tile (gsgd_b); one "block" for sign
+    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
+    float* tab = reinterpret_cast<float*>(smem_raw + L::tables(nb_stage));
+    float* tab_self = tab + nb_stage * nbk * kTabLevels;
+    float* ws = reinterpret_cast<float*>(smem_raw + L::misc(nb_stage, nbk)); // [NIT][8] warp sums
+    double* rnu = reinterpret_cast<double*>(ws + NIT * 8);                   // [16] 1 / nu per block of the norm
+    uint64_t* bar = reinterpret_cast<uint64_t*>(rnu + 16);
 
     const int row = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kDTile;
     const int nvalid = (int)((dv.d - c0) < kDTile ? (dv.d - c0) : kDTile); // multiple of 4
-    const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
+    const int e0 = dv.row_ptr[row], deg = dv.row_ptr[row + 1] - e0;
     const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
     float* xr = a.X + (int64_t)row * dv.ld + c0;
     float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
     float* sr = a.S + (int64_t)row * dv.ld + c0;
     float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
+    // sizes of the slices actually present in this tile, rounded up to whole 16-byte units (the
+    // message rows are padded so that the rounded slice of the last tile stays inside the row)
+    const uint32_t dense_bytes = (uint32_t)nvalid * sizeof(float);
+    const uint32_t bits_bytes = ((((uint32_t)nvalid + 31u) >> 5) * 4u + 15u) & ~15u;
+    const uint32_t lev_bytes = (((uint32_t)nvalid * WBITS + 7u) / 8u + 15u) & ~15u;
+    const uint32_t msg_bytes = bits_bytes + (WBITS > 0 ? lev_bytes : 0u);
+    const int64_t bits_off = (int64_t)blockIdx.x * (kDTile / 32);            // words into a row's sign plane
+    const int64_t lev_off = (int64_t)blockIdx.x * L::kLevTile;               // bytes into a row's level fields
 
-    if (threadIdx.x == 0) {
-        mbar_init(bar, 1);
-        const uint32_t bytes = (uint32_t)nvalid * sizeof(float);
-        mbar_expect_tx(bar, bytes * n_arrays<HAS_G, HAS_M>());
-        bulk_load(xs, xr, bytes, bar);
-        bulk_load(hs, hr, bytes, bar);
-        bulk_load(ss, sr, bytes, bar);
-        if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, bytes, bar);
-        if (HAS_M) bulk_load(ms, mrow, bytes, bar);
-    }
-    // message pieces of the first kPre neighbours, fetched while the tiles are in flight
-    Piece pre[NIT][kPre];
-    int prej[kPre];
-    float prew[kPre], pmag[kPre];
-#pragma unroll
-    for (int q = 0; q < kPre; ++q) {
-        prej[q] = -1;
-        prew[q] = 0.f;
-        pmag[q] = 0.f;
-        if (e0 + q < e1) {
-            prej[q] = dv.col[e0 + q];
-            prew[q] = dv.wval[e0 + q];
-            if (KIND == CHOCO_Q_SIGN) pmag[q] = load_mag<KIND>(dv, prej[q], 0);
+    // stage the message slices of neighbours [first, first + count): lane r of warp 0 issues r's copies
+    auto stage_messages = [&](int first, int count) {
+        if (lane < count) {
+            const int j = dv.col[e0 + first + lane];
+            unsigned char* dst = msg_in + lane * L::kMsgTile;
+            bulk_load(dst, dv.msg_bits + (int64_t)j * dv.wpitch + bits_off, bits_bytes, bar);
+            if (WBITS > 0) bulk_load(dst + L::kBitsTile, dv.msg_levels + (int64_t)j * dv.lpitch + lev_off, lev_bytes, bar);
         }
-    }
-#pragma unroll
-    for (int it = 0; it < NIT; ++it) {
-        const int li = (it * NT + threadIdx.x) * kQuad;
-#pragma unroll
-        for (int q = 0; q < kPre; ++q) {
-            pre[it][q].nib = 0u; pre[it][q].packed = 0u;
-            if (prej[q] >= 0 && li < nvalid) pre[it][q] = load_piece<KIND>(dv, prej[q], c0 + li);
+    };
+    if (warp == 0) {
+        const int count = deg < nb_stage ? deg : nb_stage;
+        if (lane == 0) {
+            mbar_init(bar, 1);
+            mbar_expect_tx(bar, dense_bytes * L::kArrays + (uint32_t)count * msg_bytes);
+            bulk_load(xs, xr, dense_bytes, bar);
+            bulk_load(hs, hr, dense_bytes, bar);
+            bulk_load(ss, sr, dense_bytes, bar);
+            if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, dense_bytes, bar);
+            if (HAS_M) bulk_load(ms, mrow, dense_bytes, bar);
         }
+        __syncwarp();
+        stage_messages(0, count);
     }
-    // gsgd_b: the 128 coordinates of a warp's quads lie in one block, so lane q fetches the
-    // norm of neighbour q's block and the warp shares norm / (tau s) by shuffles later
-    float nraw[NIT];
-    bool ntail[NIT];
-#pragma unroll
-    for (int it = 0; it < NIT; ++it) {
-        nraw[it] = 0.f;
-        ntail[it] = false;
-        if (KIND == CHOCO_Q_QSGD) {
-            const int64_t bucket = (c0 + (int64_t)(it * NT + warp * 32) * kQuad) >> dv.bucket_shift;
-            ntail[it] = bucket == dv.tail_bucket;
-            if (lane < kPre && e0 + lane < e1 && bucket < dv.nbuckets)
-                nraw[it] = __ldg(dv.msg_norms + (int64_t)dv.col[e0 + lane] * dv.npitch + bucket);
-        }
-    }
-    // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
-    // completed phase itself so that the copied tiles are visible to it
-    int ok = 1;
-    if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats, dv.wait_polls) ? 1 : 0;
-    if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
-    (void)mbar_wait_bounded(bar, 0, dv.stats, kSpinLimit);
 
+    float acc[NIT][4], qs[NIT][4];
+#pragma unroll
+    for (int it = 0; it < NIT; ++it)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { acc[it][e] = 0.f; qs[it][e] = 0.f; }
+
+    for (int first = 0; first < deg; first += nb_stage) {
+        const int count = (deg - first) < nb_stage ? (deg - first) : nb_stage;
+        if (first > 0) {
+            // every thread is done with the previous batch's slices and tables
+            fence_before_bulk_copy();
+            __syncthreads();
+            if (warp == 0) {
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)count * msg_bytes);
+                __syncwarp();
+                stage_messages(first, count);
+            }
+        }
+        // magnitudes of this batch's neighbours, while the copies fly
+        int self_r = -1;
+        for (int r = 0; r < count; ++r)
+            if (dv.col[e0 + first + r] == row) self_r = r;
+        if (KIND == CHOCO_Q_SIGN) {
+            if ((int)threadIdx.x < count) {
+                const int j = dv.col[e0 + first + threadIdx.x];
+                const float sc = __ldg(dv.msg_scale + j);
+                tab[threadIdx.x] = __fmul_rn(dv.wval[e0 + first + threadIdx.x], sc);
+                if ((int)threadIdx.x == self_r) tab_self[0] = sc;
+            }
+        } else {
+            constexpr int per = L::kTable ? kTabLevels : 2;
+            for (int t = threadIdx.x; t < count * nbk * per; t += NT) {
+                const int l = t % per, b = (t / per) % nbk, r = t / (per * nbk);
+                const int64_t gb = (c0 >> dv.bucket_shift) + b;
+                float mag = 0.f;
+                const float w = dv.wval[e0 + first + r];
+                if (gb < dv.nbuckets) {
+                    const float nu = __ldg(dv.msg_norms + (int64_t)dv.col[e0 + first + r] * dv.npitch + gb);
+                    mag = __fdiv_rn(nu, __fmul_rn(gb == dv.tail_bucket ? dv.tau_tail : dv.tau_full, (float)dv.s));
+                }
+                if (L::kTable) {
+                    const float m = __fmul_rn(mag, (float)l);
+                    tab[(r * nbk + b) * kTabLevels + l] = __fmul_rn(w, m);
+                    if (r == self_r) tab_self[b * kTabLevels + l] = m;
+                } else {
+                    tab[(r * nbk + b) * kTabLevels + l] = l == 0 ? mag : w;
+                }
+            }
+        }
+        // thread 0 polls (bounded); the others wait at the barrier, then each thread observes the
+        // completed phase itself so that the copied data is visible to it
+        const uint32_t parity = (uint32_t)((first / nb_stage) & 1);
+        int ok = 1;
+        if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, parity, dv.stats, dv.wait_polls) ? 1 : 0;
+        if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
+        (void)mbar_wait_bounded(bar, parity, dv.stats, kSpinLimit);
+
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int q4 = it * NT + threadIdx.x;
+            const int li = q4 * kQuad;
+            const int b = KIND == CHOCO_Q_QSGD ? (li >> dv.bucket_shift) : 0; // the same for the whole warp
+            for (int r = 0; r < count; ++r) {
+                const unsigned char* slice = msg_in + r * L::kMsgTile;
+                const uint32_t word = reinterpret_cast<const uint32_t*>(slice)[li >> 5];
+                const uint32_t nib = (word >> (li & 31)) & 0xFu;
+                float q[4];
+                if (KIND == CHOCO_Q_SIGN) {
+                    const float m = tab[r];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) q[e] = with_sign(m, nib, e);
+                    if (r == self_r) {
+                        const float sc = tab_self[0];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(sc, nib, e);
+                    }
+                } else {
+                    const unsigned char* lev = slice + L::kBitsTile;
+                    uint32_t packed;
+                    if (WBITS == 8) packed = reinterpret_cast<const uint32_t*>(lev)[q4];
+                    else if (WBITS == 4) packed = reinterpret_cast<const uint16_t*>(lev)[q4];
+                    else if (WBITS == 2) packed = lev[q4];
+                    else packed = (uint32_t)(lev[q4 >> 1] >> (li & 4));
+                    constexpr uint32_t mask = (1u << (WBITS > 0 ? WBITS : 1)) - 1u;
+                    const float* t = tab + (r * nbk + b) * kTabLevels;
+                    if (L::kTable) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) q[e] = with_sign(t[(packed >> (e * WBITS)) & mask], nib, e);
+                        if (r == self_r) {
+                            const float* ts = tab_self + b * kTabLevels;
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(ts[(packed >> (e * WBITS)) & mask], nib, e);
+                        }
+                    } else {
+                        const float mag = t[0], w = t[1];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float m = __fmul_rn(mag, small_uint_to_float((packed >> (e * WBITS)) & mask));
+                            if (r == self_r) qs[it][e] = with_sign(m, nib, e);
+                            q[e] = with_sign(__fmul_rn(w, m), nib, e);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[it][e] = __fadd_rn(acc[it][e], q[e]);
+            }
+        }
+    }
+
+    // the update itself, written back over the staged tiles
     float4 vn[NIT]; // x' - x^': the next step's argument of Q
 #pragma unroll
     for (int it = 0; it < NIT; ++it) {
         const int q4 = it * NT + threadIdx.x;
         const int li = q4 * kQuad;
-        const int64_t c = c0 + li;
         vn[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-        float lane_mag = 0.f; // lane q: norm / (tau s) of neighbour q's block
-        if (KIND == CHOCO_Q_QSGD)
-            lane_mag = __fdiv_rn(nraw[it], __fmul_rn(ntail[it] ? dv.tau_tail : dv.tau_full, (float)dv.s));
-        float qmag[kPre];
-#pragma unroll
-        for (int q = 0; q < kPre; ++q)
-            qmag[q] = KIND == CHOCO_Q_SIGN ? pmag[q] : __shfl_sync(0xffffffffu, lane_mag, q);
         if (li < nvalid) {
             const float4 x = reinterpret_cast<const float4*>(xs)[q4];
             const float4 h = reinterpret_cast<const float4*>(hs)[q4];
@@ -204,41 +303,19 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f), m = g;
             if (HAS_G) g = reinterpret_cast<const float4*>(gs)[q4];
             if (HAS_M) m = reinterpret_cast<const float4*>(ms)[q4];
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), qs = acc;
-#pragma unroll
-            for (int q = 0; q < kPre; ++q) {
-                if (prej[q] < 0) continue;
-                const float4 qv = decode_piece<KIND>(dv, pre[it][q], qmag[q], c);
-                acc.x = __fadd_rn(acc.x, __fmul_rn(prew[q], qv.x));
-                acc.y = __fadd_rn(acc.y, __fmul_rn(prew[q], qv.y));
-                acc.z = __fadd_rn(acc.z, __fmul_rn(prew[q], qv.z));
-                acc.w = __fadd_rn(acc.w, __fmul_rn(prew[q], qv.w));
-                if (prej[q] == row) qs = qv;
-            }
-            for (int e = e0 + kPre; e < e1; ++e) { // rows with more neighbours: fetched on the spot
-                const int j = dv.col[e];
-                const float w = dv.wval[e];
-                const Piece p = load_piece<KIND>(dv, j, c);
-                const float4 qv = decode_piece<KIND>(dv, p, load_mag<KIND>(dv, j, c >> dv.bucket_shift), c);
-                acc.x = __fadd_rn(acc.x, __fmul_rn(w, qv.x));
-                acc.y = __fadd_rn(acc.y, __fmul_rn(w, qv.y));
-                acc.z = __fadd_rn(acc.z, __fmul_rn(w, qv.z));
-                acc.w = __fadd_rn(acc.w, __fmul_rn(w, qv.w));
-                if (j == row) qs = qv;
-            }
-            const float4 hn = make_float4(__fadd_rn(h.x, qs.x), __fadd_rn(h.y, qs.y),
-                                          __fadd_rn(h.z, qs.z), __fadd_rn(h.w, qs.w));
-            const float4 sn = make_float4(__fadd_rn(s.x, acc.x), __fadd_rn(s.y, acc.y),
-                                          __fadd_rn(s.z, acc.z), __fadd_rn(s.w, acc.w));
+            const float4 hn = make_float4(__fadd_rn(h.x, qs[it][0]), __fadd_rn(h.y, qs[it][1]),
+                                          __fadd_rn(h.z, qs[it][2]), __fadd_rn(h.w, qs[it][3]));
+            const float4 sn = make_float4(__fadd_rn(s.x, acc[it][0]), __fadd_rn(s.y, acc[it][1]),
+                                          __fadd_rn(s.z, acc[it][2]), __fadd_rn(s.w, acc[it][3]));
             float4 xn;
             xn.x = next_x<HAS_G, HAS_M>(x.x, sn.x, hn.x, g.x, m.x, u);
             xn.y = next_x<HAS_G, HAS_M>(x.y, sn.y, hn.y, g.y, m.y, u);
             xn.z = next_x<HAS_G, HAS_M>(x.z, sn.z, hn.z, g.z, m.z, u);
             xn.w = next_x<HAS_G, HAS_M>(x.w, sn.w, hn.w, g.w, m.w, u);
-            *reinterpret_cast<float4*>(hr + li) = hn;
-            *reinterpret_cast<float4*>(sr + li) = sn;
-            *reinterpret_cast<float4*>(xr + li) = xn;
-            if (HAS_M) *reinterpret_cast<float4*>(mrow + li) = m;
+            reinterpret_cast<float4*>(hs)[q4] = hn;
+            reinterpret_cast<float4*>(ss)[q4] = sn;
+            reinterpret_cast<float4*>(xs)[q4] = xn;
+            if (HAS_M) reinterpret_cast<float4*>(ms)[q4] = m;
             if (EMIT)
                 vn[it] = make_float4(__fsub_rn(xn.x, hn.x), __fsub_rn(xn.y, hn.y), __fsub_rn(xn.z, hn.z),
                                      __fsub_rn(xn.w, hn.w));
@@ -247,100 +324,144 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
             const float4 v = vn[it];
             float t;
             if (KIND == CHOCO_Q_SIGN) t = quad_tree(fabsf(v.x), fabsf(v.y), fabsf(v.z), fabsf(v.w));
-            else t = quad_tree(__fmul_rn(v.x, v.x), __fmul_rn(v.y, v.y), __fmul_rn(v.z, v.z),
-                               __fmul_rn(v.w, v.w));
+            else t = quad_tree(__fmul_rn(v.x, v.x), __fmul_rn(v.y, v.y), __fmul_rn(v.z, v.z), __fmul_rn(v.w, v.w));
             t = warp_tree(t);
             if (lane == 0) ws[it * 8 + warp] = t;
-            const uint32_t word = gather_sign_word(sign_nibble4(v), lane);
-            if ((lane & 7) == 0 && li < nvalid) dv.nxt_bits[(int64_t)row * dv.wpitch + (c >> 5)] = word;
+            // sign plane of the next message: this quad's four bits and its neighbour's make a byte
+            const uint32_t nib = (uint32_t)(v.x < 0.f) | ((uint32_t)(v.y < 0.f) << 1) | ((uint32_t)(v.z < 0.f) << 2) |
+                                 ((uint32_t)(v.w < 0.f) << 3);
+            const uint32_t other = __shfl_xor_sync(0xffffffffu, nib, 1);
+            if ((lane & 1) == 0) msg_out[q4 >> 1] = (unsigned char)(nib | (other << 4));
         }
     }
-    if (!EMIT) return;
+    fence_before_bulk_copy();
     __syncthreads();
+    const bool storer = threadIdx.x == 0;
+    if (storer) {
+        bulk_store(xr, xs, dense_bytes);
+        bulk_store(hr, hs, dense_bytes);
+        bulk_store(sr, ss, dense_bytes);
+        if (HAS_M) bulk_store(mrow, ms, dense_bytes);
+        if (EMIT) bulk_store(dv.nxt_bits + (int64_t)row * dv.wpitch + bits_off, msg_out, bits_bytes);
+    }
+    if (!EMIT) {
+        if (storer) bulk_store_commit_and_drain();
+        return;
+    }
     if (KIND == CHOCO_Q_SIGN) {
         // per-1024 partial sums of |v|; a small kernel finishes the tree and the scale
         if (threadIdx.x < NIT) {
             const int64_t chunk = (int64_t)blockIdx.x * NIT + threadIdx.x;
             if (chunk < dv.nchunks) dv.partial[(int64_t)row * dv.nchunks + chunk] = tree8(ws + threadIdx.x * 8);
         }
+        if (storer) bulk_store_commit_and_drain();
         return;
     }
-    // gsgd_b with blocks of dv.bucket (128..1024) coordinates: norms, dithered levels, packing
-    const float sf = (float)dv.s;
-    const int G = dv.bucket >> 7; // warps per block of coordinates: 1, 2, 4 or 8
-#pragma unroll
-    for (int it = 0; it < NIT; ++it) {
-        const int li = (it * NT + threadIdx.x) * kQuad;
-        const int64_t c = c0 + li;
-        const float* wsi = ws + it * 8;
-        const int w0 = warp & ~(G - 1);
+    // gsgd_b with blocks of dv.bucket (128..1024) coordinates: one thread per block of the norm
+    // finishes its tree over the warp sums, stores the norm and leaves 1 / nu for the others
+    const int G = dv.bucket >> 7; // warps per block of the norm: 1, 2, 4 or 8
+    if ((int)threadIdx.x < nbk) {
+        const int per_it = 8 / G;
+        const float* wsi = ws + ((int)threadIdx.x / per_it) * 8 + ((int)threadIdx.x % per_it) * G;
         float sq;
-        if (G == 1) sq = wsi[w0];
-        else if (G == 2) sq = __fadd_rn(wsi[w0], wsi[w0 + 1]);
-        else if (G == 4) sq = __fadd_rn(__fadd_rn(wsi[w0], wsi[w0 + 1]), __fadd_rn(wsi[w0 + 2], wsi[w0 + 3]));
+        if (G == 1) sq = wsi[0];
+        else if (G == 2) sq = __fadd_rn(wsi[0], wsi[1]);
+        else if (G == 4) sq = __fadd_rn(__fadd_rn(wsi[0], wsi[1]), __fadd_rn(wsi[2], wsi[3]));
         else sq = tree8(wsi);
         const float nu = __fsqrt_rn(sq);
-        const int64_t bucket = c >> dv.bucket_shift;
-        if (lane == 0 && warp == w0 && bucket < dv.nbuckets)
-            dv.nxt_norms[(int64_t)row * dv.npitch + bucket] = nu;
+        const int64_t gb = (c0 >> dv.bucket_shift) + threadIdx.x;
+        if (gb < dv.nbuckets) dv.nxt_norms[(int64_t)row * dv.npitch + gb] = nu;
+        rnu[threadIdx.x] = nu != 0.f ? 1.0 / (double)nu : 0.0; // nu = 0: every level is 0
+    }
+    __syncthreads();
+    const float sf = (float)dv.s, top = __fsub_rn((float)dv.s, 0.5f);
+    unsigned char* lev_out = msg_out + L::kBitsTile;
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int q4 = it * NT + threadIdx.x;
+        const int li = q4 * kQuad;
+        const double y = rnu[li >> dv.bucket_shift];
         // the dither of the message that the NEXT step applies
-        const uint4 rw = coord_words(dv.seed, step_of(a) + 1, (uint32_t)row, kStreamDither, c);
+        const uint64_t step = step_of(a) + 1;
+        const uint4 rw = philox_with_round_keys(
+            make_uint4((uint32_t)((c0 + li) >> 2), (uint32_t)row, (uint32_t)step,
+                       ((uint32_t)(step >> 32) << 8) | kStreamDither), dv);
         const float uu[4] = {word_to_unit(rw.x), word_to_unit(rw.y), word_to_unit(rw.z), word_to_unit(rw.w)};
         const float vv[4] = {vn[it].x, vn[it].y, vn[it].z, vn[it].w};
-        uint32_t lev[4] = {0u, 0u, 0u, 0u};
-        if (nu != 0.f) { // the same for every lane of the warp
+        uint32_t lv[4]; // 2^23 + level, as float bits
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float r = __fdiv_rn(__fmul_rn(sf, fabsf(vv[e])), nu);
-                const int l = __float2int_rz(__fadd_rn(r, uu[e])); // r + u >= 0: truncation is the floor
-                lev[e] = (uint32_t)(l > dv.s - 1 ? dv.s - 1 : l);
-            }
+        for (int e = 0; e < 4; ++e) {
+            const float r = (float)((double)__fmul_rn(sf, fabsf(vv[e])) * y); // = fl(fl(s |v|) / nu)
+            const float t = fminf(__fadd_rn(r, uu[e]), top);  // floor(min(t, s - 1/2)) = min(floor t, s - 1)
+            lv[e] = __float_as_uint(__fadd_rd(t, 8388608.f));
         }
-        uint8_t* lrow = dv.nxt_levels + (int64_t)row * dv.lpitch;
-        const bool in = li < nvalid;
-        if (dv.wbits == 8) {
-            if (in) *reinterpret_cast<uint32_t*>(lrow + c) = lev[0] | (lev[1] << 8) | (lev[2] << 16) | (lev[3] << 24);
-        } else if (dv.wbits == 4) {
-            if (in) *reinterpret_cast<uint16_t*>(lrow + (c >> 1)) =
-                        (uint16_t)(lev[0] | (lev[1] << 4) | (lev[2] << 8) | (lev[3] << 12));
-        } else if (dv.wbits == 2) {
-            if (in) lrow[c >> 2] = (uint8_t)(lev[0] | (lev[1] << 2) | (lev[2] << 4) | (lev[3] << 6));
+        constexpr uint32_t kMagic = 0x4B000000u;
+        if (WBITS == 8) {
+            reinterpret_cast<uint32_t*>(lev_out)[q4] =
+                (((lv[3] * 256u + lv[2]) * 256u + lv[1]) * 256u + lv[0]) - kMagic * 0x01010101u;
+        } else if (WBITS == 4) {
+            reinterpret_cast<uint16_t*>(lev_out)[q4] =
+                (uint16_t)((((lv[3] * 16u + lv[2]) * 16u + lv[1]) * 16u + lv[0]) - kMagic * 0x1111u);
+        } else if (WBITS == 2) {
+            lev_out[q4] = (unsigned char)((((lv[3] * 4u + lv[2]) * 4u + lv[1]) * 4u + lv[0]) - kMagic * 0x55u);
         } else {
-            const uint32_t lw = gather_sign_word(lev[0] | (lev[1] << 1) | (lev[2] << 2) | (lev[3] << 3), lane);
-            if ((lane & 7) == 0 && in) *reinterpret_cast<uint32_t*>(lrow + (c >> 3)) = lw;
+            const uint32_t four = ((((lv[3] * 2u + lv[2]) * 2u + lv[1]) * 2u + lv[0]) - kMagic * 0xFu) & 0xFu;
+            const uint32_t other = __shfl_xor_sync(0xffffffffu, four, 1);
+            if ((lane & 1) == 0) lev_out[q4 >> 1] = (unsigned char)(four | (other << 4));
         }
+    }
+    fence_before_bulk_copy();
+    __syncthreads();
+    if (storer) {
+        bulk_store(dv.nxt_levels + (int64_t)row * dv.lpitch + lev_off, lev_out, lev_bytes);
+        bulk_store_commit_and_drain();
     }
 }
 
-template <int KIND, bool HAS_G, bool HAS_M, bool EMIT>
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT>
 cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    constexpr size_t smem = (size_t)n_arrays<HAS_G, HAS_M>() * kDTile * sizeof(float) +
-                            NIT * 8 * sizeof(float) + 16;
-    static bool configured[64] = {};
+    using L = Layout<WBITS, HAS_G, HAS_M>;
+    const int nb_stage = dv.maxdeg < kBatch ? dv.maxdeg : kBatch;
+    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
+    const size_t smem = (size_t)L::total(nb_stage, nbk);
+    auto kern = update_dense_bulk_kernel<KIND, WBITS, HAS_G, HAS_M, EMIT>;
+    // Once per device, instantiation and size: allow the dynamic shared memory and ask for the
+    // largest shared-memory carve-out, so that as many tiles as possible are in flight per SM.
+    static size_t configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        auto kern = update_dense_bulk_kernel<KIND, HAS_G, HAS_M, EMIT>;
+    if (dev < 0 || dev >= 64 || configured[dev] < smem) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                     cudaSharedmemCarveoutMaxShared);
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
+        if (dev >= 0 && dev < 64) configured[dev] = smem;
     }
     const dim3 grid((unsigned)((dv.d + kDTile - 1) / kDTile), (unsigned)dv.n);
-    update_dense_bulk_kernel<KIND, HAS_G, HAS_M, EMIT><<<grid, NT, smem, st>>>(dv, a);
+    kern<<<grid, NT, smem, st>>>(dv, a, nb_stage);
     return cudaGetLastError();
 }
 
-template <int KIND, bool EMIT>
+template <int KIND, int WBITS, bool EMIT>
 cudaError_t launch_terms(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    if (a.M) return launch_one<KIND, true, true, EMIT>(dv, a, st);
-    if (a.G) return launch_one<KIND, true, false, EMIT>(dv, a, st);
-    return launch_one<KIND, false, false, EMIT>(dv, a, st);
+    if (a.M) return launch_one<KIND, WBITS, true, true, EMIT>(dv, a, st);
+    if (a.G) return launch_one<KIND, WBITS, true, false, EMIT>(dv, a, st);
+    return launch_one<KIND, WBITS, false, false, EMIT>(dv, a, st);
+}
+
+template <bool EMIT>
+cudaError_t launch_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    if (dv.kind == CHOCO_Q_SIGN) return launch_terms<CHOCO_Q_SIGN, 0, EMIT>(dv, a, st);
+    switch (dv.wbits) {
+    case 1: return launch_terms<CHOCO_Q_QSGD, 1, EMIT>(dv, a, st);
+    case 2: return launch_terms<CHOCO_Q_QSGD, 2, EMIT>(dv, a, st);
+    case 4: return launch_terms<CHOCO_Q_QSGD, 4, EMIT>(dv, a, st);
+    default: return launch_terms<CHOCO_Q_QSGD, 8, EMIT>(dv, a, st);
+    }
 }
 
 } // namespace
@@ -353,9 +474,7 @@ bool update_dense_bulk_usable(const Dev& dv, const StepArgs& a)
 
 cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {
-    if (dv.kind == CHOCO_Q_SIGN)
-        return emit ? launch_terms<CHOCO_Q_SIGN, true>(dv, a, st) : launch_terms<CHOCO_Q_SIGN, false>(dv, a, st);
-    return emit ? launch_terms<CHOCO_Q_QSGD, true>(dv, a, st) : launch_terms<CHOCO_Q_QSGD, false>(dv, a, st);
+    return emit ? launch_kind<true>(dv, a, st) : launch_kind<false>(dv, a, st);
 }
 
 } // namespace choco
