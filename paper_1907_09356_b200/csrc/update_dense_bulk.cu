@@ -1,5 +1,4 @@
-// Update kernel for scaled sign and bucketed gsgd_b (rows 16-byte aligned, d a multiple of 4):
-// Algorithm 1's update of the public copies, gossip step and gradient step (Algorithm 2 with
+// Update kernel for scaled sign and bucketed gsgd_b: Algorithm 1's update of the public copies, gossip step and gradient step (Algorithm 2 with
 // momentum) for one tile of 2048 coordinates of one worker per block,
 //     x^_i += q_i ;  s_i += sum_j w_ij q_j  (CSR column order, from +0) ;
 //     x_i  = (x_i - eta g_i) + gamma (s_i - x^_i),
@@ -11,6 +10,12 @@
 // message (sign plane, level fields) are fetched with one mbarrier to wait on; the results are
 // written back over the staged tiles and leave by bulk stores, as do the sign plane and the level
 // fields of the next message.  No thread holds a global address or a loaded value across a wait.
+// A bulk copy needs 16-byte aligned addresses and sizes.  With AL (rows 16-byte aligned, d a
+// multiple of 4) a tile is copied as it is and leaves the same way; otherwise each copy in starts
+// at the 16-byte boundary at or below the tile's first element and ends at the one at or above
+// its last, the tile is read from shared memory at the resulting offset of 0..3 elements, and the
+// results are stored from registers (a bulk store would overwrite the neighbours of a tile that
+// starts or ends inside a 16-byte unit).  The message planes are library-owned and always aligned.
 //
 // The per-coordinate work is kept to what the definition needs:
 //   * a neighbour's contribution w_ij q_j takes only s distinct magnitudes per block of the norm,
@@ -105,7 +110,8 @@ struct Layout {
     static constexpr int kLevTile = kDTile * WBITS / 8;        // level fields of a tile
     static constexpr int kMsgTile = kBitsTile + kLevTile;      // one neighbour's slice
     static constexpr bool kTable = WBITS >= 1 && WBITS <= 4;   // s <= 16: magnitudes tabulated
-    __host__ __device__ static constexpr int msg_in() { return kArrays * kDTile * 4; }
+    static constexpr int kStage = kDTile + 4;                  // floats per staged tile (slack: it may start mid-unit)
+    __host__ __device__ static constexpr int msg_in() { return kArrays * kStage * 4; }
     __host__ __device__ static int msg_out(int nb) { return msg_in() + nb * kMsgTile; }
     __host__ __device__ static int tables(int nb) { return msg_out(nb) + kMsgTile; }
     // per neighbour and block of the norm: 16 weighted magnitudes (or, without a table, one
@@ -116,17 +122,42 @@ struct Layout {
     __host__ __device__ static int total(int nb, int nbk) { return misc(nb, nbk) + NIT * 8 * 4 + 16 * 8 + 16; }
 };
 
-template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT>
+// element offset of p inside its 16-byte unit
+__device__ __forceinline__ uint32_t unit_shift(const float* p) { return (uint32_t)(((uintptr_t)p & 15u) >> 2); }
+
+// four consecutive floats of a staged tile that starts `sh` elements into its buffer
+template <bool AL>
+__device__ __forceinline__ float4 staged_quad(const float* buf, uint32_t sh, int q4)
+{
+    if (AL) return reinterpret_cast<const float4*>(buf)[q4];
+    const float* p = buf + sh + q4 * kQuad;
+    if ((sh & 1u) == 0u) { // 8-byte aligned: two 64-bit reads
+        const float2 lo = *reinterpret_cast<const float2*>(p), hi = *reinterpret_cast<const float2*>(p + 2);
+        return make_float4(lo.x, lo.y, hi.x, hi.y);
+    }
+    return make_float4(p[0], p[1], p[2], p[3]);
+}
+
+// store the first `left` (1..4) elements of v at p (4-byte aligned)
+__device__ __forceinline__ void store_some(float* p, const float4& v, int left)
+{
+    p[0] = v.x;
+    if (left > 1) p[1] = v.y;
+    if (left > 2) p[2] = v.z;
+    if (left > 3) p[3] = v.w;
+}
+
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
 {
     using L = Layout<WBITS, HAS_G, HAS_M>;
     static_assert((KIND == CHOCO_Q_SIGN) == (WBITS == 0), "sign has no level fields");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* xs = reinterpret_cast<float*>(smem_raw);
-    float* hs = xs + kDTile;
-    float* ss = hs + kDTile;
-    float* gs = ss + kDTile;                     // used when HAS_G
-    float* ms = gs + (HAS_G ? kDTile : 0);       // used when HAS_M
+    float* hs = xs + L::kStage;
+    float* ss = hs + L::kStage;
+    float* gs = ss + L::kStage;                     // used when HAS_G
+    float* ms = gs + (HAS_G ? L::kStage : 0);       // used when HAS_M
     unsigned char* msg_in = smem_raw + L::msg_in();
     unsigned char* msg_out = smem_raw + L::msg_out(nb_stage);
     // blocks of the norm per tile (gsgd_b); one "block" for sign
@@ -140,13 +171,18 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     const int row = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kDTile;
-    const int nvalid = (int)((dv.d - c0) < kDTile ? (dv.d - c0) : kDTile); // multiple of 4
+    const int nvalid = (int)((dv.d - c0) < kDTile ? (dv.d - c0) : kDTile); // AL: a multiple of 4
     const int e0 = dv.row_ptr[row], deg = dv.row_ptr[row + 1] - e0;
     const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
     float* xr = a.X + (int64_t)row * dv.ld + c0;
     float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
     float* sr = a.S + (int64_t)row * dv.ld + c0;
     float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
+    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld + c0 : nullptr;
+    // where each staged tile's first element sits in its shared-memory buffer
+    const uint32_t shx = AL ? 0u : unit_shift(xr), shh = AL ? 0u : unit_shift(hr), shs = AL ? 0u : unit_shift(sr);
+    const uint32_t shg = (AL || !HAS_G) ? 0u : unit_shift(gr), shm = (AL || !HAS_M) ? 0u : unit_shift(mrow);
+    auto span = [&](uint32_t sh) { return (((uint32_t)nvalid + sh) * (uint32_t)sizeof(float) + 15u) & ~15u; };
     // sizes of the slices actually present in this tile, rounded up to whole 16-byte units (the
     // message rows are padded so that the rounded slice of the last tile stays inside the row)
     const uint32_t dense_bytes = (uint32_t)nvalid * sizeof(float);
@@ -169,12 +205,13 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         const int count = deg < nb_stage ? deg : nb_stage;
         if (lane == 0) {
             mbar_init(bar, 1);
-            mbar_expect_tx(bar, dense_bytes * L::kArrays + (uint32_t)count * msg_bytes);
-            bulk_load(xs, xr, dense_bytes, bar);
-            bulk_load(hs, hr, dense_bytes, bar);
-            bulk_load(ss, sr, dense_bytes, bar);
-            if (HAS_G) bulk_load(gs, a.G + (int64_t)row * dv.ld + c0, dense_bytes, bar);
-            if (HAS_M) bulk_load(ms, mrow, dense_bytes, bar);
+            mbar_expect_tx(bar, span(shx) + span(shh) + span(shs) + (HAS_G ? span(shg) : 0u) + (HAS_M ? span(shm) : 0u) +
+                                    (uint32_t)count * msg_bytes);
+            bulk_load(xs, xr - shx, span(shx), bar);
+            bulk_load(hs, hr - shh, span(shh), bar);
+            bulk_load(ss, sr - shs, span(shs), bar);
+            if (HAS_G) bulk_load(gs, gr - shg, span(shg), bar);
+            if (HAS_M) bulk_load(ms, mrow - shm, span(shm), bar);
         }
         __syncwarp();
         stage_messages(0, count);
@@ -297,12 +334,12 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
         const int li = q4 * kQuad;
         vn[it] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (li < nvalid) {
-            const float4 x = reinterpret_cast<const float4*>(xs)[q4];
-            const float4 h = reinterpret_cast<const float4*>(hs)[q4];
-            const float4 s = reinterpret_cast<const float4*>(ss)[q4];
+            const float4 x = staged_quad<AL>(xs, shx, q4);
+            const float4 h = staged_quad<AL>(hs, shh, q4);
+            const float4 s = staged_quad<AL>(ss, shs, q4);
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f), m = g;
-            if (HAS_G) g = reinterpret_cast<const float4*>(gs)[q4];
-            if (HAS_M) m = reinterpret_cast<const float4*>(ms)[q4];
+            if (HAS_G) g = staged_quad<AL>(gs, shg, q4);
+            if (HAS_M) m = staged_quad<AL>(ms, shm, q4);
             const float4 hn = make_float4(__fadd_rn(h.x, qs[it][0]), __fadd_rn(h.y, qs[it][1]),
                                           __fadd_rn(h.z, qs[it][2]), __fadd_rn(h.w, qs[it][3]));
             const float4 sn = make_float4(__fadd_rn(s.x, acc[it][0]), __fadd_rn(s.y, acc[it][1]),
@@ -312,13 +349,25 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
             xn.y = next_x<HAS_G, HAS_M>(x.y, sn.y, hn.y, g.y, m.y, u);
             xn.z = next_x<HAS_G, HAS_M>(x.z, sn.z, hn.z, g.z, m.z, u);
             xn.w = next_x<HAS_G, HAS_M>(x.w, sn.w, hn.w, g.w, m.w, u);
-            reinterpret_cast<float4*>(hs)[q4] = hn;
-            reinterpret_cast<float4*>(ss)[q4] = sn;
-            reinterpret_cast<float4*>(xs)[q4] = xn;
-            if (HAS_M) reinterpret_cast<float4*>(ms)[q4] = m;
-            if (EMIT)
-                vn[it] = make_float4(__fsub_rn(xn.x, hn.x), __fsub_rn(xn.y, hn.y), __fsub_rn(xn.z, hn.z),
-                                     __fsub_rn(xn.w, hn.w));
+            const int left = nvalid - li; // >= 4 except in the last quad of an unaligned row
+            if (AL) {
+                reinterpret_cast<float4*>(hs)[q4] = hn;
+                reinterpret_cast<float4*>(ss)[q4] = sn;
+                reinterpret_cast<float4*>(xs)[q4] = xn;
+                if (HAS_M) reinterpret_cast<float4*>(ms)[q4] = m;
+            } else {
+                store_some(hr + li, hn, left);
+                store_some(sr + li, sn, left);
+                store_some(xr + li, xn, left);
+                if (HAS_M) store_some(mrow + li, m, left);
+            }
+            if (EMIT) {
+                // coordinates past d inside the last quad count as +0
+                vn[it].x = __fsub_rn(xn.x, hn.x);
+                if (AL || left > 1) vn[it].y = __fsub_rn(xn.y, hn.y);
+                if (AL || left > 2) vn[it].z = __fsub_rn(xn.z, hn.z);
+                if (AL || left > 3) vn[it].w = __fsub_rn(xn.w, hn.w);
+            }
         }
         if (EMIT) {
             const float4 v = vn[it];
@@ -338,10 +387,12 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     __syncthreads();
     const bool storer = threadIdx.x == 0;
     if (storer) {
-        bulk_store(xr, xs, dense_bytes);
-        bulk_store(hr, hs, dense_bytes);
-        bulk_store(sr, ss, dense_bytes);
-        if (HAS_M) bulk_store(mrow, ms, dense_bytes);
+        if (AL) {
+            bulk_store(xr, xs, dense_bytes);
+            bulk_store(hr, hs, dense_bytes);
+            bulk_store(sr, ss, dense_bytes);
+            if (HAS_M) bulk_store(mrow, ms, dense_bytes);
+        }
         if (EMIT) bulk_store(dv.nxt_bits + (int64_t)row * dv.wpitch + bits_off, msg_out, bits_bytes);
     }
     if (!EMIT) {
@@ -418,14 +469,14 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     }
 }
 
-template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT>
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
     using L = Layout<WBITS, HAS_G, HAS_M>;
     const int nb_stage = dv.maxdeg < kBatch ? dv.maxdeg : kBatch;
     const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
     const size_t smem = (size_t)L::total(nb_stage, nbk);
-    auto kern = update_dense_bulk_kernel<KIND, WBITS, HAS_G, HAS_M, EMIT>;
+    auto kern = update_dense_bulk_kernel<KIND, WBITS, HAS_G, HAS_M, EMIT, AL>;
     // Once per device, instantiation and size: allow the dynamic shared memory and ask for the
     // largest shared-memory carve-out, so that as many tiles as possible are in flight per SM.
     static size_t configured[64] = {};
@@ -444,23 +495,23 @@ cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
     return cudaGetLastError();
 }
 
-template <int KIND, int WBITS, bool EMIT>
+template <int KIND, int WBITS, bool EMIT, bool AL>
 cudaError_t launch_terms(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    if (a.M) return launch_one<KIND, WBITS, true, true, EMIT>(dv, a, st);
-    if (a.G) return launch_one<KIND, WBITS, true, false, EMIT>(dv, a, st);
-    return launch_one<KIND, WBITS, false, false, EMIT>(dv, a, st);
+    if (a.M) return launch_one<KIND, WBITS, true, true, EMIT, AL>(dv, a, st);
+    if (a.G) return launch_one<KIND, WBITS, true, false, EMIT, AL>(dv, a, st);
+    return launch_one<KIND, WBITS, false, false, EMIT, AL>(dv, a, st);
 }
 
-template <bool EMIT>
+template <bool EMIT, bool AL>
 cudaError_t launch_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    if (dv.kind == CHOCO_Q_SIGN) return launch_terms<CHOCO_Q_SIGN, 0, EMIT>(dv, a, st);
+    if (dv.kind == CHOCO_Q_SIGN) return launch_terms<CHOCO_Q_SIGN, 0, EMIT, AL>(dv, a, st);
     switch (dv.wbits) {
-    case 1: return launch_terms<CHOCO_Q_QSGD, 1, EMIT>(dv, a, st);
-    case 2: return launch_terms<CHOCO_Q_QSGD, 2, EMIT>(dv, a, st);
-    case 4: return launch_terms<CHOCO_Q_QSGD, 4, EMIT>(dv, a, st);
-    default: return launch_terms<CHOCO_Q_QSGD, 8, EMIT>(dv, a, st);
+    case 1: return launch_terms<CHOCO_Q_QSGD, 1, EMIT, AL>(dv, a, st);
+    case 2: return launch_terms<CHOCO_Q_QSGD, 2, EMIT, AL>(dv, a, st);
+    case 4: return launch_terms<CHOCO_Q_QSGD, 4, EMIT, AL>(dv, a, st);
+    default: return launch_terms<CHOCO_Q_QSGD, 8, EMIT, AL>(dv, a, st);
     }
 }
 
@@ -468,13 +519,14 @@ cudaError_t launch_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
 
 bool update_dense_bulk_usable(const Dev& dv, const StepArgs& a)
 {
-    if (!(a.vec && dv.d % 4 == 0)) return false;
     return dv.kind == CHOCO_Q_SIGN || (dv.kind == CHOCO_Q_QSGD && dv.bucket > 0);
 }
 
 cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {
-    return emit ? launch_kind<true>(dv, a, st) : launch_kind<false>(dv, a, st);
+    // a.vec: every row of every array starts on a 16-byte boundary
+    if (a.vec && dv.d % 4 == 0) return emit ? launch_kind<true, true>(dv, a, st) : launch_kind<false, true>(dv, a, st);
+    return emit ? launch_kind<true, false>(dv, a, st) : launch_kind<false, false>(dv, a, st);
 }
 
 } // namespace choco
