@@ -11,10 +11,10 @@
 // written back over the staged tiles and leave by bulk stores, as do the sign plane and the level
 // fields of the next message.  No thread holds a global address or a loaded value across a wait.
 // A bulk copy needs 16-byte aligned addresses and sizes.  With AL (rows 16-byte aligned, d a
-// multiple of 4) a tile is copied as it is and leaves the same way; otherwise each copy in starts
-// at the 16-byte boundary at or below the tile's first element and ends at the one at or above
-// its last, the tile is read from shared memory at the resulting offset of 0..3 elements, and the
-// results are stored from registers (a bulk store would overwrite the neighbours of a tile that
+// multiple of 4) a tile is copied as it is and leaves the same way; otherwise (rows that start on
+// 8-byte boundaries, any d) each copy in starts at the 16-byte boundary at or below the tile's
+// first element and ends at the one at or above its last, the tile is read from shared memory at
+// the resulting offset of 0 or 2 elements, and the results are stored from registers (a bulk store would overwrite the neighbours of a tile that
 // starts or ends inside a 16-byte unit).  The message planes are library-owned and always aligned.
 //
 // The per-coordinate work is kept to what the definition needs:
@@ -125,17 +125,15 @@ struct Layout {
 // element offset of p inside its 16-byte unit
 __device__ __forceinline__ uint32_t unit_shift(const float* p) { return (uint32_t)(((uintptr_t)p & 15u) >> 2); }
 
-// four consecutive floats of a staged tile that starts `sh` elements into its buffer
+// four consecutive floats of a staged tile that starts `sh` (0 or 2 unless AL) elements into its
+// buffer: 8-byte aligned, so two 64-bit reads
 template <bool AL>
 __device__ __forceinline__ float4 staged_quad(const float* buf, uint32_t sh, int q4)
 {
     if (AL) return reinterpret_cast<const float4*>(buf)[q4];
     const float* p = buf + sh + q4 * kQuad;
-    if ((sh & 1u) == 0u) { // 8-byte aligned: two 64-bit reads
-        const float2 lo = *reinterpret_cast<const float2*>(p), hi = *reinterpret_cast<const float2*>(p + 2);
-        return make_float4(lo.x, lo.y, hi.x, hi.y);
-    }
-    return make_float4(p[0], p[1], p[2], p[3]);
+    const float2 lo = *reinterpret_cast<const float2*>(p), hi = *reinterpret_cast<const float2*>(p + 2);
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
 }
 
 // store the first `left` (1..4) elements of v at p (4-byte aligned)
@@ -519,7 +517,11 @@ cudaError_t launch_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
 
 bool update_dense_bulk_usable(const Dev& dv, const StepArgs& a)
 {
-    return dv.kind == CHOCO_Q_SIGN || (dv.kind == CHOCO_Q_QSGD && dv.bucket > 0);
+    if (!(dv.kind == CHOCO_Q_SIGN || (dv.kind == CHOCO_Q_QSGD && dv.bucket > 0))) return false;
+    // every row of every array must start on an 8-byte boundary (16 with AL); rows that start
+    // at an odd element go to the register kernel
+    auto even = [](const void* p) { return ((uintptr_t)p & 7u) == 0; };
+    return dv.ld % 2 == 0 && even(a.X) && even(a.Xhat) && even(a.S) && even(a.G) && even(a.M);
 }
 
 cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
