@@ -445,6 +445,15 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             if (dv.emit_masks_smem) left -= 2 * dv.slab_pitch * 4;
             dv.emit_keys_cap = std::min<int64_t>(dv.cap, (left / 8) & ~(int64_t)3); // value bits and index per candidate
             dv.emit_smem_bytes = kEmitSmemBudget - left + dv.emit_keys_cap * 8;
+            // Few rows leave most SMs idle in a kernel with one block per row: let a cluster of
+            // 2 or 4 blocks serve each row, as long as all clusters still run at once.
+            int nsm = 0;
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, ctx->device);
+            dv.emit_cluster = n * 4 <= nsm ? 4 : (n * 2 <= nsm ? 2 : 1);
+            // candidates per block: what fits beside the fixed arrays, no more than a row can have
+            const int64_t budget_words = kEmitSmemBudget / 4;
+            int64_t cl = ((budget_words - 5152) * 8 / 17) & ~(int64_t)31; // 2.125 words per candidate
+            dv.emit_cap_local = std::min<int64_t>(cl, round_up(dv.cap, 32));
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_c, n * dv.slab_pitch);

@@ -90,6 +90,8 @@ struct Dev {
     int32_t emit_masks_smem;     // slab ballots in shared memory
     int64_t emit_keys_cap;       // candidate keys cached in shared memory up to this many
     int64_t emit_smem_bytes;     // dynamic shared memory of the emit kernel
+    int32_t emit_cluster;        // blocks that serve one row together (a thread-block cluster); 1 = one block
+    int64_t emit_cap_local;      // candidates one block of the cluster can hold in shared memory
     Stats* stats;
     uint32_t wait_polls;         // bound of the kernels' first wait for their staged copies
     // what steps ask the L2 cache to keep resident (sparse Q): messages, range records, tables

@@ -15,6 +15,10 @@
 //             next step.
 //   exact   : rows whose candidates are unusable (too many, too few, overflow) are selected
 //             exactly, by the same block, straight from the dense row.
+#include <cooperative_groups.h>
+
+#include <algorithm>
+
 #include "bulk.cuh"
 #include "select.cuh"
 
@@ -515,16 +519,12 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
 // `rescue`: 0 = a row whose candidates cannot be used is selected exactly by this block;
 // 1 = such a row is flagged kRowRescue instead and left to the rescue kernels that follow;
 // 2 = this launch is their last stage and serves the flagged rows only.
+// One block serves one row.  `dyn` is the block's dynamic shared memory (dv.emit_smem_bytes), `h`
+// kHistBins words, `sm` 64 words and `s_carry` 2 words of shared memory.
 template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
+__device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a, int row, int fused, int rescue,
+                                                uint32_t* dyn, uint32_t* h, uint32_t* sm, uint32_t* s_carry)
 {
-    extern __shared__ __align__(16) uint32_t dyn[];
-    __shared__ uint32_t h[kHistBins];
-    __shared__ uint32_t sm[64];
-    __shared__ uint32_t s_carry[2];
-    wait_for_previous_kernel(); // the candidates come from the kernel before this one
-    allow_next_kernel();
-    const int row = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ncand = dv.row_count[row];
     const uint32_t flags = dv.row_flags[row];
@@ -729,6 +729,355 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     }
 }
 
+template <int KIND, bool VEC>
+__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
+{
+    extern __shared__ __align__(16) uint32_t dyn[];
+    __shared__ uint32_t h[kHistBins];
+    __shared__ uint32_t sm[64];
+    __shared__ uint32_t s_carry[2];
+    wait_for_previous_kernel(); // the candidates come from the kernel before this one
+    allow_next_kernel();
+    emit_row_single<KIND, VEC>(dv, a, (int)blockIdx.x, fused, rescue, dyn, h, sm, s_carry);
+}
+
+// ---------------------------------------------------------------------------------------
+// emit, several blocks per row: a thread-block cluster serves one row.
+//
+// The candidates of a row lie in the candidate arrays tile by tile, ascending inside a tile,
+// but the tiles in the order in which their blocks of the update kernel happened to reserve
+// space.  Here the tiles are cut into one run per block of the cluster, of about equal
+// candidate counts, and every block gathers its run into shared memory IN TILE ORDER.  The
+// concatenation of the blocks' arrays is then the row's candidate list in ascending coordinate
+// order, and the message is simply its ordered compaction:
+//   1. k-th key T: histogram refinement as in the one-block kernel, each block counting its own
+//      keys and all blocks adding the counts up through distributed shared memory;
+//   2. per 32-candidate slab the ballots of "above T" / "equal to T", prefix sums inside the
+//      block, the blocks' totals exchanged: every candidate then knows how many chosen ones
+//      precede it in the whole row and writes itself;
+//   3. tile_ptr and the range records follow from the same prefixes at each tile's first candidate.
+// Every decision that steers the control flow (usable or not, number of refinement rounds) is
+// taken from values all blocks of the cluster hold alike, so they reach every cluster barrier
+// together.  A row whose candidates cannot be used, or whose share per block does not fit the
+// shared memory, is left to block 0, which runs the one-block algorithm above.
+// ---------------------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+
+constexpr int kMaxCluster = 4;
+constexpr int kGroup = 8; // lanes that copy one tile's candidates
+
+// words of dynamic shared memory the cluster algorithm needs for `cap_local` candidates per block
+__host__ __device__ inline int64_t cluster_emit_words(int64_t cap_local)
+{
+    const int64_t spitch = ((cap_local >> 5) + 2 + 3) & ~(int64_t)3;
+    return 2 * cap_local + 4 * spitch + 3 * (kSelThreads + 4) + 2 * kListCap;
+}
+
+template <int KIND, bool VEC>
+__global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepArgs a, int fused, int rescue)
+{
+    extern __shared__ __align__(16) uint32_t dyn[];
+    __shared__ uint32_t h2[2][kHistBins]; // this block's histogram of the current / the previous round
+    __shared__ uint32_t hsum[kHistBins];  // the cluster's
+    __shared__ uint32_t sm[64];
+    __shared__ uint32_t s_carry[2];
+    __shared__ uint32_t xch[8];           // what this block shows the others: key range, counts
+    __shared__ uint32_t part_t[kMaxCluster + 1], part_p[kMaxCluster + 1]; // first tile / candidate of each block's run
+    wait_for_previous_kernel(); // the candidates come from the kernel before this one
+    allow_next_kernel();
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t C = cluster.num_blocks(), rank = cluster.block_rank();
+    const int row = (int)(blockIdx.x / C);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ncand = dv.row_count[row], flags = dv.row_flags[row], k = (uint32_t)dv.k;
+    if (rescue == 2 && !(flags & kRowRescue)) return;
+    const bool unusable = (flags & kRowExact) || ncand > (uint32_t)dv.cap || ncand < k;
+    const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
+    const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
+    const uint32_t ntiles = (uint32_t)dv.ntiles;
+
+    // the runs: tile t goes to block floor(candidates before t * C / ncand)
+    if (threadIdx.x <= C) {
+        part_t[threadIdx.x] = threadIdx.x == 0 ? 0u : ntiles;
+        part_p[threadIdx.x] = threadIdx.x == 0 ? 0u : ncand;
+    }
+    __syncthreads();
+    if (!unusable) {
+        uint32_t carry = 0;
+        for (uint32_t t0 = 0; t0 < ntiles; t0 += kSelThreads) {
+            const uint32_t t = t0 + threadIdx.x;
+            const uint32_t cnt = t < ntiles ? sc[t] : 0u;
+            uint32_t tot;
+            const uint32_t ex = carry + block_scan_excl<kSelThreads>(cnt, sm, &tot);
+            if (t < ntiles) {
+                const uint32_t top = C - 1u;
+                uint32_t mine = (uint32_t)(((uint64_t)ex * C) / ncand);
+                mine = mine < top ? mine : top;
+                int prev = -1;
+                if (t > 0) {
+                    const uint32_t pv = (uint32_t)(((uint64_t)(ex - sc[t - 1]) * C) / ncand);
+                    prev = (int)(pv < top ? pv : top);
+                }
+                for (uint32_t c = 1; c < C; ++c)
+                    if (mine >= c && prev < (int)c) { part_t[c] = t; part_p[c] = ex; }
+            }
+            carry += tot;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && carry != ncand) part_p[1] = 0xFFFFFFFFu; // inconsistent counts: do not trust the runs
+        __syncthreads();
+    }
+    const int64_t cap_local = dv.emit_cap_local;
+    bool fits = !unusable;
+    for (uint32_t c = 0; c < C && fits; ++c)
+        fits = part_p[c + 1] >= part_p[c] && (int64_t)(part_p[c + 1] - part_p[c]) <= cap_local;
+    // Every block has now read the row's state; none has changed it yet.  Only behind this
+    // barrier may block 0 go its own way (it rewrites the row's flags and counts), so that all
+    // blocks reach the same verdict from the same values.
+    cluster.sync();
+    if (!fits) { // block 0 serves the row alone, with the one-block algorithm
+        if (rank == 0) emit_row_single<KIND, VEC>(dv, a, row, fused, rescue, dyn, h2[0], sm, s_carry);
+        return;
+    }
+
+    // carve the dynamic shared memory
+    const int64_t spitch = ((cap_local >> 5) + 2 + 3) & ~(int64_t)3;
+    uint32_t* keys = dyn;                       // value bits of this block's candidates, in tile order
+    uint32_t* idxs = keys + cap_local;          // their coordinates
+    uint32_t* slab_g = idxs + cap_local;        // per slab: keys above T (then: before the slab)
+    uint32_t* slab_e = slab_g + spitch;         //           keys equal to T
+    uint32_t* slab_gm = slab_e + spitch;        //           ballots of the two
+    uint32_t* slab_em = slab_gm + spitch;
+    uint32_t* st_a = slab_em + spitch;          // per tile of the pass: first candidate in the arrays / output position
+    uint32_t* st_b = st_a + (kSelThreads + 4);  //                        candidates
+    uint32_t* st_c = st_b + (kSelThreads + 4);  //                        first candidate in this block's order
+    uint32_t* list_mine = st_c + (kSelThreads + 4);
+    uint32_t* list_all = list_mine + kListCap;
+
+    const uint32_t Tb = part_t[rank], Te = part_t[rank + 1];
+    const uint32_t L = part_p[rank + 1] - part_p[rank];   // this block's candidates
+    const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
+    const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
+
+    // gather: a group of kGroup lanes copies one tile's candidates
+    uint32_t klo = 0xFFFFFFFFu, khi = 0u;
+    {
+        uint32_t carry = 0;
+        for (uint32_t t0 = Tb; t0 < Te; t0 += kSelThreads) {
+            const uint32_t t = t0 + threadIdx.x;
+            const uint32_t cnt = t < Te ? sc[t] : 0u;
+            uint32_t tot;
+            const uint32_t ex = carry + block_scan_excl<kSelThreads>(cnt, sm, &tot);
+            st_a[threadIdx.x] = t < Te ? so[t] : 0u;
+            st_b[threadIdx.x] = cnt;
+            st_c[threadIdx.x] = ex;
+            __syncthreads();
+            const uint32_t nt = (Te - t0) < (uint32_t)kSelThreads ? (Te - t0) : (uint32_t)kSelThreads;
+            for (uint32_t i = threadIdx.x / kGroup; i < nt; i += kSelThreads / kGroup) {
+                const uint32_t g = st_a[i], c = st_b[i], l = st_c[i];
+                for (uint32_t j = threadIdx.x % kGroup; j < c; j += kGroup) {
+                    const uint32_t bits = __ldg(cv + g + j);
+                    keys[l + j] = bits;
+                    idxs[l + j] = __ldg(ci + g + j);
+                    const uint32_t kk = order_key<KIND>(bits);
+                    klo = kk < klo ? kk : klo;
+                    khi = kk > khi ? kk : khi;
+                }
+            }
+            carry += tot;
+            __syncthreads(); // the staging arrays are written again by the next pass
+        }
+    }
+    block_min_max(klo, khi, sm);
+    if (threadIdx.x == 0) { xch[0] = klo; xch[1] = khi; }
+    cluster.sync();
+    for (uint32_t c = 0; c < C; ++c) {
+        const uint32_t* o = cluster.map_shared_rank(xch, c);
+        const uint32_t a0 = o[0], a1 = o[1];
+        klo = a0 < klo ? a0 : klo;
+        khi = a1 > khi ? a1 : khi;
+    }
+    auto key_at = [&](uint32_t p) -> uint32_t { return order_key<KIND>(keys[p]); };
+
+    // 1. the k-th key: refinement over the range the keys span, counts added up over the cluster
+    uint32_t T, above_total = 0;
+    {
+        uint32_t need = k, lo = klo, hi = khi;
+        int buf = 0;
+        for (;;) {
+            const uint32_t width = hi - lo;
+            const int shift = width < (uint32_t)kHistBins ? 0 : (32 - __clz(width)) - 11;
+            const int nbins = (int)(width >> shift) + 1; // <= kHistBins
+            uint32_t* h = h2[buf];
+            for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
+            __syncthreads();
+            for (uint32_t p = threadIdx.x; p < L; p += kSelThreads) {
+                const uint32_t kk = key_at(p);
+                if (kk >= lo && kk <= hi) atomicAdd(&h[(kk - lo) >> shift], 1u);
+            }
+            cluster.sync(); // every block's counts of this round are complete
+            for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) {
+                uint32_t v = 0;
+                for (uint32_t c = 0; c < C; ++c) v += cluster.map_shared_rank(&h2[buf][0], c)[b];
+                hsum[b] = v;
+            }
+            __syncthreads();
+            uint32_t digit, above;
+            block_find_digit<kSelThreads>(hsum, nbins, need, sm, &digit, &above);
+            const uint32_t inbin = hsum[digit];
+            need -= above;
+            above_total += above;
+            const uint32_t nlo = lo + (digit << shift);
+            const uint32_t span = shift ? ((1u << shift) - 1u) : 0u;
+            const uint32_t nhi = (hi - nlo) < span ? hi : nlo + span;
+            lo = nlo;
+            hi = nhi;
+            __syncthreads();
+            if (shift == 0) break;
+            if (inbin <= (uint32_t)kListCap) {
+                // few keys left in [lo, hi]: every block lists its own, all read all lists and rank directly
+                uint32_t* count = sm + 40;
+                if (threadIdx.x == 0) { *count = 0u; sm[41] = lo; sm[42] = 0u; }
+                __syncthreads();
+                for (uint32_t p = threadIdx.x; p < L; p += kSelThreads) {
+                    const uint32_t kk = key_at(p);
+                    if (kk >= lo && kk <= hi) list_mine[atomicAdd(count, 1u)] = kk;
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) xch[2] = *count;
+                cluster.sync();
+                uint32_t m = 0;
+                for (uint32_t c = 0; c < C; ++c) {
+                    const uint32_t mc = cluster.map_shared_rank(xch, c)[2];
+                    const uint32_t* src = cluster.map_shared_rank(list_mine, c);
+                    if (m + mc <= (uint32_t)kListCap)
+                        for (uint32_t q = threadIdx.x; q < mc; q += kSelThreads) list_all[m + q] = src[q];
+                    m += mc;
+                }
+                m = m < (uint32_t)kListCap ? m : (uint32_t)kListCap; // == inbin
+                __syncthreads();
+                if (threadIdx.x < m) {
+                    const uint32_t mine = list_all[threadIdx.x];
+                    uint32_t g = 0, e = 0;
+                    for (uint32_t q = 0; q < m; ++q) {
+                        g += list_all[q] > mine;
+                        e += list_all[q] == mine;
+                    }
+                    if (g < need && need <= g + e) { sm[41] = mine; sm[42] = g; } // same values from every such thread
+                }
+                __syncthreads();
+                lo = sm[41];
+                above_total += sm[42];
+                __syncthreads();
+                break;
+            }
+            buf ^= 1;
+        }
+        T = lo;
+    }
+    const uint32_t r = k - above_total; // how many coordinates with key == T are kept (lowest first)
+
+    if (KIND == SEL_TOPK && rank == 0 && threadIdx.x == 0) {
+        // candidate bound for the next step (see the one-block kernel)
+        uint32_t aim = dv.row_aim[row];
+        aim = aim > kAimMin + kAimStep ? aim - kAimStep : kAimMin;
+        dv.row_aim[row] = aim;
+        dv.row_lo[row] = next_bound(dv.row_lo[row], T, ncand, k, aim);
+    }
+
+    // 2. ballots per slab of 32 candidates, prefixes inside the block, totals over the cluster
+    const int64_t nslab = ((int64_t)L + 31) >> 5;
+    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+        const uint32_t p = (uint32_t)(sl << 5) + lane;
+        bool gt = false, eq = false;
+        if (p < L) {
+            const uint32_t kk = key_at(p);
+            gt = kk > T;
+            eq = kk == T;
+        }
+        const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) { slab_g[sl] = __popc(bg); slab_e[sl] = __popc(be); slab_gm[sl] = bg; slab_em[sl] = be; }
+    }
+    __syncthreads();
+    uint32_t tot_g, tot_e;
+    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
+    if (threadIdx.x == 0) { xch[4] = tot_g; xch[5] = tot_e; }
+    cluster.sync();
+    uint32_t og = 0, oe = 0; // keys above / equal to T in the blocks before this one
+    for (uint32_t c = 0; c < rank; ++c) {
+        const uint32_t* o = cluster.map_shared_rank(xch, c);
+        og += o[4];
+        oe += o[5];
+    }
+    // output position of the candidate at position `pos` of this block (pos == L: of the next block's first)
+    auto out_pos = [&](uint32_t pos) -> uint32_t {
+        uint32_t g = tot_g, e = tot_e;
+        const uint32_t s0 = pos >> 5;
+        if ((int64_t)s0 < nslab) {
+            const uint32_t below = (1u << (pos & 31u)) - 1u;
+            g = slab_g[s0] + __popc(slab_gm[s0] & below);
+            e = slab_e[s0] + __popc(slab_em[s0] & below);
+        }
+        e += oe;
+        return og + g + (e < r ? e : r);
+    };
+    // every chosen candidate writes itself
+    uint32_t* mi = dv.msg_idx + (int64_t)row * dv.kpitch;
+    float* mv = dv.msg_val + (int64_t)row * dv.kpitch;
+    const float* xr = a.X + (int64_t)row * dv.ld;
+    const float* hr = a.Xhat + (int64_t)row * dv.ld;
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+        const uint32_t bg = slab_gm[sl], be = slab_em[sl];
+        const bool gt = (bg >> lane) & 1u, eq = (be >> lane) & 1u;
+        if (gt | eq) {
+            const uint32_t p = (uint32_t)(sl << 5) + lane;
+            const uint32_t e_before = oe + slab_e[sl] + __popc(be & lt);
+            if (gt || e_before < r) {
+                const uint32_t pos = og + slab_g[sl] + __popc(bg & lt) + (e_before < r ? e_before : r);
+                const uint32_t id = idxs[p];
+                mi[pos] = id;
+                mv[pos] = KIND == SEL_TOPK ? __uint_as_float(keys[p]) : __fsub_rn(xr[id], hr[id]);
+            }
+        }
+    }
+    // 3. tile_ptr and the range records of this block's tiles
+    uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
+    {
+        const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
+        uint32_t carry = 0;
+        for (uint32_t t0 = Tb; t0 < Te; t0 += kSelThreads) {
+            const uint32_t t = t0 + threadIdx.x;
+            const uint32_t cnt = t < Te ? sc[t] : 0u;
+            uint32_t tot;
+            const uint32_t ex = carry + block_scan_excl<kSelThreads>(cnt, sm, &tot);
+            // (a tile past the pass reads the position behind the pass's last candidate)
+            st_a[threadIdx.x] = out_pos(ex);
+            if (threadIdx.x == 0) st_a[kSelThreads] = out_pos(carry + tot);
+            __syncthreads();
+            if (t < Te) {
+                const uint32_t first = st_a[threadIdx.x], count = st_a[threadIdx.x + 1] - first;
+                tp[t] = first;
+                for (int e = e0; e < e1; ++e) {
+                    const int64_t reader = dv.col[e];
+                    dv.rec[(reader * dv.ntiles + t) * dv.maxdeg + dv.rd_pos[e]] =
+                        make_uint4((uint32_t)row, first, count, __float_as_uint(dv.rd_w[e]));
+                }
+            }
+            carry += tot;
+            __syncthreads();
+        }
+    }
+    if (rank == C - 1 && threadIdx.x == 0) tp[dv.ntiles] = k;
+    // no block may leave while another still reads its shared memory
+    cluster.sync();
+    if (rank == 0 && threadIdx.x == 0) {
+        dv.row_count[row] = 0u;
+        dv.row_flags[row] = 0u;
+        atomicAdd(fused ? &dv.stats->prepared_rows : &dv.stats->recompressed_rows, 1ull);
+    }
+}
+
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
@@ -769,19 +1118,58 @@ cudaError_t launch_select_prepare(const Dev& dv, const StepArgs& a, cudaStream_t
 template <int KIND>
 static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int rescue, cudaStream_t st)
 {
-    auto kern = a.vec ? emit_kernel<KIND, true> : emit_kernel<KIND, false>;
-    static bool configured[64][2] = {};
+    const int vec = a.vec ? 1 : 0;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev][a.vec ? 1 : 0]) {
+    if (dv.emit_cluster > 1) {
+        // several blocks per row (a thread-block cluster); shared memory for either algorithm
+        auto kern = a.vec ? emit_cluster_kernel<KIND, true> : emit_cluster_kernel<KIND, false>;
+        const size_t bytes = std::max<size_t>((size_t)dv.emit_smem_bytes, (size_t)cluster_emit_words(dv.emit_cap_local) * 4);
+        static size_t configured[64][2] = {};
+        if (dev < 0 || dev >= 64 || configured[dev][vec] < bytes) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) configured[dev][vec] = bytes;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)dv.n * (unsigned)dv.emit_cluster);
+        cfg.blockDim = dim3(kSelThreads);
+        cfg.dynamicSmemBytes = bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[3];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)dv.emit_cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+        const HotRange hot = hot_range_of(dv);
+        if (hot.base && hot.bytes > 0 && hot.ratio > 0.f) {
+            attr[2].id = cudaLaunchAttributeAccessPolicyWindow;
+            attr[2].val.accessPolicyWindow.base_ptr = hot.base;
+            attr[2].val.accessPolicyWindow.num_bytes = hot.bytes;
+            attr[2].val.accessPolicyWindow.hitRatio = hot.ratio;
+            attr[2].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+            attr[2].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+            cfg.numAttrs = 3;
+        }
+        cfg.attrs = attr;
+        e = cudaLaunchKernelEx(&cfg, kern, dv, a, fused ? 1 : 0, rescue);
+        if (e != cudaSuccess) return e;
+        *a.launches += 1;
+        return cudaGetLastError();
+    }
+    auto kern = a.vec ? emit_kernel<KIND, true> : emit_kernel<KIND, false>;
+    static bool configured[64][2] = {};
+    if (dev < 0 || dev >= 64 || !configured[dev][vec]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmitSmemBudget);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev][a.vec ? 1 : 0] = true;
+        if (dev >= 0 && dev < 64) configured[dev][vec] = true;
     }
     e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st,
-                          hot_range_of(dv), dv, a,
-                          fused ? 1 : 0, rescue);
+                          hot_range_of(dv), dv, a, fused ? 1 : 0, rescue);
     if (e != cudaSuccess) return e;
     *a.launches += 1;
     return cudaGetLastError();
