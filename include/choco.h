@@ -199,6 +199,16 @@ int choco_set_graphs(choco_ctx* ctx, int32_t enable);
  */
 int choco_set_rescue(choco_ctx* ctx, int32_t enable);
 
+/*
+ * The kernel that selects the k entries of a row among its candidates runs one thread block per
+ * row, or -- for rows with many candidates (capacity of 32 768 or more) when the workers are few
+ * enough that all SMs would not be busy otherwise -- a cluster of 2 or 4 blocks per row that
+ * share the row through distributed shared memory.  choco_set_select_blocks -- blocks = 1, 2 or
+ * 4 overrides that choice for the context (TOPK / RANDK only; CHOCO_ERR_UNSUPPORTED otherwise).
+ * The result is the same either way.
+ */
+int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks);
+
 /* Step counter t (keys the generator).  Setting it, together with restoring X, Xhat and S,
  * resumes a run bit-exactly; choco_set_step implies choco_invalidate. */
 int choco_get_step(const choco_ctx* ctx, uint64_t* t);

@@ -21,7 +21,7 @@ Q_KINDS = {"identity": Q_IDENTITY, "topk": Q_TOPK, "randk": Q_RANDK, "qsgd": Q_Q
 EXPORTS = [
     "choco_init", "choco_destroy", "choco_gossip_step", "choco_sgd_step",
     "choco_sgd_momentum_step", "choco_sgd_step_host", "choco_invalidate", "choco_set_carry",
-    "choco_get_step", "choco_set_graphs", "choco_set_rescue",
+    "choco_get_step", "choco_set_graphs", "choco_set_rescue", "choco_set_select_blocks",
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
@@ -79,6 +79,7 @@ def load() -> ctypes.CDLL:
         lib.choco_set_carry.argtypes = [vp, i32]
         lib.choco_set_graphs.argtypes = [vp, i32]
         lib.choco_set_rescue.argtypes = [vp, i32]
+        lib.choco_set_select_blocks.argtypes = [vp, i32]
         lib.choco_get_step.argtypes = [vp, ctypes.POINTER(u64)]
         lib.choco_set_step.argtypes = [vp, u64]
         lib.choco_message_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -194,6 +195,10 @@ def choco_set_graphs(ctx, enable: bool) -> None:
 
 def choco_set_rescue(ctx, enable: bool) -> None:
     _check(load().choco_set_rescue(ctx, 1 if enable else 0), ctx)
+
+
+def choco_set_select_blocks(ctx, blocks: int) -> None:
+    _check(load().choco_set_select_blocks(ctx, blocks), ctx)
 
 
 def choco_get_step(ctx) -> int:

@@ -450,6 +450,9 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             int nsm = 0;
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, ctx->device);
             dv.emit_cluster = n * 4 <= nsm ? 4 : (n * 2 <= nsm ? 2 : 1);
+            // (rows with few candidates are served faster by one block: the cluster's barriers
+            // and exchanges cost more than the shared work saves; measured on d = 272 474, k = 2 724)
+            if (dv.cap < 32768) dv.emit_cluster = 1;
             // candidates per block: what fits beside the fixed arrays, no more than a row can have
             const int64_t budget_words = kEmitSmemBudget / 4;
             int64_t cl = ((budget_words - 5152) * 8 / 17) & ~(int64_t)31; // 2.125 words per candidate
@@ -609,6 +612,18 @@ int choco_set_rescue(choco_ctx* ctx, int32_t enable)
     // the kernels a step enqueues change: no captured step stands for it any more
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) { cudaGraphExecDestroy(ctx->graphs[i].exec); }
+    ctx->ngraphs = 0;
+    return CHOCO_OK;
+}
+
+int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks)
+{
+    if (!ctx || !(blocks == 1 || blocks == 2 || blocks == 4)) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->dv.kind != CHOCO_Q_TOPK && ctx->dv.kind != CHOCO_Q_RANDK) return CHOCO_ERR_UNSUPPORTED;
+    ctx->dv.emit_cluster = blocks;
+    // the kernels a step enqueues change: no captured step stands for it any more
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
     ctx->ngraphs = 0;
     return CHOCO_OK;
 }

@@ -61,13 +61,15 @@ def check_messages(ctx, kind, msgs, d):
 
 def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed=0, ld=None,
                  eta=0.1, gamma=0.2, x_var=1.0, g_var=0.01, sgd=True, momentum=False,
-                 x_init=None, check_msgs=True, grad_fn=None):
+                 x_init=None, check_msgs=True, grad_fn=None, select_blocks=None):
     ld = ld or d
     X = workloads.normal_rows(n, d, x_var, 1000 + seed) if x_init is None else x_init.copy()
     Xh, S = np.zeros_like(X), np.zeros_like(X)
     M = np.zeros_like(X) if momentum else None
     p = oracle.Params(kind, k=k, s=s, bucket=bucket, biased=biased, seed=seed)
     ch = choco.Choco(w, d, kind, k=k, s=s, bucket=bucket, qsgd_biased=biased, seed=seed, ld=ld)
+    if select_blocks:
+        choco.choco_set_select_blocks(ch.ctx, select_blocks)
     dX, dXh, dS = _dev(X, ld), _dev(Xh, ld), _dev(S, ld)
     dM = _dev(M, ld) if momentum else None
     try:
@@ -147,6 +149,34 @@ def test_topk_shapes(d, k, ld):
 def test_randk_shapes(d, k, ld):
     ch, _, _ = run_lockstep(workloads.ring(5), "randk", 5, d, 3, k=k, ld=ld, seed=d + k)
     assert choco.choco_message_bytes(ch.ctx) == (4 * k, 4 * k * 5)
+    ch.close()
+
+
+@pytest.mark.parametrize("blocks", [2, 4])
+@pytest.mark.parametrize("kind,d,k,ld", [("topk", 1, 1, None), ("topk", 33, 33, 36), ("topk", 2000, 20, None),
+                                         ("topk", 4097, 300, 4100), ("topk", 10007, 10007, None),
+                                         ("topk", 50000, 500, None), ("topk", 300000, 3000, None),
+                                         ("randk", 2000, 20, None), ("randk", 50000, 5000, None)])
+def test_selection_by_a_cluster_of_blocks_per_row(kind, d, k, ld, blocks):
+    """The selection kernel with 2 or 4 blocks per row (normally chosen for large rows only):
+    one tile, ragged tiles, k = d, more tiles than threads in a block's pass, several steps so
+    that carried candidates are selected from too."""
+    ch, _, _ = run_lockstep(workloads.ring(5), kind, 5, d, 4, k=k, ld=ld, seed=d + k + blocks, select_blocks=blocks)
+    ch.close()
+
+
+@pytest.mark.parametrize("blocks", [2, 4])
+def test_ties_with_a_cluster_of_blocks_per_row(blocks):
+    """Ties at the k-th key that straddle the blocks' shares: rows of few distinct magnitudes."""
+    n, d, k = 4, 60000, 700
+    rng = np.random.default_rng(blocks)
+    x = np.zeros((n, d), dtype=np.float32)
+    x[0] = rng.choice([-2.0, 2.0, 1.0, -1.0], size=d).astype(np.float32)
+    x[1] = rng.integers(-3, 4, size=d).astype(np.float32)
+    x[2] = rng.standard_normal(d).astype(np.float32)
+    x[2, 1000:1400] = x[2, 50]
+    x[3] = np.round(rng.standard_normal(d) * 4).astype(np.float32) / 4
+    ch, _, _ = run_lockstep(workloads.ring(n), "topk", n, d, 5, k=k, x_init=x, seed=2, select_blocks=blocks)
     ch.close()
 
 
