@@ -282,15 +282,20 @@ int choco_consensus_error_noalloc(const float* X, int32_t n, int64_t d, int64_t 
  *   the generator of layer l is keyed with seed + l and the coordinate's index inside the layer.
  * Everything else (Algorithm 1 / 2, arithmetic, determinism) is as for the plain calls: a
  * layered step gives the same bits as running choco_*_step with d = d_l, seed + l and
- * pointers advanced by layer_off[l] for every layer.  That is also how it is carried out: one
- * library context per layer, their kernels spread over a few internal streams that fork from
- * and join `stream`, a few kernel launches per layer.  A steady-state step is captured into a
- * CUDA graph the second time it is seen with a given set of arguments (the array pointers, eta,
- * gamma, lambda, beta) and replayed by one graph launch afterwards; up to 32 such graphs are
- * kept.  (QSGD and RANDK contexts of a layered context keep the step number in device memory
- * for this and bump it with one more tiny kernel per step.)  A step call made while `stream`
- * is itself being captured, or on the legacy default stream, which cannot be captured, is
- * enqueued kernel by kernel instead.
+ * pointers advanced by layer_off[l] for every layer.  One library context per layer holds the
+ * layer's parameters, messages and workspace.  For TOPK, SIGN and QSGD with blocks, when the
+ * layers are small enough for launches to dominate (at most 32 768 tiles of 2048 coordinates
+ * over all layers and workers, at most 512 layers), the steady-state step of all layers
+ * together is two or three kernel launches whose blocks look their layer up in a table (layers whose rows start at odd elements, which those kernels do
+ * not take for the dense operators, run their own few launches beside them).  First steps, steps
+ * after choco_layers_invalidate and the other operators run layer by layer, their kernels spread
+ * over a few internal streams that fork from and join `stream`; for those operators a
+ * steady-state step is captured into a CUDA graph the second time it is seen with a given set
+ * of arguments (the array pointers, eta, gamma, lambda, beta) and replayed by one graph launch
+ * afterwards; up to 32 such graphs are kept.  (Whole-row QSGD and RANDK contexts of a layered
+ * context keep the step number in device memory for this and bump it with one more tiny kernel
+ * per step.)  A step call made while `stream` is itself being captured, or on the legacy default
+ * stream, which cannot be captured, is enqueued kernel by kernel instead.
  *   layer_off[n_layers + 1]   HOST, strictly increasing from 0; ld >= layer_off[n_layers].
  *   a_num, a_den              used by TOPK / RANDK only.
  * Errors are those of choco_init; on error nothing is left allocated.
@@ -316,6 +321,8 @@ int choco_layers_get_layer(const choco_layers* layers, int32_t layer, choco_ctx*
 /* enable = 0 / 1 turns the graph replay described above off / on (default on), a negative
  * value leaves it as it is; *replays (may be NULL) receives the number of steps replayed so far. */
 int choco_layers_set_graphs(choco_layers* layers, int32_t enable, uint64_t* replays);
+/* Number of step calls so far that were enqueued as the combined launches described above. */
+int choco_layers_combined_steps(const choco_layers* layers, uint64_t* steps);
 /* choco_invalidate / choco_set_step for every layer. */
 int choco_layers_invalidate(choco_layers* layers);
 int choco_layers_set_step(choco_layers* layers, uint64_t t);

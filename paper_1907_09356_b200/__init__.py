@@ -28,7 +28,7 @@ EXPORTS = [
     "choco_last_cuda_error", "choco_debug_set_wait_polls",
     "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
     "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
-    "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_graphs",
+    "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_graphs", "choco_layers_combined_steps",
 ]
 
 
@@ -107,6 +107,7 @@ def load() -> ctypes.CDLL:
         lib.choco_layers_invalidate.argtypes = [vp]
         lib.choco_layers_set_step.argtypes = [vp, u64]
         lib.choco_layers_set_graphs.argtypes = [vp, i32, ctypes.POINTER(u64)]
+        lib.choco_layers_combined_steps.argtypes = [vp, ctypes.POINTER(u64)]
         for name in EXPORTS:
             if name not in ("choco_strerror",):
                 getattr(lib, name).restype = ctypes.c_int
@@ -330,6 +331,13 @@ def choco_layers_set_graphs(layers, enable: int = -1) -> int:
     returns the number of steps replayed so far."""
     n = ctypes.c_uint64()
     _check(load().choco_layers_set_graphs(layers, enable, ctypes.byref(n)))
+    return n.value
+
+
+def choco_layers_combined_steps(layers) -> int:
+    """Step calls so far that were enqueued as launches over all layers at once."""
+    n = ctypes.c_uint64()
+    _check(load().choco_layers_combined_steps(layers, ctypes.byref(n)))
     return n.value
 
 

@@ -609,6 +609,7 @@ int choco_set_rescue(choco_ctx* ctx, int32_t enable)
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
     if (ctx->dv.kind != CHOCO_Q_TOPK) return enable ? CHOCO_ERR_UNSUPPORTED : CHOCO_OK;
     ctx->dv.rescue = enable ? 1 : 0;
+    ctx->dv_epoch += 1;
     // the kernels a step enqueues change: no captured step stands for it any more
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) { cudaGraphExecDestroy(ctx->graphs[i].exec); }
@@ -621,6 +622,7 @@ int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks)
     if (!ctx || !(blocks == 1 || blocks == 2 || blocks == 4)) return CHOCO_ERR_INVALID_ARG;
     if (ctx->dv.kind != CHOCO_Q_TOPK && ctx->dv.kind != CHOCO_Q_RANDK) return CHOCO_ERR_UNSUPPORTED;
     ctx->dv.emit_cluster = blocks;
+    ctx->dv_epoch += 1;
     // the kernels a step enqueues change: no captured step stands for it any more
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
@@ -759,6 +761,7 @@ int choco_debug_set_wait_polls(choco_ctx* ctx, uint32_t polls)
 {
     if (!ctx) return CHOCO_ERR_INVALID_ARG;
     ctx->dv.wait_polls = polls > kSpinLimit ? kSpinLimit : polls;
+    ctx->dv_epoch += 1;
     // the bound is a kernel argument: no captured step stands for it any more
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);

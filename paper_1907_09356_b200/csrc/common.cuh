@@ -188,6 +188,35 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
 }
 
 
+// Layered launches.  entry_of_block: the table entry whose blocks include `block`.
+__device__ __forceinline__ int entry_of_block(const LayerTable& tab, uint32_t block)
+{
+    int lo = 0, hi = tab.entries; // first_block[lo] <= block < first_block[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (tab.first_block[mid] <= block) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+// Copy a layer's parameters from device memory into `sdev` (shared memory); all threads of the
+// block call this, it ends with a block barrier.
+__device__ __forceinline__ void load_layer_params(const Dev* src, Dev* sdev)
+{
+    const uint32_t* s = reinterpret_cast<const uint32_t*>(src);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(sdev);
+    for (unsigned i = threadIdx.x; i < sizeof(Dev) / 4; i += blockDim.x) dst[i] = s[i];
+    __syncthreads();
+}
+// advance the state arrays to a layer's first coordinate
+__device__ __forceinline__ void shift_arrays(StepArgs& a, int64_t o)
+{
+    a.X += o;
+    a.Xhat += o;
+    a.S += o;
+    if (a.G) a.G += o;
+    if (a.M) a.M += o;
+}
+
 __device__ __forceinline__ uint32_t abs_key(float v)
 {
     return __float_as_uint(v) & 0x7FFFFFFFu;

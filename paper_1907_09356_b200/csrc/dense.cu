@@ -66,9 +66,8 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(Dev dv, StepArgs
 // Finish the tree over a row's partial sums.  MODE L1: scale = root / d (sign).
 // MODE L2SQ: norm = sqrt(root) (QSGD with one block per row).
 template <int MODE>
-__global__ void __launch_bounds__(1024) norm_finish_kernel(Dev dv)
+__device__ __forceinline__ void norm_finish_row(const Dev& dv, int row)
 {
-    const int row = blockIdx.x;
     float* src = dv.partial + (int64_t)row * dv.nchunks;
     float* dst = dv.partial2 + (int64_t)row * dv.nchunks;
     int64_t m = dv.nchunks;
@@ -85,6 +84,24 @@ __global__ void __launch_bounds__(1024) norm_finish_kernel(Dev dv)
         if (MODE == NORM_L1) dv.msg_scale[row] = __fdiv_rn(src[0], (float)dv.d);
         else dv.msg_norms[(int64_t)row * dv.npitch] = __fsqrt_rn(src[0]);
     }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(1024) norm_finish_kernel(Dev dv)
+{
+    norm_finish_row<MODE>(dv, (int)blockIdx.x);
+}
+
+// several layers in one launch (scaled sign: the scale of the NEXT message, whose partial sums
+// the update kernel left): block b serves row b % n of the table's entry b / n
+__global__ void __launch_bounds__(1024) sign_scale_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, int n)
+{
+    __shared__ Dev sdev;
+    const int en = (int)(blockIdx.x / (unsigned)n), row = (int)(blockIdx.x % (unsigned)n);
+    load_layer_params(ls.devs + tab.layer[en], &sdev);
+    if (threadIdx.x == 0) sdev.msg_scale = sdev.nxt_scale;
+    __syncthreads();
+    norm_finish_row<NORM_L1>(sdev, row);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -237,6 +254,12 @@ cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st)
     Dev dn = dv;
     dn.msg_scale = dv.nxt_scale;
     norm_finish_kernel<NORM_L1><<<dv.n, 1024, 0, st>>>(dn);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sign_scale_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, cudaStream_t st)
+{
+    sign_scale_layers_kernel<<<(unsigned)(tab.entries * n), 1024, 0, st>>>(tab, ls, n);
     return cudaGetLastError();
 }
 

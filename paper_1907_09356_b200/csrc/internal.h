@@ -144,6 +144,23 @@ struct StepArgs {
     unsigned long long* launches; // host counter of kernels enqueued (not used on the device)
 };
 
+// One launch over the tiles (or rows) of several layers of a layered context.  The table comes
+// as a kernel argument (constant memory): a block finds its entry by bisection over first_block
+// (launches over tiles) or as blockIdx.x / n (launches over rows) and can request its tiles at
+// once; the rest of the layer's parameters it reads from devs[layer[entry]] in device memory.
+constexpr int kMaxComboLayers = 512;
+struct LayerTable {
+    int32_t entries;                            // layers served by this launch
+    uint32_t first_block[kMaxComboLayers + 1];  // blocks (of a row) before each entry's, then the total
+    int32_t layer[kMaxComboLayers];             // the layer an entry stands for
+    int32_t d[kMaxComboLayers];                 // its length
+    int64_t off[kMaxComboLayers];               // its first coordinate
+};
+struct LayerSet {
+    const Dev* devs;      // per layer, device memory: the layer's parameters for this step
+    int64_t ld;           // row pitch of the state arrays
+};
+
 #ifdef __CUDACC__
 // The step number that keys the generator.  A context may keep it in device memory (and bump it
 // there after every step) so that a captured launch sequence stays valid from step to step.
@@ -172,6 +189,15 @@ cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit
 // sign: finish the tree over the partial sums the update kernel left and set nxt_scale
 cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st);
 cudaError_t launch_apply(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st);
+// the same kernels over several layers at once (see LayerTable): every layer of a launch shares
+// kind, level width, block of the norm, row count n and alignment class
+cudaError_t launch_update_dense_bulk_layers(const Dev& proto, const LayerTable& tab, const LayerSet& ls, const StepArgs& a,
+                                            bool aligned, cudaStream_t st);
+cudaError_t launch_sign_scale_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, cudaStream_t st);
+cudaError_t launch_update_bulk_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, const StepArgs& a, bool aligned,
+                                      cudaStream_t st);
+cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes,
+                                      const StepArgs& a, cudaStream_t st);
 // metrics
 cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,
                              int64_t nblocks, double* out, cudaStream_t st);
@@ -223,6 +249,7 @@ struct choco_ctx {
     struct DenseBuf { uint32_t* bits; float* scale; float* norms; uint8_t* levels; float* dense; } dbuf[2];
     int msg_cur, msg_last;
     bool timed_out;              // a synchronising call saw device_timeouts != 0: steps refuse
+    uint64_t dv_epoch;           // bumped whenever a setter changes `dv` (a layered context keeps device copies)
     bool hot_l2;                 // the context asked for persisting L2 lines (reset on destroy)
     // host staging for choco_sgd_step_host
     float* stage[4];

@@ -741,6 +741,24 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     emit_row_single<KIND, VEC>(dv, a, (int)blockIdx.x, fused, rescue, dyn, h, sm, s_carry);
 }
 
+// several layers in one launch: block b serves row b % n of the table's entry b / n (top-k, one
+// block per row; rows may start at any element, so the exact selection reads them element by element)
+__global__ void __launch_bounds__(kSelThreads)
+emit_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs a, int n)
+{
+    extern __shared__ __align__(16) uint32_t dyn[];
+    __shared__ uint32_t h[kHistBins];
+    __shared__ uint32_t sm[64];
+    __shared__ uint32_t s_carry[2];
+    __shared__ Dev sdev;
+    const int en = (int)(blockIdx.x / (unsigned)n), row = (int)(blockIdx.x % (unsigned)n);
+    load_layer_params(ls.devs + tab.layer[en], &sdev); // (set up by the host: not the previous kernel's output)
+    shift_arrays(a, tab.off[en]);
+    wait_for_previous_kernel(); // the candidates come from the kernel before this one
+    allow_next_kernel();
+    emit_row_single<SEL_TOPK, false>(sdev, a, row, 1, 0, dyn, h, sm, s_carry);
+}
+
 // ---------------------------------------------------------------------------------------
 // emit, several blocks per row: a thread-block cluster serves one row.
 //
@@ -1173,6 +1191,22 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int r
     if (e != cudaSuccess) return e;
     *a.launches += 1;
     return cudaGetLastError();
+}
+
+cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes,
+                                      const StepArgs& a, cudaStream_t st)
+{
+    static size_t configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || configured[dev] < smem_bytes) {
+        e = cudaFuncSetAttribute(emit_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = smem_bytes;
+    }
+    return launch_overlapped(emit_layers_kernel, dim3((unsigned)(tab.entries * n)), dim3(kSelThreads), smem_bytes, st,
+                             HotRange{nullptr, 0, 0.f}, tab, ls, a, (int)n);
 }
 
 cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)

@@ -74,11 +74,15 @@ constexpr size_t bulk_smem_bytes()
 // element offset of p inside its 16-byte unit
 __device__ __forceinline__ uint32_t unit_shift(const float* p) { return (uint32_t)(((uintptr_t)p & 15u) >> 2); }
 
-template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
-__global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepArgs a)
+// tile: the block's tile of the row; row: the worker; d, ld: dv.d and dv.ld.  With LAYERS `dv` is
+// the block's shared-memory copy of its layer's parameters, still to be filled from `dv_src`: the
+// tiles are requested first (that needs d, ld and the array pointers only), the copy is made
+// while they fly.
+template <bool HAS_G, bool HAS_M, bool EMIT, bool AL, bool LAYERS>
+__device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const StepArgs& a, int64_t tile, int row, int64_t d,
+                                                        int64_t ld, unsigned char* smem_raw, const Dev* dv_src)
 {
     static_assert(NT >= kTile / 32 && NT >= kMaxNb, "one thread per mask word / neighbour");
-    extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int kStage = kTile + (AL ? 0 : kShiftPad);
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* hs = xs + kStage;
@@ -93,18 +97,15 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     uint32_t* s_base = reinterpret_cast<uint32_t*>(scan) + 2 * (NT / 32 + 1);
     NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
 
-    const int row = blockIdx.y;
-    const int64_t tile = blockIdx.x;
     const int64_t c0 = tile * kTile;
-    const int nvalid = (int)((dv.d - c0) < kTile ? (dv.d - c0) : kTile); // AL: a multiple of 4
+    const int nvalid = (int)((d - c0) < kTile ? (d - c0) : kTile); // AL: a multiple of 4
     const int lane = threadIdx.x & 31;
-    float* xr = a.X + (int64_t)row * dv.ld + c0;
-    float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
-    float* sr = a.S + (int64_t)row * dv.ld + c0;
-    const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
+    float* xr = a.X + (int64_t)row * ld + c0;
+    float* hr = a.Xhat + (int64_t)row * ld + c0;
+    float* sr = a.S + (int64_t)row * ld + c0;
 
-    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld + c0 : nullptr;
-    float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
+    const float* gr = HAS_G ? a.G + (int64_t)row * ld + c0 : nullptr;
+    float* mrow = HAS_M ? a.M + (int64_t)row * ld + c0 : nullptr;
     // where each staged tile's first element sits in its shared-memory buffer
     const uint32_t shx = AL ? 0u : unit_shift(xr), shh = AL ? 0u : unit_shift(hr), shs = AL ? 0u : unit_shift(sr);
     const uint32_t shg = (AL || !HAS_G) ? 0u : unit_shift(gr), shm = (AL || !HAS_M) ? 0u : unit_shift(mrow);
@@ -123,6 +124,8 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (threadIdx.x < kTile / 32) { touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; }
+    if (LAYERS) load_layer_params(dv_src, const_cast<Dev*>(&dv));
+    const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
     // Messages, range records and the candidate bound come from the kernel before this one.
     // The dense arrays requested above do not: the kernel before either ran to completion
     // before this one started, or is the emit kernel, which lets its successor start only
@@ -330,6 +333,55 @@ __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepA
 }
 
 template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
+__global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    update_sparse_bulk_body<HAS_G, HAS_M, EMIT, AL, false>(dv, a, (int64_t)blockIdx.x, (int)blockIdx.y, dv.d, dv.ld, smem_raw,
+                                                          nullptr);
+}
+
+// several layers in one launch: blockIdx.x picks (layer, tile), blockIdx.y the worker
+template <bool HAS_G, bool HAS_M, bool AL>
+__global__ void __launch_bounds__(NT, 5)
+update_sparse_bulk_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ Dev sdev;
+    const int en = entry_of_block(tab, blockIdx.x);
+    shift_arrays(a, tab.off[en]);
+    update_sparse_bulk_body<HAS_G, HAS_M, true, AL, true>(sdev, a, (int64_t)(blockIdx.x - tab.first_block[en]), (int)blockIdx.y,
+                                                         (int64_t)tab.d[en], ls.ld, smem_raw, ls.devs + tab.layer[en]);
+}
+
+template <bool HAS_G, bool HAS_M, bool AL>
+cudaError_t launch_bulk_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, const StepArgs& a, cudaStream_t st)
+{
+    constexpr size_t smem = bulk_smem_bytes<HAS_G, HAS_M, AL>();
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    auto kern = update_sparse_bulk_layers_kernel<HAS_G, HAS_M, AL>;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    return launch_overlapped(kern, dim3(tab.first_block[tab.entries], (unsigned)n), dim3(NT), smem, st,
+                             HotRange{nullptr, 0, 0.f}, tab, ls, a);
+}
+
+template <bool AL>
+cudaError_t launch_terms_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, const StepArgs& a, cudaStream_t st)
+{
+    if (a.M) return launch_bulk_layers<true, true, AL>(tab, ls, n, a, st);
+    if (a.G) return launch_bulk_layers<true, false, AL>(tab, ls, n, a, st);
+    return launch_bulk_layers<false, false, AL>(tab, ls, n, a, st);
+}
+
+template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
     constexpr size_t smem = bulk_smem_bytes<HAS_G, HAS_M, AL>();
@@ -362,6 +414,12 @@ cudaError_t launch_terms(const Dev& dv, const StepArgs& a, bool emit, cudaStream
 }
 
 } // namespace
+
+cudaError_t launch_update_bulk_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, const StepArgs& a, bool aligned,
+                                      cudaStream_t st)
+{
+    return aligned ? launch_terms_layers<true>(tab, ls, n, a, st) : launch_terms_layers<false>(tab, ls, n, a, st);
+}
 
 cudaError_t launch_update_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)
 {

@@ -145,12 +145,17 @@ __device__ __forceinline__ void store_some(float* p, const float4& v, int left)
     if (left > 3) p[3] = v.w;
 }
 
-template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
-__global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
+// bx: the block's tile of the row; row: the worker; d, ld: dv.d and dv.ld; nbk: blocks of the
+// norm per tile (1 for sign).  With LAYERS `dv` is the block's shared-memory copy of its layer's
+// parameters, still to be filled from `dv_src`: the tiles are requested first (that needs d, ld
+// and the array pointers only), the copy is made while they fly.
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL, bool LAYERS>
+__device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const StepArgs& a, int nb_stage, int nbk, int64_t bx,
+                                                       int row, int64_t d, int64_t ld, unsigned char* smem_raw,
+                                                       const Dev* dv_src)
 {
     using L = Layout<WBITS, HAS_G, HAS_M>;
     static_assert((KIND == CHOCO_Q_SIGN) == (WBITS == 0), "sign has no level fields");
-    extern __shared__ __align__(128) unsigned char smem_raw[];
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* hs = xs + L::kStage;
     float* ss = hs + L::kStage;
@@ -158,25 +163,21 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     float* ms = gs + (HAS_G ? L::kStage : 0);       // used when HAS_M
     unsigned char* msg_in = smem_raw + L::msg_in();
     unsigned char* msg_out = smem_raw + L::msg_out(nb_stage);
-    // blocks of the norm per tile (gsgd_b); one "block" for sign
-    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
     float* tab = reinterpret_cast<float*>(smem_raw + L::tables(nb_stage));
     float* tab_self = tab + nb_stage * nbk * kTabLevels;
     float* ws = reinterpret_cast<float*>(smem_raw + L::misc(nb_stage, nbk)); // [NIT][8] warp sums
     double* rnu = reinterpret_cast<double*>(ws + NIT * 8);                   // [16] 1 / nu per block of the norm
     uint64_t* bar = reinterpret_cast<uint64_t*>(rnu + 16);
 
-    const int row = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t c0 = (int64_t)blockIdx.x * kDTile;
-    const int nvalid = (int)((dv.d - c0) < kDTile ? (dv.d - c0) : kDTile); // AL: a multiple of 4
-    const int e0 = dv.row_ptr[row], deg = dv.row_ptr[row + 1] - e0;
+    const int64_t c0 = bx * kDTile;
+    const int nvalid = (int)((d - c0) < kDTile ? (d - c0) : kDTile); // AL: a multiple of 4
     const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
-    float* xr = a.X + (int64_t)row * dv.ld + c0;
-    float* hr = a.Xhat + (int64_t)row * dv.ld + c0;
-    float* sr = a.S + (int64_t)row * dv.ld + c0;
-    float* mrow = HAS_M ? a.M + (int64_t)row * dv.ld + c0 : nullptr;
-    const float* gr = HAS_G ? a.G + (int64_t)row * dv.ld + c0 : nullptr;
+    float* xr = a.X + (int64_t)row * ld + c0;
+    float* hr = a.Xhat + (int64_t)row * ld + c0;
+    float* sr = a.S + (int64_t)row * ld + c0;
+    float* mrow = HAS_M ? a.M + (int64_t)row * ld + c0 : nullptr;
+    const float* gr = HAS_G ? a.G + (int64_t)row * ld + c0 : nullptr;
     // where each staged tile's first element sits in its shared-memory buffer
     const uint32_t shx = AL ? 0u : unit_shift(xr), shh = AL ? 0u : unit_shift(hr), shs = AL ? 0u : unit_shift(sr);
     const uint32_t shg = (AL || !HAS_G) ? 0u : unit_shift(gr), shm = (AL || !HAS_M) ? 0u : unit_shift(mrow);
@@ -187,9 +188,28 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     const uint32_t bits_bytes = ((((uint32_t)nvalid + 31u) >> 5) * 4u + 15u) & ~15u;
     const uint32_t lev_bytes = (((uint32_t)nvalid * WBITS + 7u) / 8u + 15u) & ~15u;
     const uint32_t msg_bytes = bits_bytes + (WBITS > 0 ? lev_bytes : 0u);
-    const int64_t bits_off = (int64_t)blockIdx.x * (kDTile / 32);            // words into a row's sign plane
-    const int64_t lev_off = (int64_t)blockIdx.x * L::kLevTile;               // bytes into a row's level fields
+    const int64_t bits_off = bx * (kDTile / 32);            // words into a row's sign plane
+    const int64_t lev_off = bx * L::kLevTile;               // bytes into a row's level fields
 
+    // The barrier takes one arrival per phase, or two with LAYERS, where the tiles are requested
+    // before the layer's parameters (and with them the neighbours) are known.
+    const uint32_t dense_tx = span(shx) + span(shh) + span(shs) + (HAS_G ? span(shg) : 0u) + (HAS_M ? span(shm) : 0u);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, LAYERS ? 2 : 1);
+        if (LAYERS) mbar_expect_tx(bar, dense_tx);
+    }
+    auto request_tiles = [&]() {
+        bulk_load(xs, xr - shx, span(shx), bar);
+        bulk_load(hs, hr - shh, span(shh), bar);
+        bulk_load(ss, sr - shs, span(shs), bar);
+        if (HAS_G) bulk_load(gs, gr - shg, span(shg), bar);
+        if (HAS_M) bulk_load(ms, mrow - shm, span(shm), bar);
+    };
+    if (LAYERS) {
+        if (threadIdx.x == 0) request_tiles();
+        load_layer_params(dv_src, const_cast<Dev*>(&dv));
+    }
+    const int e0 = dv.row_ptr[row], deg = dv.row_ptr[row + 1] - e0;
     // stage the message slices of neighbours [first, first + count): lane r of warp 0 issues r's copies
     auto stage_messages = [&](int first, int count) {
         if (lane < count) {
@@ -202,14 +222,8 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     if (warp == 0) {
         const int count = deg < nb_stage ? deg : nb_stage;
         if (lane == 0) {
-            mbar_init(bar, 1);
-            mbar_expect_tx(bar, span(shx) + span(shh) + span(shs) + (HAS_G ? span(shg) : 0u) + (HAS_M ? span(shm) : 0u) +
-                                    (uint32_t)count * msg_bytes);
-            bulk_load(xs, xr - shx, span(shx), bar);
-            bulk_load(hs, hr - shh, span(shh), bar);
-            bulk_load(ss, sr - shs, span(shs), bar);
-            if (HAS_G) bulk_load(gs, gr - shg, span(shg), bar);
-            if (HAS_M) bulk_load(ms, mrow - shm, span(shm), bar);
+            mbar_expect_tx(bar, (LAYERS ? 0u : dense_tx) + (uint32_t)count * msg_bytes);
+            if (!LAYERS) request_tiles();
         }
         __syncwarp();
         stage_messages(0, count);
@@ -228,7 +242,10 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
             fence_before_bulk_copy();
             __syncthreads();
             if (warp == 0) {
-                if (lane == 0) mbar_expect_tx(bar, (uint32_t)count * msg_bytes);
+                if (lane == 0) {
+                    mbar_expect_tx(bar, (uint32_t)count * msg_bytes);
+                    if (LAYERS) mbar_arrive(bar); // the phase's second arrival
+                }
                 __syncwarp();
                 stage_messages(first, count);
             }
@@ -400,7 +417,7 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
     if (KIND == CHOCO_Q_SIGN) {
         // per-1024 partial sums of |v|; a small kernel finishes the tree and the scale
         if (threadIdx.x < NIT) {
-            const int64_t chunk = (int64_t)blockIdx.x * NIT + threadIdx.x;
+            const int64_t chunk = bx * NIT + threadIdx.x;
             if (chunk < dv.nchunks) dv.partial[(int64_t)row * dv.nchunks + chunk] = tree8(ws + threadIdx.x * 8);
         }
         if (storer) bulk_store_commit_and_drain();
@@ -468,16 +485,33 @@ __global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepAr
 }
 
 template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
-cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
+__global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
 {
-    using L = Layout<WBITS, HAS_G, HAS_M>;
-    const int nb_stage = dv.maxdeg < kBatch ? dv.maxdeg : kBatch;
-    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
-    const size_t smem = (size_t)L::total(nb_stage, nbk);
-    auto kern = update_dense_bulk_kernel<KIND, WBITS, HAS_G, HAS_M, EMIT, AL>;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1; // blocks of the norm per tile
+    update_dense_bulk_body<KIND, WBITS, HAS_G, HAS_M, EMIT, AL, false>(dv, a, nb_stage, nbk, (int64_t)blockIdx.x,
+                                                                      (int)blockIdx.y, dv.d, dv.ld, smem_raw, nullptr);
+}
+
+// several layers in one launch: blockIdx.x picks (layer, tile), blockIdx.y the worker
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool AL>
+__global__ void __launch_bounds__(NT, 4)
+update_dense_bulk_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs a, int nb_stage, int nbk)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ Dev sdev;
+    const int en = entry_of_block(tab, blockIdx.x);
+    shift_arrays(a, tab.off[en]);
+    update_dense_bulk_body<KIND, WBITS, HAS_G, HAS_M, true, AL, true>(
+        sdev, a, nb_stage, nbk, (int64_t)(blockIdx.x - tab.first_block[en]), (int)blockIdx.y, (int64_t)tab.d[en], ls.ld,
+        smem_raw, ls.devs + tab.layer[en]);
+}
+
+template <typename K>
+cudaError_t allow_shared_memory(K kern, size_t smem, size_t* configured)
+{
     // Once per device, instantiation and size: allow the dynamic shared memory and ask for the
     // largest shared-memory carve-out, so that as many tiles as possible are in flight per SM.
-    static size_t configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -488,6 +522,55 @@ cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = smem;
     }
+    return cudaSuccess;
+}
+
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool AL>
+cudaError_t launch_layers_one(const Dev& proto, const LayerTable& tab, const LayerSet& ls, const StepArgs& a, cudaStream_t st)
+{
+    using L = Layout<WBITS, HAS_G, HAS_M>;
+    const int nb_stage = proto.maxdeg < kBatch ? proto.maxdeg : kBatch;
+    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> proto.bucket_shift) : 1;
+    const size_t smem = (size_t)L::total(nb_stage, nbk);
+    auto kern = update_dense_bulk_layers_kernel<KIND, WBITS, HAS_G, HAS_M, AL>;
+    static size_t configured[64] = {};
+    const cudaError_t e = allow_shared_memory(kern, smem, configured);
+    if (e != cudaSuccess) return e;
+    kern<<<dim3(tab.first_block[tab.entries], (unsigned)proto.n), NT, smem, st>>>(tab, ls, a, nb_stage, nbk);
+    return cudaGetLastError();
+}
+
+template <int KIND, int WBITS, bool AL>
+cudaError_t launch_layers_terms(const Dev& proto, const LayerTable& tab, const LayerSet& ls, const StepArgs& a, cudaStream_t st)
+{
+    if (a.M) return launch_layers_one<KIND, WBITS, true, true, AL>(proto, tab, ls, a, st);
+    if (a.G) return launch_layers_one<KIND, WBITS, true, false, AL>(proto, tab, ls, a, st);
+    return launch_layers_one<KIND, WBITS, false, false, AL>(proto, tab, ls, a, st);
+}
+
+template <bool AL>
+cudaError_t launch_layers_kind(const Dev& proto, const LayerTable& tab, const LayerSet& ls, const StepArgs& a, cudaStream_t st)
+{
+    if (proto.kind == CHOCO_Q_SIGN) return launch_layers_terms<CHOCO_Q_SIGN, 0, AL>(proto, tab, ls, a, st);
+    switch (proto.wbits) {
+    case 1: return launch_layers_terms<CHOCO_Q_QSGD, 1, AL>(proto, tab, ls, a, st);
+    case 2: return launch_layers_terms<CHOCO_Q_QSGD, 2, AL>(proto, tab, ls, a, st);
+    case 4: return launch_layers_terms<CHOCO_Q_QSGD, 4, AL>(proto, tab, ls, a, st);
+    default: return launch_layers_terms<CHOCO_Q_QSGD, 8, AL>(proto, tab, ls, a, st);
+    }
+}
+
+template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
+cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
+{
+    using L = Layout<WBITS, HAS_G, HAS_M>;
+    const int nb_stage = dv.maxdeg < kBatch ? dv.maxdeg : kBatch;
+    const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
+    const size_t smem = (size_t)L::total(nb_stage, nbk);
+    auto kern = update_dense_bulk_kernel<KIND, WBITS, HAS_G, HAS_M, EMIT, AL>;
+    static size_t configured[64] = {};
+    const cudaError_t e = allow_shared_memory(kern, smem, configured);
+    if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)((dv.d + kDTile - 1) / kDTile), (unsigned)dv.n);
     kern<<<grid, NT, smem, st>>>(dv, a, nb_stage);
     return cudaGetLastError();
@@ -522,6 +605,12 @@ bool update_dense_bulk_usable(const Dev& dv, const StepArgs& a)
     // at an odd element go to the register kernel
     auto even = [](const void* p) { return ((uintptr_t)p & 7u) == 0; };
     return dv.ld % 2 == 0 && even(a.X) && even(a.Xhat) && even(a.S) && even(a.G) && even(a.M);
+}
+
+cudaError_t launch_update_dense_bulk_layers(const Dev& proto, const LayerTable& tab, const LayerSet& ls, const StepArgs& a,
+                                            bool aligned, cudaStream_t st)
+{
+    return aligned ? launch_layers_kind<true>(proto, tab, ls, a, st) : launch_layers_kind<false>(proto, tab, ls, a, st);
 }
 
 cudaError_t launch_update_dense_bulk(const Dev& dv, const StepArgs& a, bool emit, cudaStream_t st)

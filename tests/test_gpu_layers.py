@@ -93,7 +93,9 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
             for l in range(len(sizes)):
                 ctx, _, _ = choco.choco_layers_get_layer(h, l)
                 assert choco.choco_get_stats(ctx)["device_timeouts"] == 0
-            return choco.choco_layers_set_graphs(h)
+            # steps served without a launch per layer: replayed from a graph, or enqueued as
+            # launches over all layers at once
+            return choco.choco_layers_set_graphs(h) + choco.choco_layers_combined_steps(h)
     finally:
         choco.choco_layers_destroy(h)
 
@@ -132,6 +134,20 @@ def test_replayed_steps_of_operators_keyed_by_the_step_number(kind, kw):
     replays = _run(workloads.torus(2, 4), RAGGED, kind, kw, steps=14, stream=torch.cuda.Stream(), g_pool=2,
                    check_layers=(0, 2, 3), invalidate_at=6, jump=(4, 1000))
     assert replays >= 3
+
+
+@pytest.mark.parametrize("kind,kw", [KINDS[0], KINDS[2], KINDS[3]], ids=["topk", "sign", "qsgd512"])
+def test_steady_steps_are_launches_over_all_layers(kind, kw):
+    """After the first step every step of these operators is enqueued as two or three launches
+    whose blocks find their layer in a table, on any stream (here the default one), layers at
+    every alignment included; an invalidation sends one step back to the layer-by-layer path."""
+    combined = _run(workloads.torus(2, 4), RAGGED, kind, kw, steps=9, check_layers=range(len(RAGGED)),
+                    invalidate_at=5)
+    assert combined == 9 - 2
+    combined = _run(workloads.ring(4), RAGGED, kind, kw, steps=6, momentum=True, ld=sum(RAGGED) + 4)
+    assert combined == 6 - 1
+    combined = _run(workloads.ring(4), [4096, 8192, 2048 * 3], kind, kw, steps=5, gossip_only=True)   # all aligned
+    assert combined == 5 - 1
 
 
 def test_gossip_only_layers():
