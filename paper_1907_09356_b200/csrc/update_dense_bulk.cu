@@ -485,7 +485,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
 }
 
 template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool EMIT, bool AL>
-__global__ void __launch_bounds__(NT, 4) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
+__global__ void __launch_bounds__(NT, 5) update_dense_bulk_kernel(Dev dv, StepArgs a, int nb_stage)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1; // blocks of the norm per tile

@@ -19,6 +19,9 @@ Runs (Algorithm 1 in the three-vector form, oracle.step):
   c3_ring8_sign      8-ring, d = 272 474, scaled sign, gradient pool of 8, 1000 steps
   c4_torus64_topk    8x8 torus, d = 1e6, top-1 %, gradient pool of 8, 500 steps, gamma = 0.2
   c4_torus64_topk_g004   the same at gamma = 0.04 (stable range; Table 4 lists 0.0375 for top-1 %)
+  c4_torus64_topk_mom    the same with Algorithm 2 (momentum 0.9, weight decay 1e-4); M is check-summed too
+  c6_social32_sign / c6_social32_topk   irregular 32-node graph (up to 15 messages per row), d = 272 474,
+                     scaled sign / top-1 %, 1000 steps each
 The d = 1e6 runs take about a quarter of an hour each on eight host threads.
 """
 from __future__ import annotations
@@ -44,7 +47,7 @@ CHECKPOINTS = (1, 2, 5, 10, 50, 100, 200, 500, 1000, 2000)
 POOL = 8                      # gradient tensors cycled through (step t uses tensor t mod POOL)
 SEED_X, SEED_G, SEED_Q, SEED_PROBLEM = 40, 4100, 9, 3
 RUNS = ("c1_ring4_topk", "c2_ring16_randk", "c2_ring16_randk_g006", "c2_ring16_qsgd", "c3_ring8_sign",
-        "c4_torus64_topk", "c4_torus64_topk_g004")
+        "c4_torus64_topk", "c4_torus64_topk_g004", "c4_torus64_topk_mom", "c6_social32_sign", "c6_social32_topk")
 
 
 def _fp(a):
@@ -58,8 +61,10 @@ def run(name: str, executor) -> dict:
     X = (workloads.normal_rows(wl.n, wl.d, wl.x_var, SEED_X) if wl.x_var > 0
          else np.zeros((wl.n, wl.d), dtype=np.float32))
     Xh, S = np.zeros_like(X), np.zeros_like(X)
+    M = np.zeros_like(X) if wl.momentum > 0 else None
     rec = {"workload": name, "n": wl.n, "d": wl.d, "graph": wl.graph, "Q": wl.q, "k": wl.k, "s": wl.s,
            "bucket": wl.bucket, "eta": wl.eta, "gamma": wl.gamma, "steps": wl.steps,
+           "momentum": wl.momentum, "weight_decay": wl.weight_decay,
            "seeds": {"x": SEED_X, "g": SEED_G, "q": SEED_Q, "problem": SEED_PROBLEM},
            "inputs": {"X0": _fp(X)}, "checkpoints": []}
     problem, pool = None, None
@@ -80,11 +85,14 @@ def run(name: str, executor) -> dict:
             grad_sum = (grad_sum + workloads.fingerprint(G)[0]) % (1 << 64)
         else:
             G = pool[t % POOL] if pool is not None else None
-        oracle.step(w, p, X, Xh, S, G, wl.eta if G is not None else 0.0, wl.gamma, t, executor=executor)
+        oracle.step(w, p, X, Xh, S, G, wl.eta if G is not None else 0.0, wl.gamma, t, executor=executor,
+                    M=M, lam=wl.weight_decay, beta=wl.momentum)
         if t + 1 in CHECKPOINTS or t + 1 == wl.steps:
             e = oracle.consensus_error(X)
             cp = {"step": t + 1, "consensus": e, "relative": (e / e0 if e0 > 0 else None),
                   "max_abs_x": float(np.max(np.abs(X))), "X": _fp(X), "Xhat": _fp(Xh), "S": _fp(S)}
+            if M is not None:
+                cp["M"] = _fp(M)
             if problem is not None:
                 # the gradients follow X, so this running sum shows whether they were the same
                 cp["gradients_so_far"] = f"{grad_sum:016x}"

@@ -50,12 +50,14 @@ def test_device_fingerprint_is_the_host_one():
     assert device_fingerprint(torch.from_numpy(a).to(DEV)) == want
 
 
-@pytest.mark.parametrize("name", ["c1_ring4_topk", "c3_ring8_sign", "c4_torus64_topk", "c4_torus64_topk_g004"])
+@pytest.mark.parametrize("name", ["c1_ring4_topk", "c3_ring8_sign", "c4_torus64_topk", "c4_torus64_topk_g004",
+                                  "c4_torus64_topk_mom", "c6_social32_sign", "c6_social32_topk"])
 def test_full_run_against_stored_oracle_run(name):
     gold = _runs()[name]
     wl = workloads.WORKLOADS[name]
     assert (wl.n, wl.d, wl.k, wl.gamma, wl.eta, wl.steps) == (gold["n"], gold["d"], gold["k"], gold["gamma"],
                                                                gold["eta"], gold["steps"])
+    assert (wl.momentum, wl.weight_decay) == (gold.get("momentum", 0.0), gold.get("weight_decay", 0.0))
     seeds = gold["seeds"]
     w = wl.mixing()
     X0 = workloads.normal_rows(wl.n, wl.d, wl.x_var, seeds["x"])
@@ -64,6 +66,7 @@ def test_full_run_against_stored_oracle_run(name):
     e0 = oracle.consensus_error(X0) if wl.d <= 4096 else None
     del X0
     dXh, dS = torch.zeros_like(dX), torch.zeros_like(dX)
+    dM = torch.zeros_like(dX) if wl.momentum > 0 else None     # Algorithm 2
     pool = None
     if wl.sgd:
         pool = []
@@ -79,7 +82,9 @@ def test_full_run_against_stored_oracle_run(name):
         cps = {c["step"]: c for c in gold["checkpoints"]}
         assert max(cps) == wl.steps
         for t in range(wl.steps):
-            if pool is not None:
+            if dM is not None:
+                ch.sgd_momentum_step(dX, dXh, dS, pool[t % POOL], dM, wl.eta, wl.gamma, wl.weight_decay, wl.momentum)
+            elif pool is not None:
                 ch.sgd_step(dX, dXh, dS, pool[t % POOL], wl.eta, wl.gamma)
             else:
                 ch.gossip_step(dX, dXh, dS, wl.gamma)
@@ -89,7 +94,7 @@ def test_full_run_against_stored_oracle_run(name):
             rel = choco.choco_consensus_error(ch.ctx, dX) / gold["e0"]
             assert abs(rel - c["relative"]) <= 1e-4 * c["relative"], f"consensus distance after step {t + 1}"
             if same_inputs:
-                for arr, key in ((dX, "X"), (dXh, "Xhat"), (dS, "S")):
+                for arr, key in ((dX, "X"), (dXh, "Xhat"), (dS, "S")) + (((dM, "M"),) if dM is not None else ()):
                     assert device_fingerprint(arr) == c[key], f"{key} after step {t + 1} differs from the oracle's"
         st = choco.choco_get_stats(ch.ctx)
         assert st["device_timeouts"] == 0

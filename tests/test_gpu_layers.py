@@ -150,6 +150,15 @@ def test_steady_steps_are_launches_over_all_layers(kind, kw):
     assert combined == 5 - 1
 
 
+@pytest.mark.parametrize("kind,kw", [KINDS[0], KINDS[2], KINDS[3]], ids=["topk", "sign", "qsgd512"])
+def test_resnet20_layers_for_thirty_steps(kind, kw):
+    """The 65 ResNet-20 tensors on an 8-ring beside the oracle for 30 steps: all but the first
+    step run as the launches over all layers."""
+    sizes = workloads.resnet20_layer_sizes()
+    combined = _run(workloads.ring(8), sizes, kind, dict(kw, a=(1, 100)), steps=30, check_layers=(0, 3, 64))
+    assert combined == 29
+
+
 def test_gossip_only_layers():
     _run(workloads.ring(4), RAGGED, "topk", dict(a=(1, 10)), steps=5, gossip_only=True)
 
