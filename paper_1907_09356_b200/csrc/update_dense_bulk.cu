@@ -289,13 +289,14 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
         if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
         (void)mbar_wait_bounded(bar, parity, dv.stats, kSpinLimit);
 
+        // neighbours in CSR order (outer loop), this thread's two quads inside
+        for (int r = 0; r < count; ++r) {
+            const unsigned char* slice = msg_in + r * L::kMsgTile;
+            const bool self = r == self_r;
 #pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int q4 = it * NT + threadIdx.x;
-            const int li = q4 * kQuad;
-            const int b = KIND == CHOCO_Q_QSGD ? (li >> dv.bucket_shift) : 0; // the same for the whole warp
-            for (int r = 0; r < count; ++r) {
-                const unsigned char* slice = msg_in + r * L::kMsgTile;
+            for (int it = 0; it < NIT; ++it) {
+                const int q4 = it * NT + threadIdx.x;
+                const int li = q4 * kQuad;
                 const uint32_t word = reinterpret_cast<const uint32_t*>(slice)[li >> 5];
                 const uint32_t nib = (word >> (li & 31)) & 0xFu;
                 float q[4];
@@ -303,12 +304,13 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
                     const float m = tab[r];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) q[e] = with_sign(m, nib, e);
-                    if (r == self_r) {
+                    if (self) {
                         const float sc = tab_self[0];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(sc, nib, e);
                     }
                 } else {
+                    const int b = li >> dv.bucket_shift; // block of the norm: the same for the whole warp
                     const unsigned char* lev = slice + L::kBitsTile;
                     uint32_t packed;
                     if (WBITS == 8) packed = reinterpret_cast<const uint32_t*>(lev)[q4];
@@ -320,7 +322,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
                     if (L::kTable) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) q[e] = with_sign(t[(packed >> (e * WBITS)) & mask], nib, e);
-                        if (r == self_r) {
+                        if (self) {
                             const float* ts = tab_self + b * kTabLevels;
 #pragma unroll
                             for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(ts[(packed >> (e * WBITS)) & mask], nib, e);
@@ -330,7 +332,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float m = __fmul_rn(mag, small_uint_to_float((packed >> (e * WBITS)) & mask));
-                            if (r == self_r) qs[it][e] = with_sign(m, nib, e);
+                            if (self) qs[it][e] = with_sign(m, nib, e);
                             q[e] = with_sign(__fmul_rn(w, m), nib, e);
                         }
                     }

@@ -13,7 +13,7 @@ from test_gpu_parity import DEV, _dev, _host, assert_state, check_messages
 pytestmark = pytest.mark.gpu
 
 
-def _run(d, ld, k, rescue, burst_steps, steps=9, n=8):
+def _run(d, ld, k, rescue, burst_steps, steps=9, n=8, select_blocks=None):
     """`burst_steps`: steps whose gradient is -50 x / eta, so that x grows 51-fold and nearly
     every coordinate of the next x - x^ exceeds the bound guessed before the burst."""
     w = workloads.torus(2, 4)
@@ -23,6 +23,8 @@ def _run(d, ld, k, rescue, burst_steps, steps=9, n=8):
     p = oracle.Params("topk", k=k)
     ch = choco.Choco(w, d, "topk", k=k, ld=ld)
     choco.choco_set_rescue(ch.ctx, rescue)
+    if select_blocks:
+        choco.choco_set_select_blocks(ch.ctx, select_blocks)
     dX, dXh, dS = _dev(X, ld), _dev(Xh, ld), _dev(S, ld)
     try:
         for t in range(steps):
@@ -50,6 +52,16 @@ def test_bursts_are_rescued(d, ld, k):
     st = _run(d, ld, k, True, burst_steps=(3, 6))
     assert st["rescued_rows"] >= 8, st              # every row of the step after a burst
     off = _run(d, ld, k, False, burst_steps=(3, 6))
+    assert off["rescued_rows"] == 0 and off["exact_rows"] >= 8, off
+
+
+@pytest.mark.parametrize("blocks", [2, 4])
+def test_bursts_with_a_cluster_of_blocks_per_row(blocks):
+    """The same with the selection kernel's cluster form: a row whose candidates are unusable is
+    handed to the rescue kernels (or selected exactly) by the cluster's first block alone."""
+    st = _run(50_000, 50_000, 500, True, burst_steps=(3, 6), select_blocks=blocks)
+    assert st["rescued_rows"] >= 8, st
+    off = _run(40_003, 40_003, 401, False, burst_steps=(3, 6), select_blocks=blocks)
     assert off["rescued_rows"] == 0 and off["exact_rows"] >= 8, off
 
 
