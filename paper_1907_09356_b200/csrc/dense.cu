@@ -259,7 +259,8 @@ cudaError_t launch_next_sign_scale(const Dev& dv, cudaStream_t st)
 
 cudaError_t launch_sign_scale_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, cudaStream_t st)
 {
-    sign_scale_layers_kernel<<<(unsigned)(tab.entries * n), 1024, 0, st>>>(tab, ls, n);
+    // small trees (layers of a launch-bound step): 128 threads each, many blocks per SM
+    sign_scale_layers_kernel<<<(unsigned)(tab.entries * n), 128, 0, st>>>(tab, ls, n);
     return cudaGetLastError();
 }
 

@@ -17,6 +17,7 @@ constexpr int64_t kRescueMinD = (int64_t)1 << 22; // rows this long are rescued 
 constexpr uint32_t kSpinLimit = 1u << 22;   // polls a kernel spends on a wait before it gives up
 
 constexpr int64_t kEmitSmemBudget = 200 * 1024; // dynamic shared memory the emit kernel may use
+constexpr int kSmallRow = 4096;       // rows up to this length are selected by small blocks, several per SM
 constexpr int kHistBins = 2048;       // first radix digit: top 11 bits of the ordering key
 
 struct Stats {
@@ -196,7 +197,8 @@ cudaError_t launch_update_dense_bulk_layers(const Dev& proto, const LayerTable& 
 cudaError_t launch_sign_scale_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, cudaStream_t st);
 cudaError_t launch_update_bulk_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, const StepArgs& a, bool aligned,
                                       cudaStream_t st);
-cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes,
+// `small`: every row of the table is at most kSmallRow long (blocks of kSelThreadsSmall threads)
+cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes, bool small,
                                       const StepArgs& a, cudaStream_t st);
 // metrics
 cudaError_t launch_consensus(const float* X, int32_t n, int64_t d, int64_t ld, double* scratch,

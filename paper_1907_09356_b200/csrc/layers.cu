@@ -77,8 +77,9 @@ struct choco_layers {
     bool groups_valid;
     choco::LayerTable tiles_al, tiles_ua; // layers whose rows are 16-byte aligned / the others the kernels take
     choco::LayerTable rows;               // all of those, for the launches over rows
+    choco::LayerTable rows_small, rows_large; // the same split by row length (top_a: two block sizes)
     std::vector<int32_t> grouped, rest;   // layers served by the combined launches / by their own context
-    size_t emit_smem;
+    size_t emit_smem_small, emit_smem_large;
     uint64_t combined_steps;
     cudaStream_t side[kLayerStreams];
     cudaEvent_t fork;
@@ -96,6 +97,7 @@ namespace {
 void free_groups(choco_layers* L)
 {
     L->tiles_al.entries = L->tiles_ua.entries = L->rows.entries = 0;
+    L->rows_small.entries = L->rows_large.entries = 0;
     L->groups_valid = false;
 }
 
@@ -198,7 +200,7 @@ int make_groups(choco_layers* L, const float* X, const float* Xhat, const float*
     L->grouped.clear();
     L->rest.clear();
     const bool sparse = L->ctx[0]->dv.kind == CHOCO_Q_TOPK;
-    size_t emit_smem = 0;
+    size_t emit_smem[2] = {0, 0};
     auto add = [](choco::LayerTable& t, int32_t l, int64_t off, int64_t dl, uint32_t blocks) {
         const int e = t.entries++;
         t.layer[e] = l;
@@ -207,6 +209,7 @@ int make_groups(choco_layers* L, const float* X, const float* Xhat, const float*
         t.first_block[e + 1] = t.first_block[e] + blocks;
     };
     L->tiles_al.first_block[0] = L->tiles_ua.first_block[0] = L->rows.first_block[0] = 0u;
+    L->rows_small.first_block[0] = L->rows_large.first_block[0] = 0u;
     for (int32_t l = 0; l < L->n_layers; ++l) {
         const int64_t o = L->off[l], dl = L->off[l + 1] - L->off[l];
         const void* ptr[5] = {X + o, Xhat + o, S + o, G ? G + o : nullptr, M ? M + o : nullptr};
@@ -217,10 +220,13 @@ int make_groups(choco_layers* L, const float* X, const float* Xhat, const float*
         const uint32_t tiles = (uint32_t)((dl + choco::kTile - 1) / choco::kTile);
         add(al_ok ? L->tiles_al : L->tiles_ua, l, o, dl, tiles);
         add(L->rows, l, o, dl, (uint32_t)L->n);
+        const int big = dl > choco::kSmallRow ? 1 : 0;
+        add(big ? L->rows_large : L->rows_small, l, o, dl, (uint32_t)L->n);
         L->grouped.push_back(l);
-        emit_smem = std::max<size_t>(emit_smem, (size_t)L->ctx[l]->dv.emit_smem_bytes);
+        emit_smem[big] = std::max<size_t>(emit_smem[big], (size_t)L->ctx[l]->dv.emit_smem_bytes);
     }
-    L->emit_smem = emit_smem;
+    L->emit_smem_small = emit_smem[0];
+    L->emit_smem_large = emit_smem[1];
     L->groups_valid = true;
     return CHOCO_OK;
 }
@@ -283,8 +289,12 @@ int combined_step(choco_layers* L, float* X, float* Xhat, float* S, const float*
     ls.ld = L->ld;
     cudaError_t e = cudaSuccess;
     if (proto.kind == CHOCO_Q_TOPK) {
-        if (L->rows.entries) {
-            e = launch_select_emit_layers(L->rows, ls, L->n, L->emit_smem, a, st);
+        if (L->rows_small.entries) {
+            e = launch_select_emit_layers(L->rows_small, ls, L->n, L->emit_smem_small, true, a, st);
+            launches += 1;
+        }
+        if (e == cudaSuccess && L->rows_large.entries) {
+            e = launch_select_emit_layers(L->rows_large, ls, L->n, L->emit_smem_large, false, a, st);
             launches += 1;
         }
         for (const auto& g : {std::make_pair(&L->tiles_al, true), std::make_pair(&L->tiles_ua, false)}) {
@@ -428,7 +438,8 @@ int choco_layers_init(choco_layers** out, int32_t n, int32_t n_layers, const int
     L->align_key = 0;
     L->groups_valid = false;
     L->tiles_al.entries = L->tiles_ua.entries = L->rows.entries = 0;
-    L->emit_smem = 0;
+    L->rows_small.entries = L->rows_large.entries = 0;
+    L->emit_smem_small = L->emit_smem_large = 0;
     L->combined_steps = 0;
     std::memset(L->side, 0, sizeof(L->side));
     std::memset(L->join, 0, sizeof(L->join));

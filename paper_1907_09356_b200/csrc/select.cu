@@ -244,7 +244,8 @@ __global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs 
 // keys actually span: candidates share their leading bits, so a fixed radix digit would pile
 // them into a handful of bins (and serialise the shared-memory atomics); bins spread over
 // [min, max] instead, then over the chosen bin, until a bin is one key wide.
-// Block-wide minimum and maximum of per-thread values (kSelThreads threads); `sm` needs 64 words.
+// Block-wide minimum and maximum of per-thread values (NT threads); `sm` needs 64 words.
+template <int NT>
 __device__ __forceinline__ void block_min_max(uint32_t& lo, uint32_t& hi, uint32_t* sm)
 {
     lo = __reduce_min_sync(0xffffffffu, lo);
@@ -252,7 +253,7 @@ __device__ __forceinline__ void block_min_max(uint32_t& lo, uint32_t& hi, uint32
     __syncthreads(); // protect sm from the previous use
     if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = lo; sm[32 + (threadIdx.x >> 5)] = hi; }
     __syncthreads();
-    for (int w = 0; w < kSelThreads / 32; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         lo = sm[w] < lo ? sm[w] : lo;
         hi = sm[32 + w] > hi ? sm[32 + w] : hi;
     }
@@ -261,7 +262,8 @@ __device__ __forceinline__ void block_min_max(uint32_t& lo, uint32_t& hi, uint32
 
 constexpr int kListCap = 1024; // a histogram bin this small is resolved by direct comparison
 
-template <typename KeyFn>
+// NT threads; a list of at most min(NT, kListCap) keys is ranked with one key per thread
+template <int NT, typename KeyFn>
 __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t rank, uint32_t lo,
                                          uint32_t hi, uint32_t* h, uint32_t* sm, uint32_t* key_out,
                                          uint32_t* above_out)
@@ -272,15 +274,15 @@ __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t ran
         const uint32_t width = hi - lo;
         const int shift = width < (uint32_t)kHistBins ? 0 : (32 - __clz(width)) - 11;
         const int nbins = (int)(width >> shift) + 1; // <= kHistBins
-        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
+        for (int b = threadIdx.x; b < kHistBins; b += NT) h[b] = 0u;
         __syncthreads();
-        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+        for (uint32_t p = threadIdx.x; p < ncand; p += NT) {
             const uint32_t kk = key(p);
             if (kk >= lo && kk <= hi) atomicAdd(&h[(kk - lo) >> shift], 1u);
         }
         __syncthreads();
         uint32_t digit, above;
-        block_find_digit<kSelThreads>(h, nbins, need, sm, &digit, &above);
+        block_find_digit<NT, kHistBins / NT>(h, nbins, need, sm, &digit, &above);
         const uint32_t inbin = h[digit];
         need -= above;
         above_total += above;
@@ -291,13 +293,13 @@ __device__ __forceinline__ void rank_key(KeyFn key, uint32_t ncand, uint32_t ran
         hi = nhi;
         __syncthreads();
         if (shift == 0) break;
-        if (inbin <= (uint32_t)kListCap) {
+        if (inbin <= (uint32_t)(NT < kListCap ? NT : kListCap)) {
             // few keys left in [lo, hi]: list them (h is free now) and rank them directly
-            uint32_t* list = h;          // kListCap keys
+            uint32_t* list = h;          // at most kListCap keys
             uint32_t* count = sm + 40;   // one word
             if (threadIdx.x == 0) { *count = 0u; sm[41] = lo; sm[42] = 0u; }
             __syncthreads();
-            for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+            for (uint32_t p = threadIdx.x; p < ncand; p += NT) {
                 const uint32_t kk = key(p);
                 if (kk >= lo && kk <= hi) list[atomicAdd(count, 1u)] = kk;
             }
@@ -368,19 +370,20 @@ __device__ __forceinline__ uint32_t next_bound(uint32_t lo, uint32_t T, uint32_t
     return lo > (uint32_t)dec ? lo - (uint32_t)dec : 0u;
 }
 
-// Exclusive prefix sums, in place, of two arrays of length n (one block, kSelThreads threads).
+// Exclusive prefix sums, in place, of two arrays of length n (one block, NT threads).
 // `carry` is two words of shared memory; totals are returned through tot_a / tot_b.
+template <int NT>
 __device__ __forceinline__ void block_scan_pair(uint32_t* a, uint32_t* b, int64_t n, uint32_t* sm,
                                                 uint32_t* carry, uint32_t* tot_a, uint32_t* tot_b)
 {
     if (threadIdx.x == 0) { carry[0] = 0u; carry[1] = 0u; }
     __syncthreads();
-    for (int64_t i0 = 0; i0 < n; i0 += kSelThreads) {
+    for (int64_t i0 = 0; i0 < n; i0 += NT) {
         const int64_t i = i0 + threadIdx.x;
         const uint32_t va = i < n ? a[i] : 0u, vb = i < n ? b[i] : 0u;
         uint32_t ta, tb;
-        const uint32_t ea = block_scan_excl<kSelThreads>(va, sm, &ta);
-        const uint32_t eb = block_scan_excl<kSelThreads>(vb, sm, &tb);
+        const uint32_t ea = block_scan_excl<NT>(va, sm, &ta);
+        const uint32_t eb = block_scan_excl<NT>(vb, sm, &tb);
         const uint32_t ca = carry[0], cb = carry[1];
         if (i < n) { a[i] = ca + ea; b[i] = cb + eb; }
         __syncthreads();
@@ -395,13 +398,12 @@ __device__ __forceinline__ void block_scan_pair(uint32_t* a, uint32_t* b, int64_
 // exact: one block selects straight from the dense row (three radix passes and an ordered
 // compaction pass).  Slow; only for rows whose candidates could not be used.
 // ---------------------------------------------------------------------------------------
-template <int KIND, bool VEC>
+template <int KIND, bool VEC, int NT>
 __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int row, uint32_t* h, uint32_t* sm)
 {
     const uint32_t k = (uint32_t)dv.k;
-    const int64_t span = (int64_t)kSelThreads * kQuad; // coordinates per block iteration
+    const int64_t span = (int64_t)NT * kQuad; // coordinates per block iteration
     const int64_t nspan = (dv.d + span - 1) / span;
-    constexpr int kTilesPerSpan = (kSelThreads * kQuad) / kTile;
     uint32_t prefix = 0, pmask = 0, need = k;
     uint32_t aim_lo = 0, aim_count = 0, aim_above = 0;
     bool aim_in_bin = false;
@@ -410,7 +412,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     const int shifts[3] = {21, 10, 0};
     const int nbins[3] = {2048, 2048, 1024};
     for (int pass = 0; pass < 3; ++pass) {
-        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0u;
+        for (int b = threadIdx.x; b < kHistBins; b += NT) h[b] = 0u;
         __syncthreads();
         for (int64_t c = (int64_t)threadIdx.x * kQuad; c < dv.d; c += span) {
             uint32_t bits[4];
@@ -424,19 +426,19 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
         }
         __syncthreads();
         uint32_t digit, above;
-        block_find_digit<kSelThreads>(h, nbins[pass], need, sm, &digit, &above);
+        block_find_digit<NT, kHistBins / NT>(h, nbins[pass], need, sm, &digit, &above);
         if (KIND == SEL_TOPK && pass == 0) {
             // a second point for the next step's bound: the eighth-of-an-octave bin that holds
             // the rank the bound aims at, and how many keys lie at or above its lower edge
             uint32_t d2, a2;
-            block_find_digit<kSelThreads>(h, nbins[0], aim_rank, sm, &d2, &a2);
+            block_find_digit<NT, kHistBins / NT>(h, nbins[0], aim_rank, sm, &d2, &a2);
             aim_lo = d2 << shifts[0];
             aim_count = a2 + h[d2];
             aim_in_bin = d2 == digit; // the same bin as rank k: the next pass resolves it further
             aim_above = above;
         } else if (KIND == SEL_TOPK && pass == 1 && aim_in_bin) {
             uint32_t d2, a2;
-            block_find_digit<kSelThreads>(h, nbins[1], aim_rank - aim_above, sm, &d2, &a2);
+            block_find_digit<NT, kHistBins / NT>(h, nbins[1], aim_rank - aim_above, sm, &d2, &a2);
             aim_lo = prefix | (d2 << shifts[1]);
             aim_count = aim_above + a2 + h[d2];
         }
@@ -468,11 +470,11 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
             }
         }
         uint32_t tot;
-        const uint32_t ex = block_scan_excl<kSelThreads>(__popc(gtm) | (__popc(eqm) << 16), sm, &tot);
+        const uint32_t ex = block_scan_excl<NT>(__popc(gtm) | (__popc(eqm) << 16), sm, &tot);
         uint32_t g = run_gt + (ex & 0xFFFFu), q = run_eq + (ex >> 16);
         // the first thread of every tile records how many coordinates were chosen before it
-        if ((threadIdx.x % (kTile / kQuad)) == 0) {
-            const int64_t t = sp * kTilesPerSpan + threadIdx.x / (kTile / kQuad);
+        if (c % kTile == 0) {
+            const int64_t t = c / kTile;
             if (t < dv.ntiles) tp[t] = g + (q < r ? q : r);
         }
 #pragma unroll
@@ -492,7 +494,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     }
     if (threadIdx.x == 0) tp[dv.ntiles] = k;
     __syncthreads();
-    publish_ranges(dv, row, tp, threadIdx.x, kSelThreads);
+    publish_ranges(dv, row, tp, threadIdx.x, NT);
     if (threadIdx.x == 0) {
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
@@ -521,7 +523,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
 // 2 = this launch is their last stage and serves the flagged rows only.
 // One block serves one row.  `dyn` is the block's dynamic shared memory (dv.emit_smem_bytes), `h`
 // kHistBins words, `sm` 64 words and `s_carry` 2 words of shared memory.
-template <int KIND, bool VEC>
+template <int KIND, bool VEC, int NT>
 __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a, int row, int fused, int rescue,
                                                 uint32_t* dyn, uint32_t* h, uint32_t* sm, uint32_t* s_carry)
 {
@@ -541,7 +543,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
             }
             return;
         }
-        exact_row<KIND, VEC>(dv, a, row, h, sm);
+        exact_row<KIND, VEC, NT>(dv, a, row, h, sm);
         return;
     }
     const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
@@ -574,7 +576,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     // a thread's own tile segment, fetched now so that the wait overlaps the copies
     const uint32_t* so = dv.seg_off + (int64_t)row * dv.ntiles;
     const uint32_t* sc = dv.seg_cnt + (int64_t)row * dv.ntiles;
-    const bool own_tile = dv.ntiles <= kSelThreads;
+    const bool own_tile = dv.ntiles <= NT;
     uint32_t my_so = 0u, my_sc = 0u;
     if (own_tile && threadIdx.x < dv.ntiles) { my_so = __ldg(so + threadIdx.x); my_sc = __ldg(sc + threadIdx.x); }
     uint32_t klo = 0xFFFFFFFFu, khi = 0u; // range of the keys
@@ -585,22 +587,22 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
         if (threadIdx.x == 0) ok = mbar_wait_bounded(bar, 0, dv.stats, dv.wait_polls) ? 1 : 0;
         if (!__syncthreads_and(ok)) return; // recorded in the stats: the step's result is invalid
         (void)mbar_wait_bounded(bar, 0, dv.stats, kSpinLimit);
-        for (uint32_t p = threadIdx.x; p < ncand; p += kSelThreads) {
+        for (uint32_t p = threadIdx.x; p < ncand; p += NT) {
             const uint32_t kk = order_key<KIND>(sbits[p]);
             klo = kk < klo ? kk : klo;
             khi = kk > khi ? kk : khi;
         }
     } else {
-        for (uint32_t p0 = threadIdx.x; p0 < ncand; p0 += 4 * kSelThreads) {
+        for (uint32_t p0 = threadIdx.x; p0 < ncand; p0 += 4 * NT) {
             uint32_t bits[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t p = p0 + j * kSelThreads;
+                const uint32_t p = p0 + j * NT;
                 if (p < ncand) bits[j] = __ldg(cv + p);
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t p = p0 + j * kSelThreads;
+                const uint32_t p = p0 + j * NT;
                 if (p < ncand) {
                     const uint32_t kk = order_key<KIND>(bits[j]);
                     klo = kk < klo ? kk : klo;
@@ -609,13 +611,13 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
             }
         }
     }
-    block_min_max(klo, khi, sm);
+    block_min_max<NT>(klo, khi, sm);
     auto bits_at = [&](uint32_t p) -> uint32_t { return cached ? sbits[p] : __ldg(cv + p); };
     auto idx_at = [&](uint32_t p) -> uint32_t { return cached ? sidx[p] : __ldg(ci + p); };
     auto key_at = [&](uint32_t p) -> uint32_t { return order_key<KIND>(bits_at(p)); };
 
     uint32_t T, above;
-    rank_key(key_at, ncand, k, klo, khi, h, sm, &T, &above);
+    rank_key<NT>(key_at, ncand, k, klo, khi, h, sm, &T, &above);
     const uint32_t r = k - above; // how many coordinates with key == T are kept (lowest first)
 
     if (KIND == SEL_TOPK) {
@@ -632,7 +634,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     }
 
     // 2. per slab of 32 candidates: which keys lie above T, which equal it (ballots), how many
-    for (int64_t sl = warp; sl < nslab; sl += kSelThreads / 32) {
+    for (int64_t sl = warp; sl < nslab; sl += NT / 32) {
         const uint32_t p = (uint32_t)(sl << 5) + lane;
         bool gt = false, eq = false;
         if (p < ncand) {
@@ -648,7 +650,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     // 3. prefixes.  Slabs first: with them the number of keys above / equal to T before any
     // candidate position follows from one prefix and one ballot ...
     uint32_t tot_g, tot_e;
-    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
+    block_scan_pair<NT>(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
     auto before = [&](uint32_t pos, uint32_t& g, uint32_t& e) {
         const uint32_t s0 = pos >> 5;
         if ((int64_t)s0 < nslab) {
@@ -661,7 +663,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
         }
     };
     // ... so a tile, whose candidates are consecutive, gets its two counts as differences
-    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += NT) {
         const uint32_t cnt = own_tile ? my_sc : sc[t];
         uint32_t g0 = 0, e0 = 0, g1 = 0, e1 = 0;
         if (cnt) {
@@ -675,9 +677,9 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     __syncthreads();
     // tiles: t_gt <- keys above T before the tile, t_eq <- equal keys before it
     uint32_t tot_a, tot_b;
-    block_scan_pair(t_gt, t_eq, dv.ntiles, sm, s_carry, &tot_a, &tot_b);
+    block_scan_pair<NT>(t_gt, t_eq, dv.ntiles, sm, s_carry, &tot_a, &tot_b);
     uint32_t* tp = dv.tile_ptr + (int64_t)row * (dv.ntiles + 1);
-    for (int64_t t = threadIdx.x; t < dv.ntiles; t += kSelThreads) {
+    for (int64_t t = threadIdx.x; t < dv.ntiles; t += NT) {
         const uint32_t gb = t_gt[t], eb = t_eq[t];
         tp[t] = gb + (eb < r ? eb : r);
         // the two flat prefixes at the tile's first candidate: t_gt <- above, t_sbe <- equal
@@ -698,7 +700,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     // Some of the warps do that while the others publish the range records (both are bound by
     // the latency of their scattered stores); the split follows the two amounts of work, one
     // slab per warp iteration here, 32 records per warp iteration there.
-    const int nwarps = kSelThreads / 32;
+    const int nwarps = NT / 32;
     const int64_t pub_iters = (dv.ntiles * (dv.row_ptr[row + 1] - dv.row_ptr[row]) + 31) / 32;
     int kWriteWarps = (int)((nslab * nwarps + (nslab + pub_iters) / 2) / (nslab + pub_iters));
     kWriteWarps = kWriteWarps < 1 ? 1 : (kWriteWarps > nwarps - 1 ? nwarps - 1 : kWriteWarps);
@@ -720,7 +722,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
             }
         }
     }
-    if (warp >= kWriteWarps) publish_ranges(dv, row, tp, threadIdx.x - kWriteWarps * 32, kSelThreads - kWriteWarps * 32);
+    if (warp >= kWriteWarps) publish_ranges(dv, row, tp, threadIdx.x - kWriteWarps * 32, NT - kWriteWarps * 32);
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
@@ -729,8 +731,8 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     }
 }
 
-template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
+template <int KIND, bool VEC, int NT>
+__global__ void __launch_bounds__(NT) emit_kernel(Dev dv, StepArgs a, int fused, int rescue)
 {
     extern __shared__ __align__(16) uint32_t dyn[];
     __shared__ uint32_t h[kHistBins];
@@ -738,12 +740,13 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(Dev dv, StepArgs a, i
     __shared__ uint32_t s_carry[2];
     wait_for_previous_kernel(); // the candidates come from the kernel before this one
     allow_next_kernel();
-    emit_row_single<KIND, VEC>(dv, a, (int)blockIdx.x, fused, rescue, dyn, h, sm, s_carry);
+    emit_row_single<KIND, VEC, NT>(dv, a, (int)blockIdx.x, fused, rescue, dyn, h, sm, s_carry);
 }
 
 // several layers in one launch: block b serves row b % n of the table's entry b / n (top-k, one
 // block per row; rows may start at any element, so the exact selection reads them element by element)
-__global__ void __launch_bounds__(kSelThreads)
+template <int NT>
+__global__ void __launch_bounds__(NT)
 emit_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs a, int n)
 {
     extern __shared__ __align__(16) uint32_t dyn[];
@@ -756,7 +759,7 @@ emit_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs
     shift_arrays(a, tab.off[en]);
     wait_for_previous_kernel(); // the candidates come from the kernel before this one
     allow_next_kernel();
-    emit_row_single<SEL_TOPK, false>(sdev, a, row, 1, 0, dyn, h, sm, s_carry);
+    emit_row_single<SEL_TOPK, false, NT>(sdev, a, row, 1, 0, dyn, h, sm, s_carry);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -854,7 +857,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
     // blocks reach the same verdict from the same values.
     cluster.sync();
     if (!fits) { // block 0 serves the row alone, with the one-block algorithm
-        if (rank == 0) emit_row_single<KIND, VEC>(dv, a, row, fused, rescue, dyn, h2[0], sm, s_carry);
+        if (rank == 0) emit_row_single<KIND, VEC, kSelThreads>(dv, a, row, fused, rescue, dyn, h2[0], sm, s_carry);
         return;
     }
 
@@ -906,7 +909,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
             __syncthreads(); // the staging arrays are written again by the next pass
         }
     }
-    block_min_max(klo, khi, sm);
+    block_min_max<kSelThreads>(klo, khi, sm);
     if (threadIdx.x == 0) { xch[0] = klo; xch[1] = khi; }
     cluster.sync();
     for (uint32_t c = 0; c < C; ++c) {
@@ -1018,7 +1021,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
     }
     __syncthreads();
     uint32_t tot_g, tot_e;
-    block_scan_pair(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
+    block_scan_pair<kSelThreads>(slab_g, slab_e, nslab, sm, s_carry, &tot_g, &tot_e);
     if (threadIdx.x == 0) { xch[4] = tot_g; xch[5] = tot_e; }
     cluster.sync();
     uint32_t og = 0, oe = 0; // keys above / equal to T in the blocks before this one
@@ -1179,34 +1182,38 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int r
         *a.launches += 1;
         return cudaGetLastError();
     }
-    auto kern = a.vec ? emit_kernel<KIND, true> : emit_kernel<KIND, false>;
-    static bool configured[64][2] = {};
-    if (dev < 0 || dev >= 64 || !configured[dev][vec]) {
+    // short rows: small blocks, several per SM (the kernel is a chain of short phases either way)
+    const int small = dv.d <= kSmallRow ? 1 : 0;
+    auto kern = small ? (a.vec ? emit_kernel<KIND, true, kSelThreadsSmall> : emit_kernel<KIND, false, kSelThreadsSmall>)
+                      : (a.vec ? emit_kernel<KIND, true, kSelThreads> : emit_kernel<KIND, false, kSelThreads>);
+    static bool configured[64][2][2] = {};
+    if (dev < 0 || dev >= 64 || !configured[dev][vec][small]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmitSmemBudget);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev][vec] = true;
+        if (dev >= 0 && dev < 64) configured[dev][vec][small] = true;
     }
-    e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(kSelThreads), (size_t)dv.emit_smem_bytes, st,
-                          hot_range_of(dv), dv, a, fused ? 1 : 0, rescue);
+    e = launch_overlapped(kern, dim3((unsigned)dv.n), dim3(small ? kSelThreadsSmall : kSelThreads),
+                          (size_t)dv.emit_smem_bytes, st, hot_range_of(dv), dv, a, fused ? 1 : 0, rescue);
     if (e != cudaSuccess) return e;
     *a.launches += 1;
     return cudaGetLastError();
 }
 
-cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes,
+cudaError_t launch_select_emit_layers(const LayerTable& tab, const LayerSet& ls, int32_t n, size_t smem_bytes, bool small,
                                       const StepArgs& a, cudaStream_t st)
 {
-    static size_t configured[64] = {};
+    static size_t configured[64][2] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || configured[dev] < smem_bytes) {
-        e = cudaFuncSetAttribute(emit_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    auto kern = small ? emit_layers_kernel<kSelThreadsSmall> : emit_layers_kernel<kSelThreads>;
+    if (dev < 0 || dev >= 64 || configured[dev][small ? 1 : 0] < smem_bytes) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = smem_bytes;
+        if (dev >= 0 && dev < 64) configured[dev][small ? 1 : 0] = smem_bytes;
     }
-    return launch_overlapped(emit_layers_kernel, dim3((unsigned)(tab.entries * n)), dim3(kSelThreads), smem_bytes, st,
-                             HotRange{nullptr, 0, 0.f}, tab, ls, a, (int)n);
+    return launch_overlapped(kern, dim3((unsigned)(tab.entries * n)), dim3(small ? kSelThreadsSmall : kSelThreads), smem_bytes,
+                             st, HotRange{nullptr, 0, 0.f}, tab, ls, a, (int)n);
 }
 
 cudaError_t launch_select_emit(const Dev& dv, const StepArgs& a, bool fused, cudaStream_t st)

@@ -9,6 +9,7 @@
 namespace choco {
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelThreadsSmall = 256; // blocks for short rows: several of them share an SM
 enum { SEL_TOPK = 0, SEL_RANDK = 1 };
 
 // Ordering key: larger key = kept first.  top_a: |v| without its sign bit, shifted up so that
@@ -52,25 +53,30 @@ __device__ __forceinline__ uint32_t block_scan_excl(uint32_t v, uint32_t* sm, ui
 }
 
 // Given hist[0..nbins) (shared memory) find the largest digit D with
-// sum_{b >= D} hist[b] >= need; *above = sum_{b > D} hist[b].  nbins <= 2 * NT.
-// All threads return the same values.  `sm` needs 36 words.
-template <int NT>
+// sum_{b >= D} hist[b] >= need; *above = sum_{b > D} hist[b].  nbins <= R * NT: a thread looks
+// at R consecutive bins.  All threads return the same values.  `sm` needs 36 words.
+template <int NT, int R = 2>
 __device__ __forceinline__ void block_find_digit(const uint32_t* hist, int nbins, uint32_t need,
                                                  uint32_t* sm, uint32_t* digit, uint32_t* above)
 {
-    const int r0 = 2 * threadIdx.x, r1 = r0 + 1;
-    const uint32_t h0 = r0 < nbins ? hist[nbins - 1 - r0] : 0u;
-    const uint32_t h1 = r1 < nbins ? hist[nbins - 1 - r1] : 0u;
+    uint32_t hv[R], sum = 0u;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        const int r = R * (int)threadIdx.x + i; // bins are walked from the top
+        hv[i] = r < nbins ? hist[nbins - 1 - r] : 0u;
+        sum += hv[i];
+    }
     uint32_t total;
-    const uint32_t ex = block_scan_excl<NT>(h0 + h1, sm, &total);
+    uint32_t run = block_scan_excl<NT>(sum, sm, &total);
     if (threadIdx.x == 0) { sm[34] = 0u; sm[35] = 0u; }
     __syncthreads();
-    if (ex < need && need <= ex + h0) {
-        sm[34] = (uint32_t)(nbins - 1 - r0);
-        sm[35] = ex;
-    } else if (ex + h0 < need && need <= ex + h0 + h1) {
-        sm[34] = (uint32_t)(nbins - 1 - r1);
-        sm[35] = ex + h0;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        if (run < need && need <= run + hv[i]) {
+            sm[34] = (uint32_t)(nbins - 1 - (R * (int)threadIdx.x + i));
+            sm[35] = run;
+        }
+        run += hv[i];
     }
     __syncthreads();
     *digit = sm[34];

@@ -120,6 +120,8 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
         if (HAS_M) bulk_load(ms, mrow - shm, span(shm), bar);
     }
     hs += shh; // the in-place x^ update below addresses the tile by coordinate
+    // every array starts on an 8-byte boundary (rows of even length): pairs instead of elements
+    const bool pairs = !AL && !((shx | shh | shs | shg | shm) & 1u);
 #pragma unroll
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -244,6 +246,10 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
     auto staged_quad = [&](const float* buf, uint32_t sh, int q4) {
         if (AL) return reinterpret_cast<const float4*>(buf)[q4];
         const float* p = buf + sh + q4 * kQuad;
+        if (pairs) { // (elements past the tile's end are read from the buffer's slack and never used)
+            const float2 lo2 = reinterpret_cast<const float2*>(p)[0], hi2 = reinterpret_cast<const float2*>(p)[1];
+            return make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
+        }
         const int left = nvalid - q4 * kQuad;
         return make_float4(p[0], left > 1 ? p[1] : 0.f, left > 2 ? p[2] : 0.f, left > 3 ? p[3] : 0.f);
     };
@@ -293,6 +299,13 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
         if (AL) {
             *reinterpret_cast<float4*>(xr + li) = make_float4(xn[0], xn[1], xn[2], xn[3]);
             if (HAS_M) *reinterpret_cast<float4*>(mrow + li) = make_float4(mv4[0], mv4[1], mv4[2], mv4[3]);
+        } else if (pairs && li + kQuad <= nvalid) {
+            reinterpret_cast<float2*>(xr + li)[0] = make_float2(xn[0], xn[1]);
+            reinterpret_cast<float2*>(xr + li)[1] = make_float2(xn[2], xn[3]);
+            if (HAS_M) {
+                reinterpret_cast<float2*>(mrow + li)[0] = make_float2(mv4[0], mv4[1]);
+                reinterpret_cast<float2*>(mrow + li)[1] = make_float2(mv4[2], mv4[3]);
+            }
         } else {
 #pragma unroll
             for (int e = 0; e < 4; ++e)
