@@ -247,7 +247,7 @@ def compress(p: Params, v: np.ndarray, step: int, worker: int) -> Message:
 # ---------------------------------------------------------------------------
 
 
-def _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M=None, lam=0.0, beta=0.0):
+def _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M=None, lam=0.0, beta=0.0, nesterov=False):
     d = X.shape[1]
     lo, hi = int(w.row_ptr[i]), int(w.row_ptr[i + 1])
     cols = [int(c) for c in w.col[lo:hi]]
@@ -268,18 +268,20 @@ def _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M=None, lam=0.0, beta=0.0)
                                         _f(M[i]), ctypes.c_int32(nnb), qarr, marr, _f(wv),
                                         ctypes.c_int32(self_pos), ctypes.c_float(eta),
                                         ctypes.c_float(gamma), ctypes.c_float(lam),
-                                        ctypes.c_float(beta))
+                                        ctypes.c_float(beta), ctypes.c_int32(1 if nesterov else 0))
 
 
 def step(w, p: Params, X: np.ndarray, Xhat: np.ndarray, S: np.ndarray,
          G: Optional[np.ndarray], eta: float, gamma: float, t: int,
          rows: Optional[Sequence[int]] = None, M: Optional[np.ndarray] = None,
-         lam: float = 0.0, beta: float = 0.0, executor=None) -> dict:
+         lam: float = 0.0, beta: float = 0.0, executor=None, nesterov: bool = False) -> dict:
     """One call on float32 [n, d] arrays, in place.  Returns {worker: Message}.
 
     With `rows`, only those workers are updated (their neighbours' messages are still
     formed): a way to check single rows of a large problem.  With `M` the momentum
-    variant of Algorithm 2 is applied instead of the plain SGD step.  `executor` (a
+    variant of Algorithm 2 is applied instead of the plain SGD step; `nesterov` takes that
+    step along (g + lam x) + beta v' instead of the new memory v' (Appendix D names the
+    variant without a formula: the usual look-ahead form is the reading).  `executor` (a
     concurrent.futures executor of threads; the C routines run without the interpreter
     lock) only spreads the per-worker calls over host cores: all messages are formed
     before any row is updated, and rows are independent of each other, so the result
@@ -293,7 +295,7 @@ def step(w, p: Params, X: np.ndarray, Xhat: np.ndarray, S: np.ndarray,
     need = sorted(need)
     run = map if executor is None else executor.map
     msgs = dict(zip(need, run(lambda j: compress(p, difference(X[j], Xhat[j]), t, j), need)))
-    list(run(lambda i: _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M, lam, beta), todo))
+    list(run(lambda i: _apply_row(i, w, X, Xhat, S, G, msgs, eta, gamma, M, lam, beta, nesterov), todo))
     return msgs
 
 

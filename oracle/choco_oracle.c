@@ -342,12 +342,17 @@ void oracle_apply_row(int64_t d, float* x, float* xhat, float* s, const float* g
  * with x the iterate the gradient was taken at, followed by the gossip correction of
  * the next iteration as in oracle_apply_row:
  *     m' = (g + lambda * x) + beta * m ;  x' = (x - eta * m') + gamma * c.
+ * Appendix D says only that Nesterov momentum can be adapted in the same way and gives no
+ * formula.  The reading taken here (nesterov != 0) is the look-ahead form common in
+ * deep-learning optimisers: the memory is updated as above and the step is taken along
+ *     (g + lambda * x) + beta * m'
+ * instead of m'.
  */
 void oracle_apply_row_momentum(int64_t d, float* x, float* xhat, float* s, const float* g,
                                float* mom, int32_t nnb, const float* const* q_nb,
                                const uint8_t* const* mask_nb, const float* w_nb,
                                int32_t self_pos, float eta, float gamma, float lambda,
-                               float beta)
+                               float beta, int32_t nesterov)
 {
     for (int64_t c = 0; c < d; ++c) {
         float xh = xhat[c];
@@ -362,8 +367,11 @@ void oracle_apply_row_momentum(int64_t d, float* x, float* xhat, float* s, const
         float sn = s[c];
         if (any) sn = sn + acc;
         float cons = sn - xh;
-        float mn = (g[c] + lambda * x[c]) + beta * mom[c];
-        float xn = (x[c] - eta * mn) + gamma * cons;
+        float gl = g[c] + lambda * x[c];
+        float mn = gl + beta * mom[c];
+        float dir = mn;
+        if (nesterov) dir = gl + beta * mn;
+        float xn = (x[c] - eta * dir) + gamma * cons;
         xhat[c] = xh;
         s[c] = sn;
         mom[c] = mn;

@@ -215,3 +215,44 @@ def test_momentum_variant_matches_algorithm2():
     W = w.dense()
     want = (X0.astype(np.float64) - eta * v1) + gamma * ((W - np.eye(n)) @ X0.astype(np.float64))
     assert np.allclose(X, want, rtol=0, atol=3e-6)
+
+
+def test_nesterov_variant_by_hand_and_special_cases():
+    # one worker (W = [1]): the gossip term vanishes and the recursion is a scalar one
+    w = workloads.MixingCSR(1, np.array([0, 1], np.int32), np.array([0], np.int32), np.array([1.0], np.float32))
+    X = np.zeros((1, 1), np.float32)
+    Xh, S, M = X.copy(), X.copy(), X.copy()
+    G = np.ones((1, 1), np.float32)
+    p = oracle.Params("identity")
+    got = []
+    for t in range(3):
+        oracle.step(w, p, X, Xh, S, G, 0.125, 0.5, t, M=M, lam=0.0, beta=0.5, nesterov=True)
+        got.append((float(M[0, 0]), float(X[0, 0])))
+    # v: 1, 1.5, 1.75; x: -(1 + .5)/8, that -(1 + .75)/8, that -(1 + .875)/8   (all exact in binary)
+    assert got == [(1.0, -0.1875), (1.5, -0.40625), (1.75, -0.640625)]
+
+    w = workloads.ring(4)
+    n, d = 4, 32
+    Xa, Xh, S = _fresh(n, d, 21)
+    M0 = workloads.normal_rows(n, d, 0.5, 22)
+    G = workloads.normal_rows(n, d, 1.0, 23)
+    X0 = Xa.copy()
+    eta, gamma, lam = 0.1, 0.2, 1e-2
+    # beta = 0: both variants are plain SGD with weight decay
+    runs = []
+    for nes in (False, True):
+        X, H, Sx, M = X0.copy(), Xh.copy(), S.copy(), M0.copy()
+        oracle.step(w, p, X, H, Sx, G, eta, gamma, 0, M=M, lam=lam, beta=0.0, nesterov=nes)
+        runs.append((X, M))
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    # beta > 0: same memory as Algorithm 2, iterate moved by a further -eta beta v'
+    beta = 0.9
+    X, H, Sx, M = X0.copy(), Xh.copy(), S.copy(), M0.copy()
+    oracle.step(w, p, X, H, Sx, G, eta, gamma, 0, M=M, lam=lam, beta=beta)
+    Xn, Hn, Sn, Mn = X0.copy(), Xh.copy(), S.copy(), M0.copy()
+    oracle.step(w, p, Xn, Hn, Sn, G, eta, gamma, 0, M=Mn, lam=lam, beta=beta, nesterov=True)
+    assert np.array_equal(M, Mn)
+    gl = G.astype(np.float64) + lam * X0
+    want = X.astype(np.float64) + eta * M - eta * (gl + beta * M)
+    assert np.allclose(Xn, want, rtol=0, atol=3e-6)
+    assert not np.allclose(Xn, X, rtol=0, atol=1e-3)
