@@ -149,6 +149,16 @@ int choco_sgd_momentum_step(choco_ctx* ctx, float* X, float* Xhat, float* S, con
                             void* stream);
 
 /*
+ * choco_set_nesterov -- Appendix D remarks that Nesterov momentum can be adapted in the same way
+ * as Algorithm 2 and gives no formula.  With enable = 1 the momentum step calls of this context
+ * keep Algorithm 2's memory update and take the step along the look-ahead direction,
+ *     m_i = (g_i + lambda x_i) + beta m_i ;   x_i = (x_i - eta ((g_i + lambda x_i) + beta m_i)) + gamma (s_i - x^_i)
+ * (the new m_i on the right), the form common in deep-learning optimisers.  enable = 0 (the
+ * default) restores Algorithm 2.  Steps captured into CUDA graphs are dropped.
+ */
+int choco_set_nesterov(choco_ctx* ctx, int32_t enable);
+
+/*
  * choco_sgd_step_host -- the same step as choco_sgd_step on HOST arrays (pageable or
  * pinned): copies X, Xhat, S, G to library-owned device staging buffers (allocated on the
  * first such call), runs the step, copies X, Xhat, S back and synchronises `stream` before
@@ -323,9 +333,10 @@ int choco_layers_get_layer(const choco_layers* layers, int32_t layer, choco_ctx*
 int choco_layers_set_graphs(choco_layers* layers, int32_t enable, uint64_t* replays);
 /* Number of step calls so far that were enqueued as the combined launches described above. */
 int choco_layers_combined_steps(const choco_layers* layers, uint64_t* steps);
-/* choco_invalidate / choco_set_step for every layer. */
+/* choco_invalidate / choco_set_step / choco_set_nesterov for every layer. */
 int choco_layers_invalidate(choco_layers* layers);
 int choco_layers_set_step(choco_layers* layers, uint64_t t);
+int choco_layers_set_nesterov(choco_layers* layers, int32_t enable);
 
 /* Counters since choco_init (HOST struct filled after synchronising `stream`). */
 typedef struct {

@@ -308,7 +308,7 @@ def layer_k(a_num: int, a_den: int, length: int) -> int:
 def step_layers(w, p: Params, layer_off: Sequence[int], a_num: int, a_den: int,
                 X: np.ndarray, Xhat: np.ndarray, S: np.ndarray, G: Optional[np.ndarray],
                 eta: float, gamma: float, t: int, M: Optional[np.ndarray] = None,
-                lam: float = 0.0, beta: float = 0.0,
+                lam: float = 0.0, beta: float = 0.0, nesterov: bool = False,
                 rows: Optional[Sequence[int]] = None) -> list:
     """Per-layer compression (Section 5, "Setup": every compression scheme is applied to
     every layer separately): the columns [layer_off[l], layer_off[l+1]) of the arrays are
@@ -325,7 +325,7 @@ def step_layers(w, p: Params, layer_off: Sequence[int], a_num: int, a_den: int,
         parts = [np.ascontiguousarray(A[:, lo:hi]) if A is not None else None
                  for A in (X, Xhat, S, G, M)]
         out.append(step(w, pl, parts[0], parts[1], parts[2], parts[3], eta, gamma, t,
-                        rows=rows, M=parts[4], lam=lam, beta=beta))
+                        rows=rows, M=parts[4], lam=lam, beta=beta, nesterov=nesterov))
         for A, part in ((X, parts[0]), (Xhat, parts[1]), (S, parts[2]), (M, parts[4])):
             if A is not None:
                 A[:, lo:hi] = part

@@ -21,14 +21,14 @@ Q_KINDS = {"identity": Q_IDENTITY, "topk": Q_TOPK, "randk": Q_RANDK, "qsgd": Q_Q
 EXPORTS = [
     "choco_init", "choco_destroy", "choco_gossip_step", "choco_sgd_step",
     "choco_sgd_momentum_step", "choco_sgd_step_host", "choco_invalidate", "choco_set_carry",
-    "choco_get_step", "choco_set_graphs", "choco_set_rescue", "choco_set_select_blocks",
+    "choco_get_step", "choco_set_graphs", "choco_set_rescue", "choco_set_select_blocks", "choco_set_nesterov",
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
     "choco_last_cuda_error", "choco_debug_set_wait_polls",
     "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
     "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
-    "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_graphs", "choco_layers_combined_steps",
+    "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_nesterov", "choco_layers_set_graphs", "choco_layers_combined_steps",
 ]
 
 
@@ -80,6 +80,7 @@ def load() -> ctypes.CDLL:
         lib.choco_set_graphs.argtypes = [vp, i32]
         lib.choco_set_rescue.argtypes = [vp, i32]
         lib.choco_set_select_blocks.argtypes = [vp, i32]
+        lib.choco_set_nesterov.argtypes = [vp, i32]
         lib.choco_get_step.argtypes = [vp, ctypes.POINTER(u64)]
         lib.choco_set_step.argtypes = [vp, u64]
         lib.choco_message_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -106,6 +107,7 @@ def load() -> ctypes.CDLL:
                                                ctypes.POINTER(i64)]
         lib.choco_layers_invalidate.argtypes = [vp]
         lib.choco_layers_set_step.argtypes = [vp, u64]
+        lib.choco_layers_set_nesterov.argtypes = [vp, i32]
         lib.choco_layers_set_graphs.argtypes = [vp, i32, ctypes.POINTER(u64)]
         lib.choco_layers_combined_steps.argtypes = [vp, ctypes.POINTER(u64)]
         for name in EXPORTS:
@@ -200,6 +202,10 @@ def choco_set_rescue(ctx, enable: bool) -> None:
 
 def choco_set_select_blocks(ctx, blocks: int) -> None:
     _check(load().choco_set_select_blocks(ctx, blocks), ctx)
+
+
+def choco_set_nesterov(ctx, enable: bool) -> None:
+    _check(load().choco_set_nesterov(ctx, 1 if enable else 0), ctx)
 
 
 def choco_get_step(ctx) -> int:
@@ -347,6 +353,10 @@ def choco_layers_invalidate(layers) -> None:
 
 def choco_layers_set_step(layers, t: int) -> None:
     _check(load().choco_layers_set_step(layers, t))
+
+
+def choco_layers_set_nesterov(layers, enable: bool) -> None:
+    _check(load().choco_layers_set_nesterov(layers, 1 if enable else 0))
 
 
 # --------------------------------------------------------------------------- convenience

@@ -343,6 +343,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
     Dev& dv = ctx->dv;
     dv.n = n; dv.d = d; dv.ld = ld; dv.kind = p->kind; dv.seed = seed;
     dv.wait_polls = kSpinLimit;
+    dv.nesterov = 0;
     for (uint32_t r = 0; r < 10; ++r) {
         dv.round_key[r][0] = (uint32_t)seed + r * 0x9E3779B9u;
         dv.round_key[r][1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
@@ -624,6 +625,18 @@ int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks)
     ctx->dv.emit_cluster = blocks;
     ctx->dv_epoch += 1;
     // the kernels a step enqueues change: no captured step stands for it any more
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+    ctx->ngraphs = 0;
+    return CHOCO_OK;
+}
+
+int choco_set_nesterov(choco_ctx* ctx, int32_t enable)
+{
+    if (!ctx) return CHOCO_ERR_INVALID_ARG;
+    ctx->dv.nesterov = enable ? 1 : 0;
+    ctx->dv_epoch += 1;
+    // captured steps hold the old parameter block
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
     ctx->ngraphs = 0;

@@ -95,6 +95,7 @@ struct Dev {
     int64_t emit_cap_local;      // candidates one block of the cluster can hold in shared memory
     Stats* stats;
     uint32_t wait_polls;         // bound of the kernels' first wait for their staged copies
+    int32_t nesterov;            // momentum steps use the look-ahead direction (choco_set_nesterov)
     // what steps ask the L2 cache to keep resident (sparse Q): messages, range records, tables
     void* hot_base;
     int64_t hot_bytes;

@@ -558,4 +558,18 @@ int choco_layers_set_step(choco_layers* L, uint64_t t)
     return CHOCO_OK;
 }
 
+int choco_layers_set_nesterov(choco_layers* L, int32_t enable)
+{
+    if (!L) return CHOCO_ERR_INVALID_ARG;
+    for (choco_ctx* c : L->ctx) {
+        const int rc = choco_set_nesterov(c, enable); // (bumps the parameter epoch: the copies are uploaded again)
+        if (rc != CHOCO_OK) return rc;
+    }
+    // captured steps hold the old parameter blocks
+    for (StepGraph& g : L->graphs)
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+    L->graphs.clear();
+    return CHOCO_OK;
+}
+
 } // extern "C"

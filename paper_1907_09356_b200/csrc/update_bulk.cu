@@ -24,6 +24,7 @@ namespace {
 
 struct Upd {
     float eta, gamma, lambda, beta;
+    int nesterov; // the step goes along (g + lambda x) + beta m' instead of the new memory m'
 };
 
 template <bool HAS_G, bool HAS_M>
@@ -32,8 +33,10 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
     const float cons = __fsub_rn(sn, hn);
     float xn = x;
     if (HAS_M) {
-        m = __fadd_rn(__fadd_rn(g, __fmul_rn(u.lambda, x)), __fmul_rn(u.beta, m));
-        xn = __fsub_rn(x, __fmul_rn(u.eta, m));
+        const float gl = __fadd_rn(g, __fmul_rn(u.lambda, x));
+        m = __fadd_rn(gl, __fmul_rn(u.beta, m));
+        const float dir = u.nesterov ? __fadd_rn(gl, __fmul_rn(u.beta, m)) : m;
+        xn = __fsub_rn(x, __fmul_rn(u.eta, dir));
     } else if (HAS_G) {
         xn = __fsub_rn(x, __fmul_rn(u.eta, g));
     }
@@ -239,7 +242,7 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
     }
     __syncthreads();
 
-    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
+    const Upd u = {a.eta, a.gamma, a.lambda, a.beta, dv.nesterov};
     uint32_t take = 0, cnt[NIT];
     uint32_t vbits[NIT][4];
     // a staged quad: one 128-bit read when the tile sits aligned, else element by element

@@ -21,6 +21,7 @@ constexpr int kUpdSpan = kChunk * kUpdIters;
 
 struct Upd {
     float eta, gamma, lambda, beta;
+    int nesterov; // the step goes along (g + lambda x) + beta m' instead of the new memory m'
 };
 
 template <bool HAS_G, bool HAS_M>
@@ -29,8 +30,10 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
     const float cons = __fsub_rn(sn, hn);
     float xn = x;
     if (HAS_M) {
-        m = __fadd_rn(__fadd_rn(g, __fmul_rn(u.lambda, x)), __fmul_rn(u.beta, m));
-        xn = __fsub_rn(x, __fmul_rn(u.eta, m));
+        const float gl = __fadd_rn(g, __fmul_rn(u.lambda, x));
+        m = __fadd_rn(gl, __fmul_rn(u.beta, m));
+        const float dir = u.nesterov ? __fadd_rn(gl, __fmul_rn(u.beta, m)) : m;
+        xn = __fsub_rn(x, __fmul_rn(u.eta, dir));
     } else if (HAS_G) {
         xn = __fsub_rn(x, __fmul_rn(u.eta, g));
     }
@@ -82,7 +85,7 @@ __global__ void __launch_bounds__(kThreads, 4) update_dense_kernel(Dev dv, StepA
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kUpdSpan;
     const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
-    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
+    const Upd u = {a.eta, a.gamma, a.lambda, a.beta, dv.nesterov};
     float* xr = a.X + (int64_t)row * dv.ld;
     float* hr = a.Xhat + (int64_t)row * dv.ld;
     float* sr = a.S + (int64_t)row * dv.ld;

@@ -42,6 +42,7 @@ constexpr int kTabLevels = 16;           // level magnitudes are tabulated for s
 
 struct Upd {
     float eta, gamma, lambda, beta;
+    int nesterov; // the step goes along (g + lambda x) + beta m' instead of the new memory m'
 };
 
 template <bool HAS_G, bool HAS_M>
@@ -50,8 +51,10 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
     const float cons = __fsub_rn(sn, hn);
     float xn = x;
     if (HAS_M) {
-        m = __fadd_rn(__fadd_rn(g, __fmul_rn(u.lambda, x)), __fmul_rn(u.beta, m));
-        xn = __fsub_rn(x, __fmul_rn(u.eta, m));
+        const float gl = __fadd_rn(g, __fmul_rn(u.lambda, x));
+        m = __fadd_rn(gl, __fmul_rn(u.beta, m));
+        const float dir = u.nesterov ? __fadd_rn(gl, __fmul_rn(u.beta, m)) : m;
+        xn = __fsub_rn(x, __fmul_rn(u.eta, dir));
     } else if (HAS_G) {
         xn = __fsub_rn(x, __fmul_rn(u.eta, g));
     }
@@ -172,7 +175,6 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = bx * kDTile;
     const int nvalid = (int)((d - c0) < kDTile ? (d - c0) : kDTile); // AL: a multiple of 4
-    const Upd u = {a.eta, a.gamma, a.lambda, a.beta};
     float* xr = a.X + (int64_t)row * ld + c0;
     float* hr = a.Xhat + (int64_t)row * ld + c0;
     float* sr = a.S + (int64_t)row * ld + c0;
@@ -209,6 +211,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
         if (threadIdx.x == 0) request_tiles();
         load_layer_params(dv_src, const_cast<Dev*>(&dv));
     }
+    const Upd u = {a.eta, a.gamma, a.lambda, a.beta, dv.nesterov}; // (dv is complete from here on)
     const int e0 = dv.row_ptr[row], deg = dv.row_ptr[row + 1] - e0;
     // stage the message slices of neighbours [first, first + count): lane r of warp 0 issues r's copies
     auto stage_messages = [&](int first, int count) {

@@ -29,7 +29,7 @@ KINDS = [
 
 
 def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, seed=5,
-         check_layers=(), stream=None, g_pool=0, invalidate_at=-1, jump=None):
+         check_layers=(), stream=None, g_pool=0, invalidate_at=-1, jump=None, nesterov=False):
     """`stream`: run the steps on that (non-default) stream, where steady-state steps may be
     replayed from a captured graph; returns the number of steps replayed.  `g_pool` > 0: the
     gradients live in that many fixed device tensors that are refilled, so pointers repeat.
@@ -47,6 +47,8 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
     p = oracle.Params(kind, s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
     h = choco.choco_layers_init(n, off, ld or d, w.row_ptr, w.col, w.val, kind, a_num, a_den,
                                 s=kw.get("s", 16), bucket=kw.get("bucket", 0), seed=seed)
+    if nesterov:
+        choco.choco_layers_set_nesterov(h, True)
     pool = [_dev(np.zeros_like(X), ld) for _ in range(g_pool)]
     t_shift = 0
     torch.cuda.synchronize()
@@ -68,7 +70,7 @@ def _run(w, sizes, kind, kw, steps, ld=None, momentum=False, gossip_only=False, 
                     t_shift = jump[1] - t
                     choco.choco_layers_set_step(h, jump[1])
                 msgs = oracle.step_layers(w, p, off, a_num, a_den, X, Xh, S, G, 0.05, 0.2, t + t_shift,
-                                          M=M, lam=1e-4, beta=0.9)
+                                          M=M, lam=1e-4, beta=0.9, nesterov=nesterov)
                 if gossip_only:
                     choco.choco_layers_gossip_step(h, dX, dXh, dS, 0.2)
                 elif momentum:
@@ -109,6 +111,14 @@ def test_ragged_layers(kind, kw):
 def test_resnet20_layers_on_a_ring(kind, kw):
     sizes = workloads.resnet20_layer_sizes()
     _run(workloads.ring(8), sizes, kind, dict(kw, a=(1, 100)), steps=3, check_layers=(0, 1, 3, 40, 64))
+
+
+def test_nesterov_momentum_over_layers():
+    # per-layer launches first, then the launches over all layers: both take the look-ahead step
+    sizes = workloads.resnet20_layer_sizes()[:12]
+    for kind, kw in (("topk", dict(a=(1, 20))), ("sign", {}), ("qsgd", dict(s=16, bucket=512))):
+        served = _run(workloads.ring(4), sizes, kind, kw, steps=5, momentum=True, nesterov=True)
+        assert served >= 2
 
 
 def test_padded_rows_and_momentum():

@@ -61,7 +61,7 @@ def check_messages(ctx, kind, msgs, d):
 
 def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed=0, ld=None,
                  eta=0.1, gamma=0.2, x_var=1.0, g_var=0.01, sgd=True, momentum=False,
-                 x_init=None, check_msgs=True, grad_fn=None, select_blocks=None):
+                 x_init=None, check_msgs=True, grad_fn=None, select_blocks=None, nesterov=False):
     ld = ld or d
     X = workloads.normal_rows(n, d, x_var, 1000 + seed) if x_init is None else x_init.copy()
     Xh, S = np.zeros_like(X), np.zeros_like(X)
@@ -70,6 +70,8 @@ def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed
     ch = choco.Choco(w, d, kind, k=k, s=s, bucket=bucket, qsgd_biased=biased, seed=seed, ld=ld)
     if select_blocks:
         choco.choco_set_select_blocks(ch.ctx, select_blocks)
+    if nesterov:
+        choco.choco_set_nesterov(ch.ctx, True)
     dX, dXh, dS = _dev(X, ld), _dev(Xh, ld), _dev(S, ld)
     dM = _dev(M, ld) if momentum else None
     try:
@@ -82,7 +84,7 @@ def run_lockstep(w, kind, n, d, steps, *, k=0, s=16, bucket=0, biased=True, seed
                 G = None
             dG = _dev(G, ld) if G is not None else None
             if momentum:
-                msgs = oracle.step(w, p, X, Xh, S, G, eta, gamma, t, M=M, lam=1e-3, beta=0.9)
+                msgs = oracle.step(w, p, X, Xh, S, G, eta, gamma, t, M=M, lam=1e-3, beta=0.9, nesterov=nesterov)
                 ch.sgd_momentum_step(dX, dXh, dS, dG, dM, eta, gamma, 1e-3, 0.9)
             elif G is not None:
                 msgs = oracle.step(w, p, X, Xh, S, G, eta, gamma, t)
@@ -339,6 +341,42 @@ def test_irregular_graph_sparse_and_dense():
 def test_momentum_variant():
     run_lockstep(workloads.ring(4), "topk", 4, 5000, 4, k=50, momentum=True, seed=4)[0].close()
     run_lockstep(workloads.ring(4), "sign", 4, 5000, 3, momentum=True, seed=5)[0].close()
+
+
+@pytest.mark.parametrize("d,ld", [(5000, None), (5002, None), (5001, None)], ids=["aligned", "8-byte rows", "odd rows"])
+def test_nesterov_variant(d, ld):
+    # the look-ahead step of every update kernel (rows 16-byte aligned, 8-byte aligned, at odd elements)
+    w = workloads.ring(4)
+    run_lockstep(w, "topk", 4, d, 4, k=50, momentum=True, nesterov=True, seed=4, ld=ld)[0].close()
+    run_lockstep(w, "sign", 4, d, 3, momentum=True, nesterov=True, seed=5, ld=ld)[0].close()
+    run_lockstep(w, "qsgd", 4, d, 3, bucket=512, momentum=True, nesterov=True, seed=6, ld=ld)[0].close()
+    run_lockstep(w, "qsgd", 4, d, 2, momentum=True, nesterov=True, seed=7, ld=ld)[0].close()
+    run_lockstep(w, "identity", 4, d, 2, momentum=True, nesterov=True, seed=8, ld=ld)[0].close()
+
+
+def test_nesterov_switch_changes_the_step_and_back():
+    # the setter takes effect on the next call, also where steps are replayed from a graph
+    w = workloads.ring(4)
+    n, d = 4, 1024
+    ch = choco.Choco(w, d, "topk", k=10, seed=2)
+    X = workloads.normal_rows(n, d, 1.0, 70)
+    Xh, S, M = np.zeros_like(X), np.zeros_like(X), np.zeros_like(X)
+    G = workloads.normal_rows(n, d, 0.01, 71)
+    p = oracle.Params("topk", k=10, seed=2)
+    dX, dXh, dS, dM, dG = _dev(X), _dev(Xh), _dev(S), _dev(M), _dev(G)
+    st = torch.cuda.Stream()
+    try:
+        with torch.cuda.stream(st):
+            for t in range(12):
+                nes = 4 <= t < 8
+                choco.choco_set_nesterov(ch.ctx, nes)
+                oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, t, M=M, lam=1e-3, beta=0.9, nesterov=nes)
+                ch.sgd_momentum_step(dX, dXh, dS, dG, dM, 0.1, 0.2, 1e-3, 0.9)
+                torch.cuda.synchronize()
+                assert_state(_host(dX, d), X, f"X after step {t}")
+                assert_state(_host(dM, d), M, f"M after step {t}")
+    finally:
+        ch.close()
 
 
 def test_config1_full_run_and_consensus():
