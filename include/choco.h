@@ -215,7 +215,8 @@ int choco_set_rescue(choco_ctx* ctx, int32_t enable);
  * enough that all SMs would not be busy otherwise -- a cluster of 2 or 4 blocks per row that
  * share the row through distributed shared memory.  choco_set_select_blocks -- blocks = 1, 2 or
  * 4 overrides that choice for the context (TOPK / RANDK only; CHOCO_ERR_UNSUPPORTED otherwise).
- * The result is the same either way.
+ * The result is the same either way.  Implies choco_invalidate (the candidates the last step
+ * collected are arranged for the other kernel).
  */
 int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks);
 
@@ -360,6 +361,18 @@ int choco_get_stats(choco_ctx* ctx, choco_stats* out, void* stream);
  * invalid after such a step.  Not for production use.
  */
 int choco_debug_set_wait_polls(choco_ctx* ctx, uint32_t polls);
+
+/*
+ * Test hook.  When a cluster of blocks selects a row (choco_set_select_blocks), the update kernel
+ * that collects the next step's candidates puts those of a 2048-coordinate tile into the tile's
+ * own slot of the candidate arrays, and only a tile with more candidates than the slot holds
+ * reserves room behind the slots with an atomic add.  The slot is sized at choco_init (three
+ * times a tile's share of 3 k candidates, at least 16); this call makes it smaller, `slot` >= 1
+ * (values above the initial size are clamped to it), so that a test reaches the path behind the
+ * slots and its exhaustion.  The result of a step does not depend on it.  TOPK contexts with
+ * more than one block per row only; CHOCO_ERR_UNSUPPORTED otherwise.  Implies choco_invalidate.
+ */
+int choco_debug_set_candidate_slot(choco_ctx* ctx, int32_t slot);
 
 /*
  * Optional timing of the update kernel (the one pass that streams X, Xhat, S and G): after

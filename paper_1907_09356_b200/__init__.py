@@ -25,7 +25,7 @@ EXPORTS = [
     "choco_set_step", "choco_message_bytes", "choco_get_message", "choco_read_message",
     "choco_consensus_error", "choco_consensus_error_noalloc",
     "choco_get_stats", "choco_profile_enable", "choco_profile_set_stride", "choco_profile_read", "choco_strerror",
-    "choco_last_cuda_error", "choco_debug_set_wait_polls",
+    "choco_last_cuda_error", "choco_debug_set_wait_polls", "choco_debug_set_candidate_slot",
     "choco_layers_init", "choco_layers_destroy", "choco_layers_gossip_step", "choco_layers_sgd_step",
     "choco_layers_sgd_momentum_step", "choco_layers_message_bytes", "choco_layers_get_layer",
     "choco_layers_invalidate", "choco_layers_set_step", "choco_layers_set_nesterov", "choco_layers_set_graphs", "choco_layers_combined_steps",
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
         lib.choco_set_rescue.argtypes = [vp, i32]
         lib.choco_set_select_blocks.argtypes = [vp, i32]
         lib.choco_set_nesterov.argtypes = [vp, i32]
+        lib.choco_debug_set_candidate_slot.argtypes = [vp, i32]
         lib.choco_get_step.argtypes = [vp, ctypes.POINTER(u64)]
         lib.choco_set_step.argtypes = [vp, u64]
         lib.choco_message_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -202,6 +203,10 @@ def choco_set_rescue(ctx, enable: bool) -> None:
 
 def choco_set_select_blocks(ctx, blocks: int) -> None:
     _check(load().choco_set_select_blocks(ctx, blocks), ctx)
+
+
+def choco_debug_set_candidate_slot(ctx, slot: int) -> None:
+    _check(load().choco_debug_set_candidate_slot(ctx, slot), ctx)
 
 
 def choco_set_nesterov(ctx, enable: bool) -> None:

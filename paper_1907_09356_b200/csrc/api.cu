@@ -396,6 +396,16 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         int64_t cap = 6 * p->k > p->k + 8192 ? 6 * p->k : p->k + 8192;
         dv.cap = round_up(cap < d ? cap : d, 4); // rows of the candidate arrays stay 16-byte aligned
         {
+            // slots of three times a tile's share of the 3 k candidates the bound aims at first
+            // (a tile cannot have more than kTile), and room for 2 k candidates behind them
+            const int64_t share = (9 * p->k + dv.ntiles - 1) / dv.ntiles;
+            const int64_t slot = std::min<int64_t>(kTile, std::max<int64_t>(16, round_up(share, 8)));
+            dv.cand_slot_alloc = (uint32_t)slot;
+            dv.cand_slot = 0;
+            const int64_t behind = std::min<int64_t>(dv.cap, std::max<int64_t>(2 * p->k, 2048));
+            dv.cand_pitch = std::max<int64_t>(dv.cap, round_up(dv.ntiles * slot + behind, 4));
+        }
+        {
             // One arena for what one kernel writes and the next reads back within a step.  Its
             // head (range records, messages, per-tile tables) is read with dependent loads by
             // the update kernel: steps ask the L2 cache to keep that part resident while the
@@ -403,10 +413,10 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             const int64_t b_rec = round_up((int64_t)n * dv.ntiles * dv.maxdeg * 16, 256);
             const int64_t b_msg = round_up(n * dv.kpitch * 4, 256);
             const int64_t b_tp = round_up(n * (dv.ntiles + 1) * 4, 256);
-            const int64_t b_cand = round_up(n * dv.cap * 4, 256);
+            const int64_t b_cand = round_up(n * dv.cand_pitch * 4, 256);
             const int64_t b_seg = round_up(n * dv.ntiles * 4, 256);
             const int64_t b_row = round_up((int64_t)n * 4, 256);
-            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 5 * b_row;
+            const int64_t total = b_rec + 2 * b_msg + b_tp + 2 * b_cand + 2 * b_seg + 6 * b_row;
             unsigned char* arena = nullptr;
             if (e == cudaSuccess) e = dev_alloc(ctx, &arena, total);
             unsigned char* q = arena;
@@ -421,6 +431,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             dv.row_flags = (uint32_t*)q; q += b_row;
             dv.row_aim = (uint32_t*)q; q += b_row;
             dv.row_above = (uint32_t*)q; q += b_row;
+            dv.row_ovf = (uint32_t*)q; q += b_row;
             const int64_t hot = q - arena; // the candidates behind it are written once, read once
             dv.cand_idx = (uint32_t*)q; q += b_cand;
             dv.cand_val = (uint32_t*)q; q += b_cand;
@@ -458,6 +469,9 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             const int64_t budget_words = kEmitSmemBudget / 4;
             int64_t cl = ((budget_words - 5152) * 8 / 17) & ~(int64_t)31; // 2.125 words per candidate
             dv.emit_cap_local = std::min<int64_t>(cl, round_up(dv.cap, 32));
+            // the cluster kernel gathers tile by tile: the update kernel may then place a tile's
+            // candidates in the tile's own slot instead of reserving room with an atomic add
+            dv.cand_slot = (p->kind == CHOCO_Q_TOPK && dv.emit_cluster > 1) ? dv.cand_slot_alloc : 0u;
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_c, n * dv.slab_pitch);
@@ -623,8 +637,23 @@ int choco_set_select_blocks(choco_ctx* ctx, int32_t blocks)
     if (!ctx || !(blocks == 1 || blocks == 2 || blocks == 4)) return CHOCO_ERR_INVALID_ARG;
     if (ctx->dv.kind != CHOCO_Q_TOPK && ctx->dv.kind != CHOCO_Q_RANDK) return CHOCO_ERR_UNSUPPORTED;
     ctx->dv.emit_cluster = blocks;
+    ctx->dv.cand_slot = (ctx->dv.kind == CHOCO_Q_TOPK && blocks > 1) ? ctx->dv.cand_slot_alloc : 0u;
+    ctx->prepared = false; // candidates collected by the last step lie in the other arrangement
     ctx->dv_epoch += 1;
     // the kernels a step enqueues change: no captured step stands for it any more
+    for (int i = 0; i < ctx->ngraphs; ++i)
+        if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+    ctx->ngraphs = 0;
+    return CHOCO_OK;
+}
+
+int choco_debug_set_candidate_slot(choco_ctx* ctx, int32_t slot)
+{
+    if (!ctx || slot < 1) return CHOCO_ERR_INVALID_ARG;
+    if (ctx->dv.kind != CHOCO_Q_TOPK || ctx->dv.emit_cluster <= 1) return CHOCO_ERR_UNSUPPORTED;
+    ctx->dv.cand_slot = (uint32_t)slot < ctx->dv.cand_slot_alloc ? (uint32_t)slot : ctx->dv.cand_slot_alloc;
+    ctx->prepared = false;
+    ctx->dv_epoch += 1;
     for (int i = 0; i < ctx->ngraphs; ++i)
         if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
     ctx->ngraphs = 0;

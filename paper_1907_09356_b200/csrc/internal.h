@@ -73,8 +73,17 @@ struct Dev {
     uint32_t* row_aim;           // [n] rank the next bound aims at, in units of k / 256
     uint32_t* row_flags;         // [n]
     uint32_t* row_above;         // [n] keys above the first digit's bin (while a row is refined)
-    uint32_t* cand_idx;          // [n, cap]
-    uint32_t* cand_val;          // [n, cap] value bits (top-k) or random word (random-k)
+    uint32_t* cand_idx;          // [n, cand_pitch]
+    uint32_t* cand_val;          // [n, cand_pitch] value bits (top-k) or random word (random-k)
+    // Where a tile's candidates go.  cand_slot == 0: wherever an atomic add on row_count puts
+    // them (the row's candidates end up contiguous, tiles in arrival order).  cand_slot > 0
+    // (update kernel, when the selection kernel gathers tile by tile anyway): tile t owns
+    // [t * cand_slot, (t + 1) * cand_slot) and needs no reservation; a tile with more candidates
+    // reserves room behind the slots, [ntiles * cand_slot, cand_pitch), through row_ovf.
+    int64_t cand_pitch;          // row stride of the candidate arrays (>= cap, a multiple of 4)
+    uint32_t cand_slot;          // slot per tile in use, or 0
+    uint32_t cand_slot_alloc;    // slot per tile the arrays were sized for
+    uint32_t* row_ovf;           // [n] candidates placed behind the slots
     uint32_t* seg_off;           // [n, ntiles] first candidate of a tile
     uint32_t* seg_cnt;           // [n, ntiles]
     uint32_t* tile_a;            // [n, ntiles] scratch

@@ -249,6 +249,7 @@ bool combinable(const choco_layers* L, const float* X, const float* Xhat)
     for (int32_t l = 0; l < L->n_layers; ++l) {
         const choco_ctx* c = L->ctx[l];
         if (c->timed_out || c->steps_enqueued == 0 || !c->carry_enabled || !c->prepared || c->dv.rescue) return false;
+        if (c->dv.emit_cluster > 1) return false; // (the launch over all layers selects with one block per row)
         if (c->last_x != X + L->off[l] || c->last_xhat != Xhat + L->off[l]) return false;
         if (c->prof_ev && c->prof_n < c->prof_cap) return false;
         if (c->step != c0->step || c->msg_cur != c0->msg_cur) return false;

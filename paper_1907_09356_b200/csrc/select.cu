@@ -149,6 +149,7 @@ __global__ void __launch_bounds__(kSelThreads) bound_kernel(Dev dv, int rescue, 
             dv.row_above[row] = above;
             dv.row_aim[row] = kAimStart;
             dv.row_count[row] = 0u;
+            dv.row_ovf[row] = 0u;
             dv.row_flags[row] = keep | (full ? kRowRefine : 0u);
         } else {
             dv.row_lo[row] = (dv.row_lo[row] & 0xFFE00000u) | (digit << 10);
@@ -165,6 +166,7 @@ __global__ void randk_bound_kernel(Dev dv, uint32_t lo)
     if (row < dv.n) {
         dv.row_lo[row] = lo;
         dv.row_count[row] = 0u;
+        dv.row_ovf[row] = 0u;
         dv.row_flags[row] = 0u;
     }
 }
@@ -217,8 +219,8 @@ __global__ void __launch_bounds__(kTileThreads) collect_kernel(Dev dv, StepArgs 
             const uint32_t base = s_base;
             __syncthreads(); // s_base and sm are written again by the next tile
             if (base == 0xFFFFFFFFu) continue;
-            uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + base;
-            uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + base;
+            uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cand_pitch + base;
+            uint32_t* cv = dv.cand_val + (int64_t)row * dv.cand_pitch + base;
 #pragma unroll
             for (int it = 0; it < kTileIters; ++it) {
                 const int64_t c = c0 + (int64_t)(it * kTileThreads + threadIdx.x) * kQuad;
@@ -498,6 +500,7 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     if (threadIdx.x == 0) {
         dv.row_flags[row] = 0u;
         dv.row_count[row] = 0u;
+        dv.row_ovf[row] = 0u;
         if (KIND == SEL_TOPK) {
             // between (rank k, key T) and (rank aim_count, key aim_lo), as after a usable step
             dv.row_lo[row] = next_bound(aim_lo, T, aim_count, k, kAimAfterMiss);
@@ -522,10 +525,13 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
 // 1 = such a row is flagged kRowRescue instead and left to the rescue kernels that follow;
 // 2 = this launch is their last stage and serves the flagged rows only.
 // One block serves one row.  `dyn` is the block's dynamic shared memory (dv.emit_smem_bytes), `h`
-// kHistBins words, `sm` 64 words and `s_carry` 2 words of shared memory.
+// kHistBins words, `sm` 64 words and `s_carry` 2 words of shared memory.  `contiguous`: the row's
+// candidates lie in [0, row_count) of its candidate arrays (false: in per-tile slots, which this
+// algorithm does not read; the row is then treated like one whose candidates cannot be used).
 template <int KIND, bool VEC, int NT>
 __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a, int row, int fused, int rescue,
-                                                uint32_t* dyn, uint32_t* h, uint32_t* sm, uint32_t* s_carry)
+                                                uint32_t* dyn, uint32_t* h, uint32_t* sm, uint32_t* s_carry,
+                                                bool contiguous = true)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ncand = dv.row_count[row];
@@ -533,7 +539,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     const uint32_t k = (uint32_t)dv.k;
     __syncthreads();
     if (rescue == 2 && !(flags & kRowRescue)) return;
-    if ((flags & kRowExact) || ncand > (uint32_t)dv.cap || ncand < k) { // the candidates cannot be used
+    if ((flags & kRowExact) || !contiguous || ncand > (uint32_t)dv.cap || ncand < k) { // the candidates cannot be used
         if (rescue == 1 && !(flags & kRowExact)) {
             // a fresh histogram would say the same for a row flagged kRowExact; any other row
             // gets new candidates from the kernels that follow
@@ -546,8 +552,8 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
         exact_row<KIND, VEC, NT>(dv, a, row, h, sm);
         return;
     }
-    const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
-    const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
+    const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cand_pitch;
+    const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cand_pitch;
     const int64_t nslab = ((int64_t)ncand + 31) >> 5;
 
     // carve the dynamic shared memory (every piece a multiple of 16 bytes)
@@ -726,6 +732,7 @@ __device__ __forceinline__ void emit_row_single(const Dev& dv, const StepArgs& a
     __syncthreads();
     if (threadIdx.x == 0) {
         dv.row_count[row] = 0u;
+        dv.row_ovf[row] = 0u;
         dv.row_flags[row] = 0u;
         atomicAdd(fused ? &dv.stats->prepared_rows : &dv.stats->recompressed_rows, 1ull);
     }
@@ -857,7 +864,11 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
     // blocks reach the same verdict from the same values.
     cluster.sync();
     if (!fits) { // block 0 serves the row alone, with the one-block algorithm
-        if (rank == 0) emit_row_single<KIND, VEC, kSelThreads>(dv, a, row, fused, rescue, dyn, h2[0], sm, s_carry);
+        // (candidates the update kernel left in per-tile slots are not contiguous; those of the
+        // collection kernel, fused == 0, are)
+        if (rank == 0)
+            emit_row_single<KIND, VEC, kSelThreads>(dv, a, row, fused, rescue, dyn, h2[0], sm, s_carry,
+                                                    !(fused && dv.cand_slot != 0u));
         return;
     }
 
@@ -877,8 +888,8 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
 
     const uint32_t Tb = part_t[rank], Te = part_t[rank + 1];
     const uint32_t L = part_p[rank + 1] - part_p[rank];   // this block's candidates
-    const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap;
-    const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap;
+    const uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cand_pitch;
+    const uint32_t* cv = dv.cand_val + (int64_t)row * dv.cand_pitch;
 
     // gather: a group of kGroup lanes copies one tile's candidates
     uint32_t klo = 0xFFFFFFFFu, khi = 0u;
@@ -1094,6 +1105,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
     cluster.sync();
     if (rank == 0 && threadIdx.x == 0) {
         dv.row_count[row] = 0u;
+        dv.row_ovf[row] = 0u;
         dv.row_flags[row] = 0u;
         atomicAdd(fused ? &dv.stats->prepared_rows : &dv.stats->recompressed_rows, 1ull);
     }

@@ -88,8 +88,9 @@ __device__ __forceinline__ void block_find_digit(const uint32_t* hist, int nbins
 // (it * NT + t) * 4 ... + 3.  Computes the slot of each thread's first chosen coordinate in
 // ascending coordinate order (start[it]) and the number chosen in the whole tile.
 // NIT is 2 or 4 (16-bit fields: a tile holds fewer than 65536 coordinates).
-// `sm` needs 2 x (NT / 32 + 1) words; contains two block barriers.
-template <int NT, int NIT>
+// `sm` needs 2 x (NT / 32 + 1) words; contains two block barriers, or one with FRESH, when
+// the caller knows that no thread of the block still reads `sm` from an earlier use.
+template <int NT, int NIT, bool FRESH = false>
 __device__ __forceinline__ void ordered_starts(const uint32_t cnt[NIT], uint32_t (*sm)[NT / 32 + 1],
                                                uint32_t start[NIT], uint32_t* total)
 {
@@ -109,7 +110,7 @@ __device__ __forceinline__ void ordered_starts(const uint32_t cnt[NIT], uint32_t
             if (lane >= o) ib += tb;
         }
     }
-    __syncthreads(); // protect sm from the previous use
+    if (!FRESH) __syncthreads(); // protect sm from the previous use
     if (lane == 31) {
         sm[0][warp] = ia;
         if constexpr (NIT == 4) sm[1][warp] = ib;

@@ -137,7 +137,15 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
     // after it has itself seen the previous update complete.
     wait_for_previous_kernel();
     allow_next_kernel();
-    const uint32_t lo_key = EMIT ? __ldg(dv.row_lo + row) : 0u; // used at the end: fetch early
+    // The candidate bound (used at the end: fetched early), as the magnitude it stands for:
+    // key(v) = bits(|v|) << 1 >= lo  <=>  bits(|v|) >= ceil(lo / 2)  <=>  |v| >= the float with
+    // those bits (finite floats order like their bit patterns; bits past infinity admit nothing)
+    float lo_mag = 0.f;
+    if (EMIT) {
+        const uint32_t lo_key = __ldg(dv.row_lo + row);
+        const uint32_t half = (lo_key >> 1) + (lo_key & 1u);
+        lo_mag = __uint_as_float(half < 0x7F800000u ? half : 0x7F800000u);
+    }
     // warp 1 builds the neighbour table of the first batch
     uint4 rc = make_uint4(0u, 0u, 0u, 0u);
     if ((threadIdx.x >> 5) == 1 && lane < dv.maxdeg) rc = __ldg(recs + lane);
@@ -293,7 +301,7 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
             xn[e] = next_x<HAS_G, HAS_M>(xv[e], sv[e], hv[e], gv[e], mv4[e], u);
             if (EMIT) {
                 vbits[it][e] = __float_as_uint(__fsub_rn(xn[e], hv[e]));
-                if ((AL || li + e < nvalid) && order_key<SEL_TOPK>(vbits[it][e]) >= lo_key) {
+                if ((AL || li + e < nvalid) && fabsf(__uint_as_float(vbits[it][e])) >= lo_mag) {
                     take |= 1u << (4 * it + e);
                     ++cnt[it];
                 }
@@ -321,18 +329,40 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
 
     if (EMIT) {
         uint32_t start[NIT], total;
-        ordered_starts<NT, NIT>(cnt, scan, start, &total);
-        if (threadIdx.x == 0) {
-            const uint32_t base = total ? atomicAdd(&dv.row_count[row], total) : 0u;
-            dv.seg_off[(int64_t)row * dv.ntiles + tile] = base;
-            dv.seg_cnt[(int64_t)row * dv.ntiles + tile] = total;
-            *s_base = ((int64_t)base + total > dv.cap) ? 0xFFFFFFFFu : base;
+        ordered_starts<NT, NIT, true>(cnt, scan, start, &total); // (the scratch has no other use in this kernel)
+        uint32_t base;
+        if (dv.cand_slot != 0u && total <= dv.cand_slot) {
+            // the tile's own slot: nothing to reserve, nothing to wait for (every thread knows
+            // `total`); the row's count is kept for the selection kernel by an add without a reader
+            base = (uint32_t)tile * dv.cand_slot;
+            if (threadIdx.x == 0) {
+                if (total) atomicAdd(&dv.row_count[row], total);
+                dv.seg_off[(int64_t)row * dv.ntiles + tile] = base;
+                dv.seg_cnt[(int64_t)row * dv.ntiles + tile] = total;
+            }
+        } else {
+            if (threadIdx.x == 0) {
+                uint32_t b = 0u;
+                bool ok = true;
+                if (dv.cand_slot != 0u) { // more than a slot holds: room behind the slots
+                    b = (uint32_t)dv.ntiles * dv.cand_slot + atomicAdd(&dv.row_ovf[row], total);
+                    ok = (int64_t)b + total <= dv.cand_pitch;
+                    // (no room left: a count above the capacity tells the selection kernel to give the candidates up)
+                    atomicAdd(&dv.row_count[row], ok ? total : (uint32_t)dv.cap + 1u);
+                } else {
+                    b = total ? atomicAdd(&dv.row_count[row], total) : 0u;
+                    ok = (int64_t)b + total <= dv.cap; // past the capacity nothing is written; the count says so
+                }
+                dv.seg_off[(int64_t)row * dv.ntiles + tile] = b;
+                dv.seg_cnt[(int64_t)row * dv.ntiles + tile] = total;
+                *s_base = ok ? b : 0xFFFFFFFFu;
+            }
+            __syncthreads();
+            base = *s_base;
         }
-        __syncthreads();
-        const uint32_t base = *s_base;
         if (base == 0xFFFFFFFFu || take == 0u) return;
-        uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cap + base;
-        uint32_t* cv = dv.cand_val + (int64_t)row * dv.cap + base;
+        uint32_t* ci = dv.cand_idx + (int64_t)row * dv.cand_pitch + base;
+        uint32_t* cv = dv.cand_val + (int64_t)row * dv.cand_pitch + base;
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             const uint32_t cbase = (uint32_t)c0 + (uint32_t)(it * NT + threadIdx.x) * kQuad;
