@@ -37,13 +37,13 @@ FALLBACK_HBM_GBS = 6650.0
 # capture of the same kernel scaled by the coordinates per launch, as the capture of the
 # full-size workload would be too large.
 NCU_TRAFFIC = {
-    "c4_torus64_topk": (1.3726e9, "profiles/update_and_emit_kernels_c4_torus64_topk.md"),
-    "c4_torus64_topk_g004": (1.3726e9, "profiles/update_and_emit_kernels_c4_torus64_topk.md (same kernel and shapes, gamma = 0.2)"),
-    "p_ring8_qsgd": (1.9916e9, "profiles/update_dense_bulk_kernel_p_ring8_qsgd.md"),
-    "p_ring8_sign": (1.8563e9, "profiles/update_dense_bulk_kernel_p_ring8_sign.md"),
-    "c5_ring32_qsgd": (29.68 * 32 * 25_557_032,
+    "c4_torus64_topk": (1.3768e9, "profiles/update_and_emit_kernels_c4_torus64_topk.md"),
+    "c4_torus64_topk_g004": (1.3768e9, "profiles/update_and_emit_kernels_c4_torus64_topk.md (same kernel and shapes, gamma = 0.2)"),
+    "p_ring8_qsgd": (1.9950e9, "profiles/update_dense_bulk_kernel_p_ring8_qsgd.md"),
+    "p_ring8_sign": (1.8544e9, "profiles/update_dense_bulk_kernel_p_ring8_sign.md"),
+    "c5_ring32_qsgd": (29.73 * 32 * 25_557_032,
                        "profiles/update_dense_bulk_kernel_p_ring8_qsgd.md (the 8-ring capture of the same kernel, "
-                       "29.68 B per coordinate, scaled by the coordinates per launch)"),
+                       "29.73 B per coordinate, scaled by the coordinates per launch)"),
 }
 
 
