@@ -12,8 +12,9 @@
 // (never touching a 16-byte unit that holds no element of the tile), and the tile is read
 // from shared memory at the resulting offset of 0..3 elements.  Meanwhile the block reads
 // the range records of its neighbours (one round trip), then all their entries that fall
-// into the tile (a second one), and adds them into a shared accumulator tile neighbour by
-// neighbour.  With EMIT the kernel also collects the candidates of the next step's top-k
+// into the tile (a second one), and adds them into a shared accumulator tile: with atomic adds
+// where a coordinate has one or two terms (the order cannot matter there), in CSR order where it
+// has more.  With EMIT the kernel also collects the candidates of the next step's top-k
 // selection from x' - x^', which it holds anyway.
 #include "bulk.cuh"
 #include "select.cuh"
@@ -46,7 +47,7 @@ __device__ __forceinline__ float next_x(float x, float sn, float hn, float g, fl
 constexpr int NT = kTileThreads;
 constexpr int NIT = kTileIters;
 constexpr int kMaxNb = 32; // neighbours handled per batch (one lane each)
-constexpr int kMaxE = 2;   // message entries a thread holds per pass
+constexpr int kMaxE = 3;   // message entries a thread holds per pass
 
 struct NbrTable {
     uint32_t lo[kMaxNb];       // first entry of neighbour r's message inside this tile
@@ -68,10 +69,17 @@ constexpr size_t bulk_smem_bytes()
 {
     return (size_t)(bulk_arrays<HAS_G, HAS_M>() + 1) * kTile * sizeof(float) // tiles + acc
            + (AL ? 0 : bulk_arrays<HAS_G, HAS_M>() * kShiftPad * sizeof(float))
-           + 2 * (kTile / 32) * sizeof(uint32_t)                              // touched, self
+           + 4 * (kTile / 32) * sizeof(uint32_t)                              // touched (once, twice, more), self
            + 8                                                                // barrier
            + 2 * (NT / 32 + 1) * sizeof(uint32_t) + 8                         // scan scratch, base
            + sizeof(NbrTable);
+}
+
+// *p += v on shared memory, atomically: an IEEE single-precision add rounded to nearest that keeps
+// subnormals (atomic float adds on shared memory do; those on global memory flush them to zero)
+__device__ __forceinline__ void shared_add(float* p, float v)
+{
+    asm volatile("red.shared.add.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v) : "memory");
 }
 
 // element offset of p inside its 16-byte unit
@@ -95,7 +103,9 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
     float* acc = ms + (HAS_M ? kStage : 0);
     uint32_t* touched = reinterpret_cast<uint32_t*>(acc + kTile);
     uint32_t* tself = touched + kTile / 32;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(tself + kTile / 32);
+    uint32_t* twice = tself + kTile / 32;  // coordinates with entries of two neighbours ...
+    uint32_t* more = twice + kTile / 32;   // ... of three or more
+    uint64_t* bar = reinterpret_cast<uint64_t*>(more + kTile / 32);
     uint32_t(*scan)[NT / 32 + 1] = reinterpret_cast<uint32_t(*)[NT / 32 + 1]>(bar + 1);
     uint32_t* s_base = reinterpret_cast<uint32_t*>(scan) + 2 * (NT / 32 + 1);
     NbrTable* nbr = reinterpret_cast<NbrTable*>(s_base + 2);
@@ -128,7 +138,9 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
 #pragma unroll
     for (int it = 0; it < NIT; ++it)
         reinterpret_cast<float4*>(acc)[it * NT + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (threadIdx.x < kTile / 32) { touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; }
+    if (threadIdx.x < kTile / 32) {
+        touched[threadIdx.x] = 0u; tself[threadIdx.x] = 0u; twice[threadIdx.x] = 0u; more[threadIdx.x] = 0u;
+    }
     if (LAYERS) load_layer_params(dv_src, const_cast<Dev*>(&dv));
     const uint4* recs = dv.rec + ((int64_t)row * dv.ntiles + tile) * dv.maxdeg;
     // Messages, range records and the candidate bound come from the kernel before this one.
@@ -185,6 +197,75 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
         const uint32_t total = nbr->pref[nb];
         const uint32_t selfr = nbr->self;
         if (selfr < (uint32_t)nb) { self_lo = nbr->lo[selfr]; self_len = nbr->len[selfr]; }
+        if (dv.maxdeg <= kMaxNb && total <= (uint32_t)(NT * kMaxE)) {
+            // All entries of the tile at once, each thread holding at most kMaxE of them.  The sum
+            // over the neighbours starts from +0 and goes in CSR order, but with one or two terms
+            // the order does not matter (0 + a is a, or +0 for a = -0; a + b = b + a): those are
+            // added with shared-memory atomics (round to nearest, subnormals kept) in whatever
+            // order the threads arrive.  Three bit planes count the terms per coordinate; a
+            // coordinate with three or more is redone in order below.
+            const int nq = (int)((total + NT - 1) / NT);
+            float prod[kMaxE];
+            bool third = false;
+#pragma unroll
+            for (int q = 0; q < kMaxE; ++q) {
+                er[q] = -1;
+                const uint32_t f = q * NT + threadIdx.x;
+                if (q < nq && f < total) {
+                    int r = 0;
+                    while (nbr->pref[r + 1] <= f) ++r;
+                    const uint32_t p = nbr->lo[r] + (f - nbr->pref[r]);
+                    const int64_t mrow = (int64_t)nbr->j[r] * dv.kpitch;
+                    er[q] = r;
+                    elc[q] = __ldg(dv.msg_idx + mrow + p) - (uint32_t)c0;
+                    ev[q] = __ldg(dv.msg_val + mrow + p);
+                    prod[q] = __fmul_rn(nbr->w[r], ev[q]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < kMaxE; ++q)
+                if (er[q] >= 0) {
+                    const uint32_t wd = elc[q] >> 5, bit = 1u << (elc[q] & 31);
+                    if (atomicOr(&touched[wd], bit) & bit)
+                        if (atomicOr(&twice[wd], bit) & bit) { atomicOr(&more[wd], bit); third = true; }
+                    shared_add(&acc[elc[q]], prod[q]);
+                }
+            if (__syncthreads_or(third)) {
+                // Some coordinate has three or more terms.  Its terms are ranked by neighbour: the
+                // accumulator word serves as the set of neighbours with an entry there (cleared,
+                // filled with one bit per neighbour, read back), then the terms are added one rank
+                // per round.
+                bool redo[kMaxE];
+                uint32_t rank[kMaxE];
+#pragma unroll
+                for (int q = 0; q < kMaxE; ++q) {
+                    redo[q] = er[q] >= 0 && ((more[elc[q] >> 5] >> (elc[q] & 31)) & 1u);
+                    rank[q] = 0u;
+                    if (redo[q]) acc[elc[q]] = 0.f; // (every thread with a term there writes the same)
+                }
+                __syncthreads();
+                uint32_t* accw = reinterpret_cast<uint32_t*>(acc);
+#pragma unroll
+                for (int q = 0; q < kMaxE; ++q)
+                    if (redo[q]) atomicOr(&accw[elc[q]], 1u << er[q]);
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < kMaxE; ++q)
+                    if (redo[q]) rank[q] = (uint32_t)__popc(accw[elc[q]] & ((1u << er[q]) - 1u));
+                __syncthreads();
+                for (uint32_t j = 0;; ++j) {
+                    bool later = false;
+#pragma unroll
+                    for (int q = 0; q < kMaxE; ++q)
+                        if (redo[q]) {
+                            if (rank[q] == j) acc[elc[q]] = __fadd_rn(j == 0u ? 0.f : acc[elc[q]], prod[q]);
+                            later = later || rank[q] > j;
+                        }
+                    if (!__syncthreads_or(later)) break;
+                }
+            }
+            self_in_regs = true; // this worker's own entries are among those the threads hold
+        } else
         for (uint32_t f0 = 0; f0 < total; f0 += NT * kMaxE) {
 #pragma unroll
             for (int q = 0; q < kMaxE; ++q) {
@@ -217,8 +298,7 @@ __device__ __forceinline__ void update_sparse_bulk_body(const Dev& dv, const Ste
                     }
                 __syncthreads();
             }
-            // a single pass over a single batch keeps this worker's own entries in registers
-            self_in_regs = (f0 == 0 && total <= NT * kMaxE && dv.maxdeg <= kMaxNb);
+            self_in_regs = false;
         }
         if (eb + kMaxNb < dv.maxdeg) __syncthreads(); // the table is rebuilt for the next batch
     }

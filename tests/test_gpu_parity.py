@@ -356,6 +356,22 @@ def test_irregular_graph_sparse_and_dense():
     run_lockstep(w, "sign", 32, 6000, 2, seed=3)[0].close()
 
 
+@pytest.mark.parametrize("graph", ["torus", "irregular"])
+def test_many_neighbours_send_the_same_coordinate(graph):
+    """Workers that start from nearly the same x select the same coordinates, so a coordinate of
+    s_i receives a term from every neighbour: the sum must still go in CSR order from +0 (the
+    update kernel adds one or two terms as they come and redoes coordinates with more in order)."""
+    w = workloads.torus(4, 4) if graph == "torus" else workloads.random_graph(32, 14, 1)
+    n, d, k = w.n, 8192, 160 if graph == "torus" else 64
+    base = workloads.normal_rows(1, d, 1.0, 77)
+    x = np.repeat(base, n, axis=0) + workloads.normal_rows(n, d, 1e-6, 78)
+    ch, _, _ = run_lockstep(w, "topk", n, d, 5, k=k, x_init=x.astype(np.float32), seed=9, gamma=0.3)
+    ch.close()
+    # the same through the general path (more entries per tile than the threads hold at once)
+    ch, _, _ = run_lockstep(w, "topk", n, d, 3, k=2000, x_init=x.astype(np.float32), seed=10, gamma=0.3)
+    ch.close()
+
+
 def test_momentum_variant():
     run_lockstep(workloads.ring(4), "topk", 4, 5000, 4, k=50, momentum=True, seed=4)[0].close()
     run_lockstep(workloads.ring(4), "sign", 4, 5000, 3, momentum=True, seed=5)[0].close()
