@@ -34,9 +34,12 @@ namespace choco {
 
 namespace {
 
-constexpr int NT = 256;
-constexpr int NIT = 2;                   // quads per thread
+constexpr int NT = 128;
+constexpr int NIT = 4;                   // quads per thread (what a thread does once per tile weighs less that way)
 constexpr int kDTile = NT * kQuad * NIT; // 2048 coordinates per block
+constexpr int kWarps = NT / 32;
+constexpr int kWarpSums = NIT * kWarps;  // one per 128 coordinates of the tile, in coordinate order
+static_assert(kDTile == 2048 && kWarpSums == 16, "tile of 2048 coordinates: two chunks of the L1 tree, up to 16 blocks of the norm");
 constexpr int kBatch = 16;               // neighbours whose message slices are staged at a time
 constexpr int kTabLevels = 16;           // level magnitudes are tabulated for s <= 16
 
@@ -121,8 +124,8 @@ struct Layout {
     // magnitude and the weight); then the worker's own unweighted magnitudes
     __host__ __device__ static int table_floats(int nb, int nbk) { return (nb + 1) * nbk * kTabLevels; }
     __host__ __device__ static int misc(int nb, int nbk) { return tables(nb) + table_floats(nb, nbk) * 4; }
-    // misc: warp sums [NIT][8] floats, per-block reciprocal norms [16] doubles, the barrier
-    __host__ __device__ static int total(int nb, int nbk) { return misc(nb, nbk) + NIT * 8 * 4 + 16 * 8 + 16; }
+    // misc: warp sums [kWarpSums] floats, per-block reciprocal norms [16] doubles, the barrier
+    __host__ __device__ static int total(int nb, int nbk) { return misc(nb, nbk) + kWarpSums * 4 + 16 * 8 + 16; }
 };
 
 // element offset of p inside its 16-byte unit
@@ -168,8 +171,8 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
     unsigned char* msg_out = smem_raw + L::msg_out(nb_stage);
     float* tab = reinterpret_cast<float*>(smem_raw + L::tables(nb_stage));
     float* tab_self = tab + nb_stage * nbk * kTabLevels;
-    float* ws = reinterpret_cast<float*>(smem_raw + L::misc(nb_stage, nbk)); // [NIT][8] warp sums
-    double* rnu = reinterpret_cast<double*>(ws + NIT * 8);                   // [16] 1 / nu per block of the norm
+    float* ws = reinterpret_cast<float*>(smem_raw + L::misc(nb_stage, nbk)); // [kWarpSums] sums over 128 coordinates
+    double* rnu = reinterpret_cast<double*>(ws + kWarpSums);                 // [16] 1 / nu per block of the norm
     uint64_t* bar = reinterpret_cast<uint64_t*>(rnu + 16);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -395,7 +398,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
             if (KIND == CHOCO_Q_SIGN) t = quad_tree(fabsf(v.x), fabsf(v.y), fabsf(v.z), fabsf(v.w));
             else t = quad_tree(__fmul_rn(v.x, v.x), __fmul_rn(v.y, v.y), __fmul_rn(v.z, v.z), __fmul_rn(v.w, v.w));
             t = warp_tree(t);
-            if (lane == 0) ws[it * 8 + warp] = t;
+            if (lane == 0) ws[it * kWarps + warp] = t;
             // sign plane of the next message: this quad's four bits and its neighbour's make a byte
             const uint32_t nib = (uint32_t)(v.x < 0.f) | ((uint32_t)(v.y < 0.f) << 1) | ((uint32_t)(v.z < 0.f) << 2) |
                                  ((uint32_t)(v.w < 0.f) << 3);
@@ -421,8 +424,8 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
     }
     if (KIND == CHOCO_Q_SIGN) {
         // per-1024 partial sums of |v|; a small kernel finishes the tree and the scale
-        if (threadIdx.x < NIT) {
-            const int64_t chunk = bx * NIT + threadIdx.x;
+        if (threadIdx.x < kDTile / kChunk) {
+            const int64_t chunk = bx * (kDTile / kChunk) + threadIdx.x;
             if (chunk < dv.nchunks) dv.partial[(int64_t)row * dv.nchunks + chunk] = tree8(ws + threadIdx.x * 8);
         }
         if (storer) bulk_store_commit_and_drain();
@@ -432,8 +435,7 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
     // finishes its tree over the warp sums, stores the norm and leaves 1 / nu for the others
     const int G = dv.bucket >> 7; // warps per block of the norm: 1, 2, 4 or 8
     if ((int)threadIdx.x < nbk) {
-        const int per_it = 8 / G;
-        const float* wsi = ws + ((int)threadIdx.x / per_it) * 8 + ((int)threadIdx.x % per_it) * G;
+        const float* wsi = ws + (int)threadIdx.x * G;
         float sq;
         if (G == 1) sq = wsi[0];
         else if (G == 2) sq = __fadd_rn(wsi[0], wsi[1]);
