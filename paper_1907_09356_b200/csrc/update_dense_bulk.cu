@@ -504,7 +504,7 @@ __global__ void __launch_bounds__(NT, MINB) update_dense_bulk_kernel(Dev dv, Ste
 
 // several layers in one launch: blockIdx.x picks (layer, tile), blockIdx.y the worker
 template <int KIND, int WBITS, bool HAS_G, bool HAS_M, bool AL>
-__global__ void __launch_bounds__(NT, 4)
+__global__ void __launch_bounds__(NT, 5)
 update_dense_bulk_layers_kernel(const __grid_constant__ LayerTable tab, LayerSet ls, StepArgs a, int nb_stage, int nbk)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
