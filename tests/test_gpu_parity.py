@@ -185,6 +185,36 @@ def test_candidates_behind_the_tiles_slots(d, k, slot):
     assert st["prepared_rows"] >= 5 * 5 - 3, st   # (a bound guessed too high may cost a row its candidates)
 
 
+def test_switching_the_selection_kernel_between_steps():
+    """One block per row reads a row's candidates as one contiguous run, a cluster reads them tile
+    by tile from the tiles' slots: switching between steps must not hand one kernel the other's
+    arrangement (the switch drops the carried candidates)."""
+    w = workloads.ring(5)
+    n, d, k = 5, 40000, 400
+    ch = choco.Choco(w, d, "topk", k=k, seed=3)
+    X = workloads.normal_rows(n, d, 1.0, 90)
+    Xh, S = np.zeros_like(X), np.zeros_like(X)
+    p = oracle.Params("topk", k=k, seed=3)
+    dX, dXh, dS = _dev(X), _dev(Xh), _dev(S)
+    try:
+        for t in range(12):
+            if t % 3 == 0:
+                choco.choco_set_select_blocks(ch.ctx, (2, 1, 4, 1)[t // 3])
+            if t == 7:
+                choco.choco_debug_set_candidate_slot(ch.ctx, 4)
+            G = workloads.normal_rows(n, d, 0.01, 500 + t)
+            msgs = oracle.step(w, p, X, Xh, S, G, 0.1, 0.2, t)
+            ch.sgd_step(dX, dXh, dS, _dev(G), 0.1, 0.2)
+            torch.cuda.synchronize()
+            check_messages(ch.ctx, "topk", msgs, d)
+            assert_state(_host(dX, d), X, f"X after step {t}")
+            assert_state(_host(dS, d), S, f"S after step {t}")
+        st = choco.choco_get_stats(ch.ctx)
+        assert st["prepared_rows"] >= n * 6, st   # steps that did not follow a switch used carried candidates
+    finally:
+        ch.close()
+
+
 @pytest.mark.parametrize("blocks", [2, 4])
 def test_ties_with_a_cluster_of_blocks_per_row(blocks):
     """Ties at the k-th key that straddle the blocks' shares: rows of few distinct magnitudes."""
