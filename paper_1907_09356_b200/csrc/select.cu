@@ -411,9 +411,10 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
     bool aim_in_bin = false;
     const uint64_t aim_want = (uint64_t)k * kAimAfterMiss / 256u;
     const uint32_t aim_rank = (uint32_t)(aim_want < (uint64_t)dv.d ? aim_want : (uint64_t)dv.d);
-    const int shifts[3] = {21, 10, 0};
-    const int nbins[3] = {2048, 2048, 1024};
     for (int pass = 0; pass < 3; ++pass) {
+        // digits of 11, 11 and 10 bits from the top (plain selects: arrays indexed by the pass would live on a stack)
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const int bins = pass == 2 ? 1024 : 2048;
         for (int b = threadIdx.x; b < kHistBins; b += NT) h[b] = 0u;
         __syncthreads();
         for (int64_t c = (int64_t)threadIdx.x * kQuad; c < dv.d; c += span) {
@@ -423,30 +424,30 @@ __device__ __forceinline__ void exact_row(const Dev& dv, const StepArgs& a, int 
             for (int e = 0; e < 4; ++e) {
                 const uint32_t key = order_key<KIND>(bits[e]);
                 if (c + e < dv.d && (key & pmask) == prefix)
-                    atomicAdd(&h[(key >> shifts[pass]) & (nbins[pass] - 1)], 1u);
+                    atomicAdd(&h[(key >> shift) & (bins - 1)], 1u);
             }
         }
         __syncthreads();
         uint32_t digit, above;
-        block_find_digit<NT, kHistBins / NT>(h, nbins[pass], need, sm, &digit, &above);
+        block_find_digit<NT, kHistBins / NT>(h, bins, need, sm, &digit, &above);
         if (KIND == SEL_TOPK && pass == 0) {
             // a second point for the next step's bound: the eighth-of-an-octave bin that holds
             // the rank the bound aims at, and how many keys lie at or above its lower edge
             uint32_t d2, a2;
-            block_find_digit<NT, kHistBins / NT>(h, nbins[0], aim_rank, sm, &d2, &a2);
-            aim_lo = d2 << shifts[0];
+            block_find_digit<NT, kHistBins / NT>(h, 2048, aim_rank, sm, &d2, &a2);
+            aim_lo = d2 << 21;
             aim_count = a2 + h[d2];
             aim_in_bin = d2 == digit; // the same bin as rank k: the next pass resolves it further
             aim_above = above;
         } else if (KIND == SEL_TOPK && pass == 1 && aim_in_bin) {
             uint32_t d2, a2;
-            block_find_digit<NT, kHistBins / NT>(h, nbins[1], aim_rank - aim_above, sm, &d2, &a2);
-            aim_lo = prefix | (d2 << shifts[1]);
+            block_find_digit<NT, kHistBins / NT>(h, 2048, aim_rank - aim_above, sm, &d2, &a2);
+            aim_lo = prefix | (d2 << 10);
             aim_count = aim_above + a2 + h[d2];
         }
         need -= above;
-        prefix |= digit << shifts[pass];
-        pmask |= (uint32_t)(nbins[pass] - 1) << shifts[pass];
+        prefix |= digit << shift;
+        pmask |= (uint32_t)(bins - 1) << shift;
         __syncthreads();
     }
     const uint32_t T = prefix, r = need;
