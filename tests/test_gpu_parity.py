@@ -142,7 +142,8 @@ def test_identity_shapes(d, ld):
 
 @pytest.mark.parametrize("d,k,ld", [(1, 1, None), (31, 5, None), (33, 33, 36), (513, 1, None),
                                     (2000, 20, None), (4097, 300, 4100), (10007, 100, None),
-                                    (10007, 10007, None), (50000, 500, None)])
+                                    (10007, 10007, None), (50000, 500, None),
+                                    (100000, 10000, None), (100000, 50000, None)])   # Table 1's top-10 %, top-50 %
 def test_topk_shapes(d, k, ld):
     ch, _, _ = run_lockstep(workloads.ring(5), "topk", 5, d, 3, k=k, ld=ld, seed=d + k)
     assert choco.choco_message_bytes(ch.ctx) == (8 * k, 8 * k * 5)
@@ -150,7 +151,8 @@ def test_topk_shapes(d, k, ld):
 
 
 @pytest.mark.parametrize("d,k,ld", [(1, 1, None), (33, 7, 36), (2000, 20, None), (4097, 300, None),
-                                    (10007, 100, None), (10007, 10007, None), (50000, 5000, None)])
+                                    (10007, 100, None), (10007, 10007, None), (50000, 5000, None),
+                                    (100000, 50000, None)])                          # Table 1's random-50 %
 def test_randk_shapes(d, k, ld):
     ch, _, _ = run_lockstep(workloads.ring(5), "randk", 5, d, 3, k=k, ld=ld, seed=d + k)
     assert choco.choco_message_bytes(ch.ctx) == (4 * k, 4 * k * 5)

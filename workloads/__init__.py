@@ -334,6 +334,23 @@ WORKLOADS = {
                              gamma=0.4, steps=100, x_var=0.01, g_var=1e-3),
 }
 
+# The operator settings of Table 1 on its shape (8-ring, ResNet-20-sized vector), each with the
+# consensus stepsize Table 4 lists for it.  QSGD with b bits has s = 2^(b-1) levels; the 16-bit row
+# is beyond the level fields of this library (s <= 128).  Scaled sign is c3_ring8_sign.
+for _name, _q, _kw, _gamma in [
+    ("t1_ring8_qsgd8", "qsgd", dict(s=128, bucket=512), 0.2),
+    ("t1_ring8_qsgd4", "qsgd", dict(s=8, bucket=512), 0.075),
+    ("t1_ring8_qsgd2", "qsgd", dict(s=2, bucket=512), 0.025),
+    ("t1_ring8_rand50", "randk", dict(k=k_of(1, 2, 272474)), 0.45),
+    ("t1_ring8_rand10", "randk", dict(k=k_of(1, 10, 272474)), 0.075),
+    ("t1_ring8_rand1", "randk", dict(k=k_of(1, 100, 272474)), 0.00625),
+    ("t1_ring8_top50", "topk", dict(k=k_of(1, 2, 272474)), 0.45),
+    ("t1_ring8_top10", "topk", dict(k=k_of(1, 10, 272474)), 0.15),
+    ("t1_ring8_top1", "topk", dict(k=k_of(1, 100, 272474)), 0.0375),
+]:
+    WORKLOADS[_name] = Workload(_name, 8, 272474, "ring", _q, eta=0.1, gamma=_gamma, steps=1000,
+                                x_var=0.01, g_var=1e-2, g_mean_var=1e-3, **_kw)
+
 
 # --------------------------------------------------------------------------
 # the convex problem of the d = 2000 workload (caller-side gradient of Algorithm 1)
