@@ -472,6 +472,8 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
             // the cluster kernel gathers tile by tile: the update kernel may then place a tile's
             // candidates in the tile's own slot instead of reserving room with an atomic add
             dv.cand_slot = (p->kind == CHOCO_Q_TOPK && dv.emit_cluster > 1) ? dv.cand_slot_alloc : 0u;
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.spill_key, n * dv.cand_pitch);
+            if (e == cudaSuccess) e = dev_alloc(ctx, &dv.spill_idx, n * dv.cand_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_a, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_b, n * dv.slab_pitch);
             if (e == cudaSuccess) e = dev_alloc(ctx, &dv.slab_c, n * dv.slab_pitch);

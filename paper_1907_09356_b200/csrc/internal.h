@@ -84,6 +84,8 @@ struct Dev {
     uint32_t cand_slot;          // slot per tile in use, or 0
     uint32_t cand_slot_alloc;    // slot per tile the arrays were sized for
     uint32_t* row_ovf;           // [n] candidates placed behind the slots
+    uint32_t* spill_key;         // [n, cand_pitch] a row's candidates in tile order, for the cluster kernel
+    uint32_t* spill_idx;         //                 when a block's share does not fit its shared memory
     uint32_t* seg_off;           // [n, ntiles] first candidate of a tile
     uint32_t* seg_cnt;           // [n, ntiles]
     uint32_t* tile_a;            // [n, ntiles] scratch

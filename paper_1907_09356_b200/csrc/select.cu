@@ -801,9 +801,15 @@ __host__ __device__ inline int64_t cluster_emit_words(int64_t cap_local)
     const int64_t spitch = ((cap_local >> 5) + 2 + 3) & ~(int64_t)3;
     return 2 * cap_local + 4 * spitch + 3 * (kSelThreads + 4) + 2 * kListCap;
 }
+// the same with the keys and coordinates of the block's `len` candidates in global memory
+__host__ __device__ inline int64_t cluster_spill_words(int64_t len)
+{
+    const int64_t spitch = ((len >> 5) + 2 + 3) & ~(int64_t)3;
+    return 4 * spitch + 3 * (kSelThreads + 4) + 2 * kListCap;
+}
 
 template <int KIND, bool VEC>
-__global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepArgs a, int fused, int rescue)
+__global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepArgs a, int fused, int rescue, uint32_t dyn_bytes)
 {
     extern __shared__ __align__(16) uint32_t dyn[];
     __shared__ uint32_t h2[2][kHistBins]; // this block's histogram of the current / the previous round
@@ -856,10 +862,20 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
         if (threadIdx.x == 0 && carry != ncand) part_p[1] = 0xFFFFFFFFu; // inconsistent counts: do not trust the runs
         __syncthreads();
     }
+    // A block keeps its run's keys and coordinates in shared memory if every block's run fits
+    // there; otherwise in the row's part of two global arrays, as long as the per-slab arrays of
+    // the longest run still fit (the same algorithm either way).
     const int64_t cap_local = dv.emit_cap_local;
     bool fits = !unusable;
-    for (uint32_t c = 0; c < C && fits; ++c)
-        fits = part_p[c + 1] >= part_p[c] && (int64_t)(part_p[c + 1] - part_p[c]) <= cap_local;
+    uint32_t longest = 0;
+    for (uint32_t c = 0; c < C && fits; ++c) {
+        fits = part_p[c + 1] >= part_p[c];
+        const uint32_t len = part_p[c + 1] - part_p[c];
+        longest = len > longest ? len : longest;
+    }
+    const bool in_smem = fits && (int64_t)longest <= cap_local;
+    if (fits && !in_smem)
+        fits = dv.spill_key != nullptr && cluster_spill_words((int64_t)longest) * 4 <= (int64_t)dyn_bytes;
     // Every block has now read the row's state; none has changed it yet.  Only behind this
     // barrier may block 0 go its own way (it rewrites the row's flags and counts), so that all
     // blocks reach the same verdict from the same values.
@@ -874,10 +890,11 @@ __global__ void __launch_bounds__(kSelThreads) emit_cluster_kernel(Dev dv, StepA
     }
 
     // carve the dynamic shared memory
-    const int64_t spitch = ((cap_local >> 5) + 2 + 3) & ~(int64_t)3;
-    uint32_t* keys = dyn;                       // value bits of this block's candidates, in tile order
-    uint32_t* idxs = keys + cap_local;          // their coordinates
-    uint32_t* slab_g = idxs + cap_local;        // per slab: keys above T (then: before the slab)
+    const int64_t spitch = (((in_smem ? cap_local : (int64_t)longest) >> 5) + 2 + 3) & ~(int64_t)3;
+    const int64_t spill_at = (int64_t)row * dv.cand_pitch + part_p[rank];
+    uint32_t* keys = in_smem ? dyn : dv.spill_key + spill_at;             // value bits of this block's candidates, in tile order
+    uint32_t* idxs = in_smem ? keys + cap_local : dv.spill_idx + spill_at; // their coordinates
+    uint32_t* slab_g = in_smem ? idxs + cap_local : dyn;                   // per slab: keys above T (then: before the slab)
     uint32_t* slab_e = slab_g + spitch;         //           keys equal to T
     uint32_t* slab_gm = slab_e + spitch;        //           ballots of the two
     uint32_t* slab_em = slab_gm + spitch;
@@ -1190,7 +1207,7 @@ static cudaError_t emit_impl(const Dev& dv, const StepArgs& a, bool fused, int r
             cfg.numAttrs = 3;
         }
         cfg.attrs = attr;
-        e = cudaLaunchKernelEx(&cfg, kern, dv, a, fused ? 1 : 0, rescue);
+        e = cudaLaunchKernelEx(&cfg, kern, dv, a, fused ? 1 : 0, rescue, (uint32_t)bytes);
         if (e != cudaSuccess) return e;
         *a.launches += 1;
         return cudaGetLastError();
