@@ -231,7 +231,8 @@ float oracle_qsgd_tau(int64_t len, int32_t s)
     return (float)(1.0 + (a < b ? a : b));
 }
 
-/* width of the stored level field: smallest of 1, 2, 4, 8 bits holding 0..s-1 */
+/* width of the stored level field: smallest of 1, 2, 4, 8, 16 bits holding 0..s-1 (b = 16 bits
+ * per coordinate, the first QSGD row of Table 1, is s = 2^15 with 16-bit fields) */
 int32_t oracle_qsgd_level_bits(int32_t s)
 {
     int32_t w = 1;
@@ -253,13 +254,14 @@ int32_t oracle_qsgd_level_bits(int32_t s)
  *   - q = (nu / (tau * s)) * level, negated where v < 0 (sig(0) = +1).
  * Message per row: float32 nu per block, one sign bit per coordinate (as for sign),
  * and the levels in fields of oracle_qsgd_level_bits(s) bits, coordinate c at bit
- * offset c * width, least significant first.
+ * offset c * width, least significant first (s <= 32768: fields of at most 16 bits).
  */
 int oracle_compress_qsgd(const float* v, const float* u, int64_t d, int32_t s, int64_t bucket,
                          int32_t biased, float* norms, uint32_t* signbits, uint8_t* levels,
                          float* q)
 {
     if (bucket <= 0) bucket = d;
+    if (s < 2 || s > 32768) return -1;
     int32_t wbits = oracle_qsgd_level_bits(s);
     int64_t nwords = (d + 31) / 32;
     int64_t nbytes = (d * wbits + 7) / 8;
@@ -286,6 +288,7 @@ int oracle_compress_qsgd(const float* v, const float* u, int64_t d, int32_t s, i
             if (neg) signbits[c / 32] |= 1u << (c % 32);
             int64_t bit = c * wbits;
             levels[bit / 8] |= (uint8_t)(level << (bit % 8));
+            if (wbits == 16) levels[bit / 8 + 1] = (uint8_t)(level >> 8); /* little-endian field */
             float mag = scale * (float)level;
             q[c] = neg ? -mag : mag;
         }

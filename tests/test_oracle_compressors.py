@@ -256,10 +256,17 @@ _HAND_V = np.array([1, -2, 2, 0, 0, 0, 0, 0, 0, 4], dtype=np.float32)
     (4, 0.0, [0, 1, 1, 0, 0, 0, 0, 0, 0, 3], [0b00010100, 0, 0b1100]),
     # s = 128, 8-bit fields: 25.6 51.2 51.2 0 ... 102.4 -> one byte per coordinate
     (128, 0.0, [25, 51, 51, 0, 0, 0, 0, 0, 0, 102], [25, 51, 51, 0, 0, 0, 0, 0, 0, 102]),
+    # s = 2^15 (16 bits per coordinate with the sign: Table 1's first QSGD row), 16-bit fields,
+    # low byte first: 6553.6 13107.2 13107.2 0 ... 26214.4 -> 0x1999 0x3333 0x3333 0 ... 0x6666
+    (32768, 0.0, [6553, 13107, 13107, 0, 0, 0, 0, 0, 0, 26214],
+     [0x99, 0x19, 0x33, 0x33, 0x33, 0x33] + [0] * 12 + [0x66, 0x66]),
+    # u = 1/2 moves 6553.6 and 26214.4 up by one, 13107.2 stays, zeros stay
+    (32768, 0.5, [6554, 13107, 13107, 0, 0, 0, 0, 0, 0, 26214],
+     [0x9A, 0x19, 0x33, 0x33, 0x33, 0x33] + [0] * 12 + [0x66, 0x66]),
 ])
 def test_qsgd_level_fields_by_hand(s, u, levels, packed):
-    """Level fields of 1, 2 and 8 bits written out by hand (Appendix C: a level is an integer
-    in {0..s-1}; stored in the smallest of 1, 2, 4, 8 bits, coordinate c at bit c * width)."""
+    """Level fields of 1, 2, 8 and 16 bits written out by hand (Appendix C: a level is an integer
+    in {0..s-1}; stored in the smallest of 1, 2, 4, 8, 16 bits, coordinate c at bit c * width)."""
     m = oracle.compress_qsgd(_HAND_V, np.full(10, u, np.float32), s=s, bucket=0, biased=False)
     assert m.norms[0] == np.float32(5.0)
     assert list(m.levels) == packed
@@ -273,7 +280,7 @@ def test_qsgd_tau_values():
     assert float(oracle.qsgd_tau(512, 16)) == pytest.approx(1 + np.sqrt(512) / 16, rel=1e-7)
     assert float(oracle.qsgd_tau(40, 16)) == pytest.approx(1.15625, rel=1e-7)
     assert float(oracle.qsgd_tau(2000, 16)) == pytest.approx(1 + np.sqrt(2000) / 16, rel=1e-7)
-    assert [oracle.qsgd_level_bits(s) for s in (2, 4, 8, 16, 32, 128)] == [1, 2, 4, 4, 8, 8]
+    assert [oracle.qsgd_level_bits(s) for s in (2, 4, 8, 16, 32, 128, 256, 32768)] == [1, 2, 4, 4, 8, 8, 8, 16]
 
 
 def test_qsgd_one_hot_saturates():
