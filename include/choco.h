@@ -93,7 +93,8 @@ typedef enum {
 
 typedef struct {
     int32_t kind;        /* choco_q_kind                                                       */
-    int32_t s;           /* QSGD: number of levels 2^(b-1), a power of two in [2, 128]         */
+    int32_t s;           /* QSGD: number of levels 2^(b-1), a power of two in [2, 32768]; the  */
+                         /*       level of a coordinate is stored in 1, 2, 4, 8 or 16 bits     */
     int32_t bucket;      /* QSGD: block length for the norm; 0 = whole row, else a power of    */
                          /*       two in [128, 1024] (the last block of a row may be shorter)  */
     int32_t qsgd_biased; /* QSGD: 1 = divide by tau = 1 + min(len/s^2, sqrt(len)/s) (the       */

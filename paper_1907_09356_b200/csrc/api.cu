@@ -322,7 +322,7 @@ int choco_init(choco_ctx** out, int32_t n, int64_t d, int64_t ld, const int32_t*
         if (p->k < 1 || p->k > d) return CHOCO_ERR_INVALID_ARG;
         break;
     case CHOCO_Q_QSGD:
-        if (!is_pow2(p->s) || p->s < 2 || p->s > 128) return CHOCO_ERR_INVALID_ARG;
+        if (!is_pow2(p->s) || p->s < 2 || p->s > 32768) return CHOCO_ERR_INVALID_ARG;
         if (p->bucket < 0) return CHOCO_ERR_INVALID_ARG;
         if (p->bucket != 0 && !(is_pow2(p->bucket) && p->bucket >= 128 && p->bucket <= 1024))
             return CHOCO_ERR_UNSUPPORTED;

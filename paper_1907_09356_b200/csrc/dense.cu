@@ -5,7 +5,7 @@
 // Message layout per worker (row):
 //   sign     : sign plane u32[ceil(d/32)], bit c%32 of word c/32 set iff v_c < 0, tail bits 0;
 //              scale f32 = ||v||_1 / d.
-//   qsgd     : block norms f32[blocks]; the same sign plane; level fields of `wbits` bits,
+//   qsgd     : block norms f32[blocks]; the same sign plane; level fields of `wbits` (1..16) bits,
 //              coordinate c at bit offset c * wbits, least significant first.
 //   identity : f32[d].
 #include "common.cuh"
@@ -169,7 +169,10 @@ __global__ void __launch_bounds__(kThreads) qsgd_pack_kernel(Dev dv, StepArgs a)
         const uint32_t word = gather_sign_word(sign_nibble(v[it]), lane);
         if ((lane & 7) == 0 && c < dv.d) dv.msg_bits[(int64_t)row * dv.wpitch + (c >> 5)] = word;
         uint8_t* lrow = dv.msg_levels + (int64_t)row * dv.lpitch;
-        if (WBITS == 8) {
+        if (WBITS == 16) {
+            if (c < dv.d)
+                *reinterpret_cast<uint2*>(lrow + 2 * c) = make_uint2(lev[0] | (lev[1] << 16), lev[2] | (lev[3] << 16));
+        } else if (WBITS == 8) {
             if (c < dv.d)
                 *reinterpret_cast<uint32_t*>(lrow + c) = lev[0] | (lev[1] << 8) | (lev[2] << 16) | (lev[3] << 24);
         } else if (WBITS == 4) {
@@ -237,7 +240,8 @@ static cudaError_t compress_impl(const Dev& dv, const StepArgs& a, cudaStream_t 
         case 1: launch_qsgd_pack<VEC, 1>(dv, a, grid, st); break;
         case 2: launch_qsgd_pack<VEC, 2>(dv, a, grid, st); break;
         case 4: launch_qsgd_pack<VEC, 4>(dv, a, grid, st); break;
-        default: launch_qsgd_pack<VEC, 8>(dv, a, grid, st); break;
+        case 8: launch_qsgd_pack<VEC, 8>(dv, a, grid, st); break;
+        default: launch_qsgd_pack<VEC, 16>(dv, a, grid, st); break;
         }
         *a.launches += 1;
         break;

@@ -59,6 +59,15 @@ __device__ __forceinline__ float4 decode_quad(const Dev& dv, int j, int64_t c)
         const float scale = __fdiv_rn(nu, __fmul_rn(tail ? dv.tau_tail : dv.tau_full, (float)dv.s));
         const uint8_t* lrow = dv.msg_levels + (int64_t)j * dv.lpitch;
         uint32_t packed, width = (uint32_t)dv.wbits;
+        if (width == 16) { // two 32-bit words hold the four fields
+            const uint2 two = __ldg(reinterpret_cast<const uint2*>(lrow + 2 * c));
+            m[0] = __fmul_rn(scale, (float)(two.x & 0xFFFFu));
+            m[1] = __fmul_rn(scale, (float)(two.x >> 16));
+            m[2] = __fmul_rn(scale, (float)(two.y & 0xFFFFu));
+            m[3] = __fmul_rn(scale, (float)(two.y >> 16));
+            return make_float4(nib & 1u ? -m[0] : m[0], nib & 2u ? -m[1] : m[1], nib & 4u ? -m[2] : m[2],
+                               nib & 8u ? -m[3] : m[3]);
+        }
         if (width == 8) packed = __ldg(reinterpret_cast<const uint32_t*>(lrow + c));
         else if (width == 4) packed = __ldg(reinterpret_cast<const uint16_t*>(lrow + (c >> 1)));
         else if (width == 2) packed = __ldg(lrow + (c >> 2));
@@ -194,7 +203,10 @@ __global__ void __launch_bounds__(kThreads, 4) update_dense_kernel(Dev dv, StepA
             lev[e] = (uint32_t)l;
         }
         uint8_t* lrow = dv.nxt_levels + (int64_t)row * dv.lpitch;
-        if (dv.wbits == 8) {
+        if (dv.wbits == 16) {
+            if (c < dv.d)
+                *reinterpret_cast<uint2*>(lrow + 2 * c) = make_uint2(lev[0] | (lev[1] << 16), lev[2] | (lev[3] << 16));
+        } else if (dv.wbits == 8) {
             if (c < dv.d)
                 *reinterpret_cast<uint32_t*>(lrow + c) = lev[0] | (lev[1] << 8) | (lev[2] << 16) | (lev[3] << 24);
         } else if (dv.wbits == 4) {

@@ -318,26 +318,34 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
                 } else {
                     const int b = li >> dv.bucket_shift; // block of the norm: the same for the whole warp
                     const unsigned char* lev = slice + L::kBitsTile;
-                    uint32_t packed;
-                    if (WBITS == 8) packed = reinterpret_cast<const uint32_t*>(lev)[q4];
+                    uint32_t packed, packed_hi = 0u; // the quad's four fields (16-bit fields: two words)
+                    if (WBITS == 16) {
+                        const uint2 two = reinterpret_cast<const uint2*>(lev)[q4];
+                        packed = two.x;
+                        packed_hi = two.y;
+                    } else if (WBITS == 8) packed = reinterpret_cast<const uint32_t*>(lev)[q4];
                     else if (WBITS == 4) packed = reinterpret_cast<const uint16_t*>(lev)[q4];
                     else if (WBITS == 2) packed = lev[q4];
                     else packed = (uint32_t)(lev[q4 >> 1] >> (li & 4));
                     constexpr uint32_t mask = (1u << (WBITS > 0 ? WBITS : 1)) - 1u;
+                    auto field = [&](int e) -> uint32_t {
+                        if constexpr (WBITS == 16) return ((e < 2 ? packed : packed_hi) >> ((e & 1) * 16)) & mask;
+                        else return (packed >> (e * WBITS)) & mask;
+                    };
                     const float* t = tab + (r * nbk + b) * kTabLevels;
                     if (L::kTable) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) q[e] = with_sign(t[(packed >> (e * WBITS)) & mask], nib, e);
+                        for (int e = 0; e < 4; ++e) q[e] = with_sign(t[field(e)], nib, e);
                         if (self) {
                             const float* ts = tab_self + b * kTabLevels;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(ts[(packed >> (e * WBITS)) & mask], nib, e);
+                            for (int e = 0; e < 4; ++e) qs[it][e] = with_sign(ts[field(e)], nib, e);
                         }
                     } else {
                         const float mag = t[0], w = t[1];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float m = __fmul_rn(mag, small_uint_to_float((packed >> (e * WBITS)) & mask));
+                            const float m = __fmul_rn(mag, small_uint_to_float(field(e)));
                             if (self) qs[it][e] = with_sign(m, nib, e);
                             q[e] = with_sign(__fmul_rn(w, m), nib, e);
                         }
@@ -469,7 +477,10 @@ __device__ __forceinline__ void update_dense_bulk_body(const Dev& dv, const Step
             lv[e] = __float_as_uint(__fadd_rd(t, 8388608.f));
         }
         constexpr uint32_t kMagic = 0x4B000000u;
-        if (WBITS == 8) {
+        if (WBITS == 16) {
+            reinterpret_cast<uint2*>(lev_out)[q4] = make_uint2((lv[1] * 65536u + lv[0]) - kMagic * 0x00010001u,
+                                                               (lv[3] * 65536u + lv[2]) - kMagic * 0x00010001u);
+        } else if (WBITS == 8) {
             reinterpret_cast<uint32_t*>(lev_out)[q4] =
                 (((lv[3] * 256u + lv[2]) * 256u + lv[1]) * 256u + lv[0]) - kMagic * 0x01010101u;
         } else if (WBITS == 4) {
@@ -582,7 +593,8 @@ cudaError_t launch_layers_kind(const Dev& proto, const LayerTable& tab, const La
     case 1: return launch_layers_terms<CHOCO_Q_QSGD, 1, AL>(proto, tab, ls, a, st);
     case 2: return launch_layers_terms<CHOCO_Q_QSGD, 2, AL>(proto, tab, ls, a, st);
     case 4: return launch_layers_terms<CHOCO_Q_QSGD, 4, AL>(proto, tab, ls, a, st);
-    default: return launch_layers_terms<CHOCO_Q_QSGD, 8, AL>(proto, tab, ls, a, st);
+    case 8: return launch_layers_terms<CHOCO_Q_QSGD, 8, AL>(proto, tab, ls, a, st);
+    default: return launch_layers_terms<CHOCO_Q_QSGD, 16, AL>(proto, tab, ls, a, st);
     }
 }
 
@@ -633,7 +645,8 @@ cudaError_t launch_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
     case 1: return launch_terms<CHOCO_Q_QSGD, 1, EMIT, AL>(dv, a, st);
     case 2: return launch_terms<CHOCO_Q_QSGD, 2, EMIT, AL>(dv, a, st);
     case 4: return launch_terms<CHOCO_Q_QSGD, 4, EMIT, AL>(dv, a, st);
-    default: return launch_terms<CHOCO_Q_QSGD, 8, EMIT, AL>(dv, a, st);
+    case 8: return launch_terms<CHOCO_Q_QSGD, 8, EMIT, AL>(dv, a, st);
+    default: return launch_terms<CHOCO_Q_QSGD, 16, EMIT, AL>(dv, a, st);
     }
 }
 

@@ -129,10 +129,20 @@ def test_qsgd_shapes(d, ld, bucket):
     run_lockstep(workloads.ring(4), "qsgd", 4, d, 3, s=16, bucket=bucket, ld=ld, seed=d + bucket)[0].close()
 
 
-@pytest.mark.parametrize("s", [2, 4, 8, 32, 128])
+@pytest.mark.parametrize("s", [2, 4, 8, 32, 128, 256, 512, 32768])
 @pytest.mark.parametrize("biased", [True, False])
 def test_qsgd_level_counts(s, biased):
     run_lockstep(workloads.ring(4), "qsgd", 4, 3000, 2, s=s, bucket=256, biased=biased, seed=s)[0].close()
+
+
+@pytest.mark.parametrize("d,ld,bucket", [(4096, None, 512), (5002, None, 128), (5001, None, 512), (3000, None, 0)],
+                         ids=["aligned", "8-byte rows", "odd rows", "whole-row norm"])
+def test_qsgd_sixteen_bit_levels(d, ld, bucket):
+    """s = 2^15 (Table 1's 16-bit row): 16-bit level fields through every kernel that packs or
+    reads them, several steps so that carried messages are decoded too, with momentum once."""
+    w = workloads.ring(5)
+    run_lockstep(w, "qsgd", 5, d, 4, s=32768, bucket=bucket, seed=d, ld=ld)[0].close()
+    run_lockstep(w, "qsgd", 5, d, 3, s=32768, bucket=bucket, seed=d + 1, ld=ld, momentum=True)[0].close()
 
 
 @pytest.mark.parametrize("d,ld", SHAPES)

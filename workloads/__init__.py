@@ -335,9 +335,10 @@ WORKLOADS = {
 }
 
 # The operator settings of Table 1 on its shape (8-ring, ResNet-20-sized vector), each with the
-# consensus stepsize Table 4 lists for it.  QSGD with b bits has s = 2^(b-1) levels; the 16-bit row
-# is beyond the level fields of this library (s <= 128).  Scaled sign is c3_ring8_sign.
+# consensus stepsize Table 4 lists for it.  QSGD with b bits has s = 2^(b-1) levels.  Scaled sign
+# is c3_ring8_sign.
 for _name, _q, _kw, _gamma in [
+    ("t1_ring8_qsgd16", "qsgd", dict(s=32768, bucket=512), 0.2),
     ("t1_ring8_qsgd8", "qsgd", dict(s=128, bucket=512), 0.2),
     ("t1_ring8_qsgd4", "qsgd", dict(s=8, bucket=512), 0.075),
     ("t1_ring8_qsgd2", "qsgd", dict(s=2, bucket=512), 0.025),
