@@ -25,6 +25,7 @@ KINDS = [
     ("qsgd", dict(s=16, bucket=512)),
     ("qsgd", dict(s=4, bucket=0)),
     ("identity", dict()),
+    ("qsgd", dict(s=32768, bucket=256)),             # 16-bit level fields
 ]
 
 
