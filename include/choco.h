@@ -163,7 +163,11 @@ int choco_set_nesterov(choco_ctx* ctx, int32_t enable);
  * choco_sgd_step_host -- the same step as choco_sgd_step on HOST arrays (pageable or
  * pinned): copies X, Xhat, S, G to library-owned device staging buffers (allocated on the
  * first such call), runs the step, copies X, Xhat, S back and synchronises `stream` before
- * returning.  G may be NULL for a gossip-only step.
+ * returning.  G may be NULL for a gossip-only step.  The copies run on two streams of the
+ * context beside `stream` (created on the first such call; they start after what `stream` holds
+ * at the call and `stream` waits for them): all of X and Xhat first, then S and G in eight chunks
+ * of rows, each chunk updated as soon as it has arrived and copied back while the next ones are
+ * still on their way, so that with pinned host arrays the link carries both directions at once.
  */
 int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G,
                         float eta, float gamma, void* stream);

@@ -109,8 +109,16 @@ __global__ void bump_step_kernel(unsigned long long* step) { *step += 1ull; }
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
 
+// The update of a step in chunks of rows (choco_sgd_step_host): chunk c waits for `ready[c]` and
+// records `done[c]` on the step's stream.
+struct RowChunks {
+    int count, rows_per_chunk;
+    cudaEvent_t* ready;
+    cudaEvent_t* done;
+};
+
 int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, float* M, float eta,
-              float gamma, float lambda, float beta, void* stream)
+              float gamma, float lambda, float beta, void* stream, const RowChunks* chunks = nullptr)
 {
     if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
     if (ctx->timed_out) return CHOCO_ERR_TIMEOUT; // the arrays are no valid state any more
@@ -150,7 +158,19 @@ int step_body(choco_ctx* ctx, float* X, float* Xhat, float* S, const float* G, f
     const bool prof = ctx->prof_ev && ctx->prof_n < ctx->prof_cap &&
                       (ctx->prof_stride <= 1 || ctx->steps_enqueued % (uint64_t)ctx->prof_stride == 0);
     if (e == cudaSuccess && prof) e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], st);
-    if (e == cudaSuccess) e = launch_apply(dv, a, emit, st);
+    if (chunks) {
+        for (int c = 0; c < chunks->count && e == cudaSuccess; ++c) {
+            a.row0 = c * chunks->rows_per_chunk;
+            a.rows = std::min(chunks->rows_per_chunk, dv.n - a.row0);
+            e = cudaStreamWaitEvent(st, chunks->ready[c], 0);
+            if (e == cudaSuccess) e = launch_apply(dv, a, emit, st);
+            if (e == cudaSuccess) e = cudaEventRecord(chunks->done[c], st);
+        }
+        a.row0 = 0;
+        a.rows = 0;
+    } else if (e == cudaSuccess) {
+        e = launch_apply(dv, a, emit, st);
+    }
     if (e == cudaSuccess && prof) {
         e = cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], st);
         ctx->prof_n += 1;
@@ -543,6 +563,12 @@ int choco_destroy(choco_ctx* ctx)
     for (int i = 0; i < ctx->nallocs; ++i) cudaFree(ctx->allocs[i]);
     for (int i = 0; i < 4; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    if (ctx->host_in) {
+        cudaStreamDestroy(ctx->host_in);
+        cudaStreamDestroy(ctx->host_out);
+        for (cudaEvent_t ev : ctx->host_ev)
+            if (ev) cudaEventDestroy(ev);
+    }
     if (ctx->prof_ev) {
         for (int i = 0; i < 2 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
         delete[] ctx->prof_ev;
@@ -576,32 +602,74 @@ int choco_sgd_step_host(choco_ctx* ctx, float* X, float* Xhat, float* S, const f
 {
     if (!ctx || !X || !Xhat || !S) return CHOCO_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t bytes = (size_t)ctx->dv.n * (size_t)ctx->dv.ld * sizeof(float);
+    const int n = ctx->dv.n;
+    const size_t row_bytes = (size_t)ctx->dv.ld * sizeof(float);
+    const size_t bytes = (size_t)n * row_bytes;
     for (int i = 0; i < 4; ++i)
         if (!ctx->stage[i]) {
             cudaError_t e = cudaMalloc((void**)&ctx->stage[i], bytes);
             if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CHOCO_ERR_ALLOC; }
         }
-    const float* src[4] = {X, Xhat, S, G};
-    for (int i = 0; i < 4; ++i) {
-        if (!src[i]) continue;
-        cudaError_t e = cudaMemcpyAsync(ctx->stage[i], src[i], bytes, cudaMemcpyHostToDevice, st);
+    if (!ctx->host_in) {
+        cudaError_t e = cudaStreamCreateWithFlags(&ctx->host_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->host_out, cudaStreamNonBlocking);
+        for (cudaEvent_t& ev : ctx->host_ev)
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
+    // Uploads on one stream, downloads on another, kernels on the caller's: the messages need all
+    // of X and X^, but a row's update needs only its own s and g, and its results can leave while
+    // later rows are still being uploaded and updated (the link carries both directions at once).
+    cudaEvent_t fork = ctx->host_ev[0], xh_in = ctx->host_ev[1], join = ctx->host_ev[2];
+    cudaEvent_t* ready = ctx->host_ev + 3;
+    cudaEvent_t* done = ready + kHostChunks;
+    RowChunks chunks;
+    chunks.rows_per_chunk = (n + kHostChunks - 1) / kHostChunks;
+    chunks.count = (n + chunks.rows_per_chunk - 1) / chunks.rows_per_chunk;
+    chunks.ready = ready;
+    chunks.done = done;
+    auto rows_of = [&](int c, size_t* off, size_t* len) {
+        const int r0 = c * chunks.rows_per_chunk, cnt = std::min(chunks.rows_per_chunk, n - r0);
+        *off = (size_t)r0 * (size_t)ctx->dv.ld; // in floats
+        *len = (size_t)cnt * row_bytes;          // in bytes
+    };
+    cudaError_t e = cudaEventRecord(fork, st);   // what the caller enqueued before comes first
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_in, fork, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_out, fork, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage[0], X, bytes, cudaMemcpyHostToDevice, ctx->host_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage[1], Xhat, bytes, cudaMemcpyHostToDevice, ctx->host_in);
+    if (e == cudaSuccess) e = cudaEventRecord(xh_in, ctx->host_in);
+    for (int c = 0; c < chunks.count && e == cudaSuccess; ++c) {
+        size_t off, len;
+        rows_of(c, &off, &len);
+        e = cudaMemcpyAsync(ctx->stage[2] + off, S + off, len, cudaMemcpyHostToDevice, ctx->host_in);
+        if (e == cudaSuccess && G) e = cudaMemcpyAsync(ctx->stage[3] + off, G + off, len, cudaMemcpyHostToDevice, ctx->host_in);
+        if (e == cudaSuccess) e = cudaEventRecord(ready[c], ctx->host_in);
+    }
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, xh_in, 0);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->prepared = false; // the staging contents changed
     const bool carry = ctx->carry_enabled;
     ctx->carry_enabled = false; // the next call overwrites the staging buffers anyway
     const int rc = step_body(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], G ? ctx->stage[3] : nullptr,
-                            nullptr, eta, gamma, 0.f, 0.f, stream);
+                            nullptr, eta, gamma, 0.f, 0.f, stream, &chunks);
     ctx->carry_enabled = carry;
-    if (rc) return rc;
-    float* dst[3] = {X, Xhat, S};
-    for (int i = 0; i < 3; ++i) {
-        cudaError_t e = cudaMemcpyAsync(dst[i], ctx->stage[i], bytes, cudaMemcpyDeviceToHost, st);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (rc) {
+        cudaDeviceSynchronize(); // the side streams may still be copying
+        return rc;
     }
-    cudaError_t e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    float* dst[3] = {X, Xhat, S};
+    for (int c = 0; c < chunks.count && e == cudaSuccess; ++c) {
+        size_t off, len;
+        rows_of(c, &off, &len);
+        e = cudaStreamWaitEvent(ctx->host_out, done[c], 0);
+        for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+            e = cudaMemcpyAsync(dst[i] + off, ctx->stage[i] + off, len, cudaMemcpyDeviceToHost, ctx->host_out);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(join, ctx->host_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, join, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { cudaDeviceSynchronize(); return fail_cuda(ctx, e); }
     ctx->prepared = false;
     return check_device_timeouts(ctx, st);
 }

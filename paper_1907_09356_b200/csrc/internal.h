@@ -155,12 +155,16 @@ struct StepArgs {
     const unsigned long long* step_dev; // if set, the step number is read from here instead
     bool vec;                    // rows 16-byte aligned: 128-bit accesses
     unsigned long long* launches; // host counter of kernels enqueued (not used on the device)
+    // an update launch may serve the workers [row0, row0 + rows) only (rows == 0: all of them)
+    int32_t row0 = 0;
+    int32_t rows = 0;
 };
 
 // One launch over the tiles (or rows) of several layers of a layered context.  The table comes
 // as a kernel argument (constant memory): a block finds its entry by bisection over first_block
 // (launches over tiles) or as blockIdx.x / n (launches over rows) and can request its tiles at
 // once; the rest of the layer's parameters it reads from devs[layer[entry]] in device memory.
+constexpr int kHostChunks = 8;     // choco_sgd_step_host moves and updates the rows in this many chunks
 constexpr int kMaxComboLayers = 512;
 struct LayerTable {
     int32_t entries;                            // layers served by this launch
@@ -265,8 +269,11 @@ struct choco_ctx {
     bool timed_out;              // a synchronising call saw device_timeouts != 0: steps refuse
     uint64_t dv_epoch;           // bumped whenever a setter changes `dv` (a layered context keeps device copies)
     bool hot_l2;                 // the context asked for persisting L2 lines (reset on destroy)
-    // host staging for choco_sgd_step_host
+    // host staging for choco_sgd_step_host: device copies of X, X^, S, G; two streams that carry the
+    // uploads and the downloads beside the caller's stream; events that order them per chunk of rows
     float* stage[4];
+    cudaStream_t host_in, host_out;
+    cudaEvent_t host_ev[3 + 2 * choco::kHostChunks]; // fork, X and X^ uploaded, join; per chunk: uploaded, updated
     // consensus scratch
     double* cons_scratch;
     int64_t cons_blocks;

@@ -462,7 +462,7 @@ template <bool HAS_G, bool HAS_M, bool EMIT, bool AL>
 __global__ void __launch_bounds__(NT, 5) update_sparse_bulk_kernel(Dev dv, StepArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    update_sparse_bulk_body<HAS_G, HAS_M, EMIT, AL, false>(dv, a, (int64_t)blockIdx.x, (int)blockIdx.y, dv.d, dv.ld, smem_raw,
+    update_sparse_bulk_body<HAS_G, HAS_M, EMIT, AL, false>(dv, a, (int64_t)blockIdx.x, (int)blockIdx.y + a.row0, dv.d, dv.ld, smem_raw,
                                                           nullptr);
 }
 
@@ -526,7 +526,7 @@ cudaError_t launch_bulk(const Dev& dv, const StepArgs& a, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    const dim3 grid((unsigned)dv.ntiles, (unsigned)dv.n);
+    const dim3 grid((unsigned)dv.ntiles, (unsigned)(a.rows > 0 ? a.rows : dv.n));
     return launch_overlapped(update_sparse_bulk_kernel<HAS_G, HAS_M, EMIT, AL>, grid, dim3(NT), smem, st,
                              hot_range_of(dv), dv, a);
 }

@@ -90,7 +90,7 @@ template <bool VEC, int KIND, bool HAS_G, bool HAS_M, bool EMIT>
 __global__ void __launch_bounds__(kThreads, 4) update_dense_kernel(Dev dv, StepArgs a)
 {
     __shared__ float ws[kUpdIters][8];
-    const int row = blockIdx.y;
+    const int row = (int)blockIdx.y + a.row0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kUpdSpan;
     const int e0 = dv.row_ptr[row], e1 = dv.row_ptr[row + 1];
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(kThreads, 4) update_dense_kernel(Dev dv, StepA
 template <bool VEC, bool HAS_G, bool HAS_M, bool EMIT>
 void pick_kind(const Dev& dv, const StepArgs& a, cudaStream_t st)
 {
-    const dim3 grid((unsigned)((dv.d + kUpdSpan - 1) / kUpdSpan), (unsigned)dv.n);
+    const dim3 grid((unsigned)((dv.d + kUpdSpan - 1) / kUpdSpan), (unsigned)(a.rows > 0 ? a.rows : dv.n));
     switch (dv.kind) {
     case CHOCO_Q_SIGN:
         update_dense_kernel<VEC, CHOCO_Q_SIGN, HAS_G, HAS_M, EMIT><<<grid, kThreads, 0, st>>>(dv, a);

@@ -510,7 +510,7 @@ __global__ void __launch_bounds__(NT, MINB) update_dense_bulk_kernel(Dev dv, Ste
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1; // blocks of the norm per tile
     update_dense_bulk_body<KIND, WBITS, HAS_G, HAS_M, EMIT, AL, false>(dv, a, nb_stage, nbk, (int64_t)blockIdx.x,
-                                                                      (int)blockIdx.y, dv.d, dv.ld, smem_raw, nullptr);
+                                                                      (int)blockIdx.y + a.row0, dv.d, dv.ld, smem_raw, nullptr);
 }
 
 // several layers in one launch: blockIdx.x picks (layer, tile), blockIdx.y the worker
@@ -605,7 +605,7 @@ cudaError_t launch_one(const Dev& dv, const StepArgs& a, cudaStream_t st)
     const int nb_stage = dv.maxdeg < kBatch ? dv.maxdeg : kBatch;
     const int nbk = KIND == CHOCO_Q_QSGD ? (kDTile >> dv.bucket_shift) : 1;
     const size_t smem = (size_t)L::total(nb_stage, nbk);
-    const dim3 grid((unsigned)((dv.d + kDTile - 1) / kDTile), (unsigned)dv.n);
+    const dim3 grid((unsigned)((dv.d + kDTile - 1) / kDTile), (unsigned)(a.rows > 0 ? a.rows : dv.n));
     if constexpr (KIND == CHOCO_Q_SIGN) {
         // a grid of at most two waves: the time is a block's latency, not the SMs' throughput
         // (measured on 8 x 272 474: 0.0190 against 0.0206 ms per step; 32 x 272 474 prefers five)

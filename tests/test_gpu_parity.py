@@ -531,3 +531,32 @@ def test_host_buffer_entry_point():
         assert_state(Xh, oXh, "Xhat (host call)")
         assert_state(S, oS, "S (host call)")
     ch.close()
+
+
+@pytest.mark.parametrize("kind,kw,n", [("topk", dict(k=300), 19), ("sign", {}, 19), ("qsgd", dict(s=16, bucket=512), 8),
+                                       ("qsgd", dict(s=16, bucket=0), 3), ("randk", dict(k=300), 19),
+                                       ("identity", {}, 5)])
+def test_host_buffer_entry_point_in_chunks_of_rows(kind, kw, n):
+    """The host entry point uploads, updates and downloads the rows in eight chunks on three
+    streams: more rows than chunks (ragged last chunk), as many, fewer; pinned host arrays; every
+    operator's update kernel takes a row range."""
+    w = workloads.ring(n)
+    d = 30000
+    host = [torch.from_numpy(a).pin_memory() for a in
+            (workloads.normal_rows(n, d, 1.0, 1), np.zeros((n, d), np.float32), np.zeros((n, d), np.float32))]
+    X, Xh, S = (t.numpy() for t in host)
+    oX, oXh, oS = X.copy(), Xh.copy(), S.copy()
+    ch = choco.Choco(w, d, kind, seed=4, **kw)
+    p = oracle.Params(kind, seed=4, **kw)
+    st = torch.cuda.Stream()
+    try:
+        with torch.cuda.stream(st):
+            for t in range(3):
+                G = workloads.normal_rows(n, d, 0.01, 20 + t)
+                oracle.step(w, p, oX, oXh, oS, G, 0.1, 0.2, t)
+                choco.choco_sgd_step_host(ch.ctx, X, Xh, S, G, 0.1, 0.2)
+                assert_state(X, oX, f"X (host call {t})")
+                assert_state(Xh, oXh, f"Xhat (host call {t})")
+                assert_state(S, oS, f"S (host call {t})")
+    finally:
+        ch.close()
